@@ -1,0 +1,223 @@
+"""Seeded synthetic workloads: shapes, weight tensors and hidden-state streams.
+
+Every tensor is a pure function of (seed, tensor kind, layer, index) through numpy's
+counter-based Philox generator, so a single expert or a single decode step can be
+regenerated in isolation and two consumers always see identical bytes.
+
+Storage conventions produced here (they are data layouts, not arithmetic):
+
+* router weights      ``[N, H]`` row-major, one row per routed expert;
+* shared-gate vector  ``[H]``;
+* expert block        ``[I, 3, H]`` row-major: for intermediate index ``i`` the three
+  consecutive rows are ``W_gate[i, :]``, ``W_up[i, :]`` and ``W_down[:, i]`` (column ``i``
+  of the down projection), so that everything needed for one intermediate channel is one
+  contiguous run of ``3*H`` elements;
+* hidden states       ``[L, B, H]`` float32 per decode step.
+
+Element type is float32 (``weight_dtype == 0``) or bfloat16 stored as ``uint16`` bit
+patterns (``weight_dtype == 1``), rounded to nearest-even once, at generation.
+"""
+from __future__ import annotations
+
+from concurrent.futures import ThreadPoolExecutor
+from dataclasses import dataclass, asdict
+import os
+
+import numpy as np
+
+KIND_ROUTER = 1
+KIND_SHARED_GATE = 2
+KIND_EXPERT = 3
+KIND_SHARED = 4
+KIND_HIDDEN = 5
+KIND_RHO = 6
+
+EXPERT_STD = 0.02
+
+
+@dataclass(frozen=True)
+class Shape:
+    n_layers: int
+    hidden: int
+    n_routed: int
+    top_k: int
+    inter_routed: int
+    n_shared: int = 0
+    inter_shared: int = 0
+    shared_gate: int = 0      # 1: shared output scaled by sigmoid(w_sg . h)
+    renorm_topk: int = 0      # 1: top-k gate weights renormalised to sum to 1
+    weight_dtype: int = 0     # 0 float32, 1 bfloat16
+    batch: int = 1
+
+    def asdict(self):
+        return asdict(self)
+
+    @property
+    def elem_bytes(self) -> int:
+        return 2 if self.weight_dtype == 1 else 4
+
+
+# The five workloads; `rhos` lists the AR(1) coefficients swept for that workload
+# (None = one coefficient per sequence drawn U(0.3, 0.95) from the seed).
+CONFIGS = {
+    "tiny_fp32": dict(
+        shape=Shape(1, 256, 16, 2, 128, 0, 0, 0, 0, 0, 1),
+        cache_slots=4, steps=64, rhos=(0.9,), seed=0),
+    "dsv2lite": dict(
+        shape=Shape(26, 2048, 64, 6, 1408, 2, 1408, 0, 0, 1, 1),
+        cache_slots=16, steps=512, rhos=(0.0, 0.5, 0.9), seed=0),
+    "qwen15moe": dict(
+        shape=Shape(24, 2048, 60, 4, 1408, 1, 5632, 1, 0, 1, 1),
+        cache_slots=12, steps=512, rhos=(0.8,), seed=0),
+    "qwen3_30b": dict(
+        shape=Shape(48, 2048, 128, 8, 768, 0, 0, 0, 1, 1, 1),
+        cache_slots=32, steps=1024, rhos=(0.5, 0.9), seed=0),
+    "dsv2lite_b32": dict(
+        shape=Shape(26, 2048, 64, 6, 1408, 2, 1408, 0, 0, 1, 32),
+        cache_slots=32, steps=1024, rhos=(None,), seed=0),
+}
+
+
+def config(name: str) -> dict:
+    return dict(CONFIGS[name])
+
+
+def expert_block_elems(hidden: int, inter: int) -> int:
+    return 3 * hidden * inter
+
+
+def expert_block_bytes(shape: Shape, shared: bool = False) -> int:
+    inter = shape.inter_shared if shared else shape.inter_routed
+    return expert_block_elems(shape.hidden, inter) * shape.elem_bytes
+
+
+def bf16_round_to_bits(x: np.ndarray) -> np.ndarray:
+    """float32 -> bfloat16 bit patterns (uint16), round to nearest, ties to even."""
+    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
+    lsb = (u >> np.uint32(16)) & np.uint32(1)
+    return ((u + np.uint32(0x7FFF) + lsb) >> np.uint32(16)).astype(np.uint16)
+
+
+def bf16_bits_to_f32(bits: np.ndarray) -> np.ndarray:
+    """bfloat16 bit patterns (uint16) -> the float32 values they denote (exact)."""
+    return (bits.astype(np.uint32) << np.uint32(16)).view(np.float32)
+
+
+def _rng(seed: int, kind: int, a: int = 0, b: int = 0) -> np.random.Generator:
+    key = np.array([(int(seed) << 32) | int(kind), (int(a) << 32) | int(b)], dtype=np.uint64)
+    return np.random.Generator(np.random.Philox(key=key))
+
+
+def _store(x32: np.ndarray, weight_dtype: int, out: np.ndarray | None) -> np.ndarray:
+    if weight_dtype == 1:
+        bits = bf16_round_to_bits(x32)
+        if out is None:
+            return bits
+        out[...] = bits.reshape(out.shape)
+        return out
+    if out is None:
+        return x32
+    out[...] = x32.reshape(out.shape)
+    return out
+
+
+def gen_router(seed: int, shape: Shape, layer: int) -> np.ndarray:
+    """Router weights [N, H], entries N(0, 1/H)."""
+    g = _rng(seed, KIND_ROUTER, layer)
+    x = g.standard_normal((shape.n_routed, shape.hidden), dtype=np.float32)
+    x *= np.float32(1.0 / np.sqrt(shape.hidden))
+    return _store(x, shape.weight_dtype, None)
+
+
+def gen_shared_gate(seed: int, shape: Shape, layer: int) -> np.ndarray:
+    """Shared-expert gate vector [H], entries N(0, 1/H)."""
+    g = _rng(seed, KIND_SHARED_GATE, layer)
+    x = g.standard_normal((shape.hidden,), dtype=np.float32)
+    x *= np.float32(1.0 / np.sqrt(shape.hidden))
+    return _store(x, shape.weight_dtype, None)
+
+
+def gen_expert_block(seed: int, shape: Shape, layer: int, expert: int,
+                     out: np.ndarray | None = None) -> np.ndarray:
+    """Routed expert block [I, 3, H] (flattened), entries N(0, 0.02^2)."""
+    n = expert_block_elems(shape.hidden, shape.inter_routed)
+    g = _rng(seed, KIND_EXPERT, layer, expert)
+    x = g.standard_normal((n,), dtype=np.float32)
+    x *= np.float32(EXPERT_STD)
+    return _store(x, shape.weight_dtype, out)
+
+
+def gen_shared_block(seed: int, shape: Shape, layer: int, idx: int,
+                     out: np.ndarray | None = None) -> np.ndarray:
+    """Shared expert block [I_s, 3, H] (flattened), entries N(0, 0.02^2)."""
+    n = expert_block_elems(shape.hidden, shape.inter_shared)
+    g = _rng(seed, KIND_SHARED, layer, idx)
+    x = g.standard_normal((n,), dtype=np.float32)
+    x *= np.float32(EXPERT_STD)
+    return _store(x, shape.weight_dtype, out)
+
+
+def fill_expert_store(seed: int, shape: Shape, store: np.ndarray, layers=None,
+                      threads: int | None = None) -> None:
+    """Fill ``store[L, N, 3*I*H]`` (a view over caller-owned, e.g. pinned, memory)."""
+    layers = range(shape.n_layers) if layers is None else layers
+    jobs = [(l, e) for l in layers for e in range(shape.n_routed)]
+    threads = threads or len(os.sched_getaffinity(0))
+
+    def one(le):
+        l, e = le
+        gen_expert_block(seed, shape, l, e, out=store[l, e])
+
+    if threads <= 1 or len(jobs) < 4:
+        for j in jobs:
+            one(j)
+    else:
+        with ThreadPoolExecutor(threads) as ex:
+            list(ex.map(one, jobs))
+
+
+def expert_matrices(block: np.ndarray, hidden: int, inter: int):
+    """Views (W_gate [I,H], W_up [I,H], W_down [H,I]) into a packed expert block."""
+    b = block.reshape(inter, 3, hidden)
+    return b[:, 0, :], b[:, 1, :], b[:, 2, :].T
+
+
+class HiddenStream:
+    """Per-layer, per-sequence AR(1) hidden states, one ``[L, B, H]`` array per step.
+
+    ``h_1 = eps_1`` and ``h_t = rho * h_{t-1} + sqrt(1 - rho^2) * eps_t`` with
+    ``eps ~ N(0, I)`` independent per (step, layer, sequence); everything in float32.
+    ``rho`` is a scalar, or ``None`` for one coefficient per sequence drawn U(0.3, 0.95).
+    """
+
+    def __init__(self, seed: int, shape: Shape, rho):
+        self.seed, self.shape = seed, shape
+        B = shape.batch
+        if rho is None:
+            r = _rng(seed, KIND_RHO).uniform(0.3, 0.95, size=B)
+        else:
+            r = np.full(B, float(rho))
+        self.rho = r.astype(np.float32)
+        self._a = self.rho.reshape(1, B, 1)
+        self._c = np.sqrt(np.float32(1.0) - self.rho * self.rho).astype(np.float32).reshape(1, B, 1)
+        self.t = 0
+        self._h = None
+
+    def step(self) -> np.ndarray:
+        s = self.shape
+        eps = _rng(self.seed, KIND_HIDDEN, self.t).standard_normal(
+            (s.n_layers, s.batch, s.hidden), dtype=np.float32)
+        if self._h is None:
+            self._h = eps
+        else:
+            self._h = (self._a * self._h + self._c * eps).astype(np.float32)
+        self.t += 1
+        return self._h
+
+    def take(self, n_steps: int) -> np.ndarray:
+        """Next ``n_steps`` states as ``[n_steps, L, B, H]`` float32."""
+        s = self.shape
+        out = np.empty((n_steps, s.n_layers, s.batch, s.hidden), dtype=np.float32)
+        for i in range(n_steps):
+            out[i] = self.step()
+        return out

@@ -1,0 +1,226 @@
+"""Pins for the oracle's expert arithmetic and for the stepped stack (counters, reuse)."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import remoe_oracle as orc
+import synth
+
+
+def test_silu_values():
+    assert orc.silu(0.0) == 0.0
+    assert abs(float(orc.silu(1.0)) - 0.7310585786300049) < 1e-15      # 1 / (1 + e^-1)
+    assert abs(float(orc.silu(-1.0)) + 0.2689414213699951) < 1e-15     # -1 / (1 + e)
+    assert abs(float(orc.silu(40.0)) - 40.0) < 1e-12
+    x = np.linspace(-6, 6, 25)
+    assert np.allclose(orc.silu(x) - orc.silu(-x), x, atol=1e-14)       # silu(x) - silu(-x) = x
+
+
+def test_expert_hand_example():
+    # H = 2, I = 1: y = W_down[:, 0] * silu(x_0) * x_1
+    wg = np.array([[1.0, 0.0]]); wu = np.array([[0.0, 1.0]]); wd = np.array([[2.0], [3.0]])
+    x = np.array([0.7, -1.5])
+    a = (0.7 / (1 + math.exp(-0.7))) * -1.5
+    assert np.allclose(orc.swiglu_expert(wg, wu, wd, x), [2 * a, 3 * a], rtol=1e-15)
+
+
+def test_single_expert_matches_library_ops():
+    """N = K = 1: the gate weight is exactly 1 and the layer is one SwiGLU expert, which
+    torch evaluates with its own silu and matmul."""
+    rng = np.random.default_rng(0)
+    H, I = 48, 20
+    wg, wu, wd = rng.standard_normal((I, H)), rng.standard_normal((I, H)), rng.standard_normal((H, I))
+    wr = rng.standard_normal((1, H))
+    x = rng.standard_normal(H)
+    z = orc.router_logits(wr, x)
+    ids, _ = orc.topk_select(z, 1)
+    g = orc.gate_weights(orc.softmax(z), ids, False)
+    assert g[0] == 1.0
+    out = orc.moe_output(x, ids, g, 1, lambda e: (wg, wu, wd))
+    tx = torch.from_numpy(x)
+    ref = torch.from_numpy(wd) @ (torch.nn.functional.silu(torch.from_numpy(wg) @ tx) * (torch.from_numpy(wu) @ tx))
+    assert np.allclose(out, ref.numpy(), rtol=1e-12, atol=1e-12)
+
+
+def _toy(seed, n=6, H=16, I=8):
+    rng = np.random.default_rng(seed)
+    ws = [(rng.standard_normal((I, H)), rng.standard_normal((I, H)), rng.standard_normal((H, I)))
+          for _ in range(n)]
+    return ws, rng.standard_normal(H)
+
+
+def test_dense_equals_selected_and_masking():
+    ws, x = _toy(1)
+    ids, g = [4, 1, 3], [0.5, 0.25, 0.125]
+    d = orc.moe_output(x, ids, g, 6, lambda e: ws[e], mode="dense")
+    s = orc.moe_output(x, ids, g, 6, lambda e: ws[e], mode="selected")
+    assert np.array_equal(d, s)
+    by_hand = 0.25 * orc.swiglu_expert(*ws[1], x) + 0.125 * orc.swiglu_expert(*ws[3], x) \
+        + 0.5 * orc.swiglu_expert(*ws[4], x)
+    assert np.allclose(d, by_hand, rtol=1e-13, atol=1e-13)
+
+
+def test_linearity_zero_and_shared():
+    ws, x = _toy(2)
+    ids = [0, 5]
+    y0, y5 = orc.swiglu_expert(*ws[0], x), orc.swiglu_expert(*ws[5], x)
+    a = orc.moe_output(x, ids, [0.3, 0.6], 6, lambda e: ws[e])
+    b = orc.moe_output(x, ids, [0.6, 1.2], 6, lambda e: ws[e])
+    assert np.allclose(2 * a, b, rtol=1e-13)
+    assert np.allclose(a, 0.3 * y0 + 0.6 * y5, rtol=1e-13)
+    zero = (np.zeros((8, 16)), np.zeros((8, 16)), np.zeros((16, 8)))
+    assert np.array_equal(orc.moe_output(x, [0], [1.0], 1, lambda e: zero), np.zeros(16))
+    sh = orc.moe_output(x, ids, [0.3, 0.6], 6, lambda e: ws[e], shared_weights=[ws[2], ws[3]])
+    assert np.allclose(sh - a, orc.swiglu_expert(*ws[2], x) + orc.swiglu_expert(*ws[3], x), rtol=1e-12, atol=1e-12)
+    sh2 = orc.moe_output(x, ids, [0.3, 0.6], 6, lambda e: ws[e], shared_weights=[ws[2]], shared_scale=0.25)
+    assert np.allclose(sh2 - a, 0.25 * orc.swiglu_expert(*ws[2], x), rtol=1e-12, atol=1e-12)
+    assert orc.sigmoid(0.0) == 0.5 and abs(orc.sigmoid(2.0) + orc.sigmoid(-2.0) - 1.0) < 1e-15
+
+
+# ------------------------------------------------------------------------------- stack
+
+def _stack(shape, cache_slots, seed=0, with_ffn=False, policy="lru"):
+    routers = [synth.gen_router(seed, shape, l) for l in range(shape.n_layers)]
+    sg = [synth.gen_shared_gate(seed, shape, l) for l in range(shape.n_layers)] if shape.shared_gate else None
+    if shape.weight_dtype == 1:
+        routers = [synth.bf16_bits_to_f32(r) for r in routers]
+        sg = None if sg is None else [synth.bf16_bits_to_f32(v) for v in sg]
+
+    def widen(b):
+        return synth.bf16_bits_to_f32(b) if shape.weight_dtype == 1 else b
+
+    def ew(l, e):
+        return synth.expert_matrices(widen(synth.gen_expert_block(seed, shape, l, e)), shape.hidden, shape.inter_routed)
+
+    def sw(l, i):
+        return synth.expert_matrices(widen(synth.gen_shared_block(seed, shape, l, i)), shape.hidden, shape.inter_shared)
+
+    return orc.OracleStack(shape, cache_slots, routers, ew if with_ffn else None, sw if with_ffn else None,
+                           shared_gates=sg, policy=policy)
+
+
+def test_tiny_config_invariants():
+    cfg = synth.config("tiny_fp32")
+    shape = cfg["shape"]
+    st = _stack(shape, cfg["cache_slots"], with_ffn=True)
+    hs = synth.HiddenStream(0, shape, 0.9)
+    T = cfg["steps"]
+    prev_ids = None
+    for t in range(T):
+        h = hs.step()
+        r = st.step(h, ffn="dense" if t < 4 else "selected")
+        if t < 4:
+            st2 = orc.moe_output(h[0, 0], r["ids"][0, 0], r["gates"][0, 0], shape.n_routed,
+                                 lambda e: st.expert_weights(0, e), mode="selected")
+            assert np.array_equal(st2, r["out"][0, 0])
+        assert r["gates"][0, 0].sum() <= 1.0 + 1e-12
+        ov = r["overlap"][0, 0]
+        if t == 0:
+            assert ov == -1 and sum(r["hit"][0]) == 0
+        else:
+            assert 0 <= ov <= shape.top_k
+            assert ov == len(set(r["ids"][0, 0]) & set(prev_ids))
+            assert len(r["hit"][0]) - sum(r["hit"][0]) <= shape.top_k - ov       # Prop. 3.1
+        prev_ids = r["ids"][0, 0]
+    assert st.tok_hits[0] + st.tok_misses[0] == shape.n_layers * shape.top_k * T
+    assert st.uniq_hits == st.tok_hits and st.uniq_misses == st.tok_misses       # B = 1: dedup is a no-op
+    assert st.pairs_counted[0] == T - 1
+    assert 0.0 <= st.eor() <= 1.0 and 0.0 <= st.uhr() <= 1.0
+
+
+def test_constant_stream_reuses_everything():
+    shape = synth.Shape(2, 64, 12, 3, 8)
+    st = _stack(shape, 3)
+    h = np.random.default_rng(0).standard_normal((2, 1, 64)).astype(np.float32)
+    for t in range(10):
+        r = st.step(h, ffn=None)
+        if t:
+            assert (r["overlap"] == 3).all() and all(all(x) for x in r["hit"])
+    assert st.eor() == 1.0 and sum(st.uniq_misses) == 2 * 3
+
+
+def test_layers_are_independent():
+    shape = synth.Shape(3, 64, 16, 2, 8)
+    full = _stack(shape, 4)
+    hs = synth.HiddenStream(1, shape, 0.7).take(40)
+    traces = [full.step(hs[t], ffn=None) for t in range(40)]
+    for l in range(3):
+        one = orc.OracleStack(synth.Shape(1, 64, 16, 2, 8), 4, [full.routers[l]])
+        for t in range(40):
+            r = one.step(hs[t, l:l + 1], ffn=None)
+            assert np.array_equal(r["ids"][0], traces[t]["ids"][l])
+            assert r["hit"][0] == traces[t]["hit"][l] and r["slot"][0] == traces[t]["slot"][l]
+        assert one.uniq_misses[0] == full.uniq_misses[l]
+    assert sum(full.uniq_misses) == sum(len(tr["hit"][l]) - sum(tr["hit"][l]) for tr in traces for l in range(3))
+
+
+def test_batched_counters():
+    shape = synth.Shape(2, 64, 16, 3, 8, batch=5)
+    st = _stack(shape, 8)
+    hs = synth.HiddenStream(2, shape, None)
+    T, sum_u = 30, 0
+    for t in range(T):
+        before = [c.resident() for c in st.caches]
+        th0 = list(st.tok_hits)
+        r = st.step(hs.step(), ffn=None)
+        for l in range(2):
+            flat = [int(e) for e in r["ids"][l].reshape(-1)]
+            assert r["requests"][l] == orc.unique_in_order(flat)
+            assert st.tok_hits[l] - th0[l] == sum(1 for e in flat if e in before[l])
+            assert r["hit"][l] == [e in before[l] for e in r["requests"][l]]
+            sum_u += len(r["requests"][l])
+    assert sum(st.tok_hits) + sum(st.tok_misses) == 2 * 5 * 3 * T
+    assert sum(st.uniq_hits) + sum(st.uniq_misses) == sum_u
+    assert st.pairs_counted == [(T - 1) * 5] * 2
+
+
+def test_iid_stream_statistics():
+    """rho = 0: consecutive selections are independent, so EOR is near K/N and, for
+    exchangeable experts, the LRU hit rate is near C/N (loose statistical check)."""
+    shape = synth.Shape(4, 64, 32, 4, 8)
+    st = _stack(shape, 8)
+    hs = synth.HiddenStream(3, shape, 0.0)
+    for _ in range(400):
+        st.step(hs.step(), ffn=None)
+    assert abs(st.eor() - 4 / 32) < 0.03
+    assert abs(st.uhr() - 8 / 32) < 0.06
+
+
+def test_id_override_and_reset():
+    shape = synth.Shape(1, 64, 16, 2, 8)
+    st = _stack(shape, 4)
+    h = synth.HiddenStream(4, shape, 0.5).take(3)
+    r0 = st.step(h[0], ffn=None)
+    forced = [int(r0["ids"][0, 0][0]), 15 if 15 not in r0["ids"][0, 0] else 14]
+    r1 = st.step(h[1], ffn=None, id_override={(0, 0): forced})
+    assert list(r1["ids"][0, 0]) == forced and r1["requests"][0] == forced
+    assert r1["hit"][0][0] is True
+    st.reset()
+    assert st.caches[0].resident() == set() and st.pairs_counted == [0]
+    r2 = st.step(h[0], ffn=None)
+    assert np.array_equal(r2["ids"], r0["ids"]) and sum(r2["hit"][0]) == 0 and r2["overlap"][0, 0] == -1
+
+
+def test_synth_is_reproducible_and_layout():
+    shape = synth.Shape(2, 32, 4, 2, 6, weight_dtype=1)
+    a = synth.gen_expert_block(0, shape, 1, 3)
+    b = synth.gen_expert_block(0, shape, 1, 3)
+    assert a.dtype == np.uint16 and np.array_equal(a, b) and a.size == 3 * 32 * 6
+    assert not np.array_equal(a, synth.gen_expert_block(0, shape, 1, 2))
+    wg, wu, wd = synth.expert_matrices(a, 32, 6)
+    assert wg.shape == (6, 32) and wd.shape == (32, 6)
+    blk = a.reshape(6, 3, 32)
+    assert np.array_equal(wg[2], blk[2, 0]) and np.array_equal(wu[2], blk[2, 1]) and np.array_equal(wd[:, 2], blk[2, 2])
+    x = np.array([1.0, 1.00390625, -2.5, 3.0e-3], dtype=np.float32)       # 1.00390625 = 1 + 2^-8: tie -> even
+    bits = synth.bf16_round_to_bits(x)
+    assert bits[0] == 0x3F80 and bits[1] == 0x3F80
+    back = synth.bf16_bits_to_f32(bits)
+    assert np.all(np.abs(back - x) <= np.abs(x) * 2.0 ** -8)
+    hs1 = synth.HiddenStream(5, shape, 0.9).take(5)
+    hs2 = synth.HiddenStream(5, shape, 0.9).take(5)
+    assert np.array_equal(hs1, hs2) and hs1.shape == (5, 2, 1, 32)
+    long = synth.HiddenStream(6, synth.Shape(1, 4096, 4, 2, 6), 0.9).take(200)[:, 0, 0]
+    c = np.mean(long[1:] * long[:-1]) / np.mean(long * long)
+    assert abs(c - 0.9) < 0.02 and abs(long.std() - 1.0) < 0.05
