@@ -1,0 +1,171 @@
+/*
+ * remoe.h -- C ABI of the bounded-cache MoE decode step for one NVIDIA B200 (sm_100a).
+ *
+ * The library runs, per decoded token and per MoE layer, the inference path that the
+ * ReMoE paper's router fine-tuning targets: router GEMV, softmax and top-K gating,
+ * resolution of the selected experts against a per-layer cache of C fixed HBM slots with
+ * LRU replacement, fetch of missing experts from pinned host memory, the SwiGLU expert
+ * GEMVs over the resident weights plus always-resident shared experts, the gate-weighted
+ * combine, and the step-to-step reuse statistic.
+ *
+ * Conventions
+ *   - Every function returns 0 (REMOE_OK) or a negative REMOE_E_* code; nothing aborts,
+ *     throws or traps across this boundary.  remoe_strerror() names a code.
+ *   - "dev" pointers are CUDA device pointers owned by the caller; "host" pointers are host
+ *     memory owned by the caller.  The handle is owned by the library.
+ *   - All tensors are dense, row-major, layer-major: [L, B, ...].
+ *   - One stack belongs to one device (the one current at creation) and one stream.
+ *     Calls on one stack must not overlap in time.
+ *
+ * Data layouts
+ *   router weights   [N, H]   one row per routed expert, element type = weight_dtype
+ *   shared-gate      [H]      element type = weight_dtype
+ *   expert block     [I, 3, H] for intermediate channel i three consecutive rows:
+ *                    W_gate[i, :], W_up[i, :], W_down[:, i]; 3*I*H elements, contiguous.
+ *                    An expert computes y = W_down (silu(W_gate x) * (W_up x)).
+ *   hidden states    [L, B, H] float32; layer l reads its own stream: out[l] = MoE_l(in[l]).
+ */
+#ifndef REMOE_H_
+#define REMOE_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  REMOE_OK = 0,
+  REMOE_E_ARG = -1,          /* null pointer, index out of range, misaligned pointer      */
+  REMOE_E_CAPACITY = -2,     /* cache_slots_per_layer < top_k at batch 1 (App. A.2, Assumption 1) */
+  REMOE_E_NOT_LOADED = -3,   /* a router, shared expert or requested routed expert is missing */
+  REMOE_E_NOT_PINNED = -4,   /* an expert pointer is not page-locked host memory          */
+  REMOE_E_CUDA = -5,         /* a CUDA runtime call failed; see remoe_last_cuda_error()   */
+  REMOE_E_DEVICE_FLAG = -6,  /* a kernel recorded an internal error (bounded wait ran out, bad index) */
+  REMOE_E_UNSUPPORTED = -7,  /* shape outside what the kernels are built for              */
+  REMOE_E_NOMEM = -8         /* host or device allocation failed                          */
+};
+
+enum { REMOE_F32 = 0, REMOE_BF16 = 1 };
+enum { REMOE_POLICY_LRU = 0, REMOE_POLICY_FIFO = 1, REMOE_POLICY_LFU = 2 };
+
+/* Shape of the stack.  Sec. 3.1: N_r routed experts, Top-K; shared experts always active. */
+typedef struct {
+  int32_t n_layers;      /* L                                                              */
+  int32_t hidden;        /* H; float32: multiple of 128, bf16: multiple of 256; <= 2048    */
+  int32_t n_routed;      /* N_r <= 256                                                     */
+  int32_t top_k;         /* K <= min(N_r, 32)                                              */
+  int32_t inter_routed;  /* I of a routed expert                                           */
+  int32_t n_shared;      /* number of shared experts (0 if none)                           */
+  int32_t inter_shared;  /* I of each shared expert                                        */
+  int32_t shared_gate;   /* 1: shared output is scaled by sigmoid(w_sg . h)                */
+  int32_t renorm_topk;   /* 1: top-K gate weights are renormalised to sum to 1             */
+  int32_t weight_dtype;  /* REMOE_F32 or REMOE_BF16 (router, shared gate, all experts)     */
+  int32_t batch;         /* B sequences per step                                           */
+} remoe_shape;
+
+/* Counters of App. E.2.3-E.2.4, summed over steps since creation or the last reset. */
+typedef struct {
+  uint64_t tok_hits, tok_misses;     /* per routed slot (B*K events per layer-step)        */
+  uint64_t uniq_hits, uniq_misses;   /* per distinct requested expert; uniq_misses = #uMiss */
+  uint64_t h2d_bytes;                /* bytes fetched from host memory for misses          */
+  uint64_t steps;                    /* decode steps taken                                 */
+} remoe_cache_counters;
+
+typedef struct remoe_stack remoe_stack;
+
+/*
+ * Create a stack with an empty cache of `cache_slots_per_layer` expert slots per layer
+ * (Sec. 3.1: per-layer expert cache of capacity C; Sec. 3: request-isolated cold start).
+ * `cuda_stream` is the cudaStream_t all kernels are ordered on (NULL = default stream); the
+ * library also owns one copy stream.  Allocates the slot pools, directory and scratch on
+ * the current device.  Errors: ARG, CAPACITY (B == 1 and C < K), UNSUPPORTED, NOMEM, CUDA.
+ */
+int remoe_stack_create(const remoe_shape* shape, int32_t cache_slots_per_layer,
+                       void* cuda_stream, remoe_stack** out);
+
+/* Copy layer `layer`'s router weights [N, H] (and, when shape.shared_gate, the gate vector
+ * [H]; else pass NULL) from host memory to the device.  Synchronous.  (Sec. 3.1: theta_gate.) */
+int remoe_load_router(remoe_stack*, int32_t layer, const void* w_router_host,
+                      const void* w_shared_gate_host);
+
+/* Copy shared expert `idx` of `layer` (one expert block, I = inter_shared) to the device,
+ * where it stays resident and never enters the cache (Sec. 3.1; App. A.1).  Synchronous. */
+int remoe_load_shared(remoe_stack*, int32_t layer, int32_t idx, const void* block_host);
+
+/* Register the host copies of routed experts first_expert .. first_expert+count-1 of
+ * `layer`: `pinned_ptrs[i]` points at one expert block in page-locked host memory, 16-byte
+ * aligned.  BORROWED: the caller keeps the memory pinned, alive and unchanged until the
+ * stack is destroyed; misses are fetched from it (Sec. 3.1: "misses trigger expert
+ * fetches").  Several experts may share one pointer.  Errors: ARG, NOT_PINNED. */
+int remoe_load_experts_host(remoe_stack*, int32_t layer, int32_t first_expert, int32_t count,
+                            const void* const* pinned_ptrs);
+
+/*
+ * One decode step for all L layers and B sequences (Sec. 3.1 routing; App. A.1-A.2 cache
+ * model; Eq. 1 reuse).  Inputs/outputs are device pointers:
+ *   hidden_in    [L, B, H] float32
+ *   hidden_out   [L, B, H] float32   sum_e g_e y_e + shared terms
+ *   selected_ids [L, B, K] int32     by descending logit, equal logits by ascending id
+ *   gate_weights [L, B, K] float32   softmax probability (renormalised if renorm_topk)
+ * Hits and misses are judged against the cache state held before the step; misses are
+ * fetched from the registered host blocks into the victim slots (empty slot first, else
+ * least recently used) on the copy stream while resident experts are already computed.
+ * The call blocks only until the step's miss list is known; on return the remaining work
+ * is enqueued and the outputs are complete once the stack's stream has drained.
+ * Errors: ARG, NOT_LOADED, CUDA, DEVICE_FLAG.
+ */
+int remoe_decode_step(remoe_stack*, const float* hidden_in_dev, float* hidden_out_dev,
+                      int32_t* selected_ids_dev, float* gate_weights_dev);
+
+/* Same step with HOST buffers (pageable or pinned): copies hidden_in to the device, runs
+ * the step, copies the three outputs back and returns when they are complete. */
+int remoe_decode_step_host(remoe_stack*, const float* hidden_in_host, float* hidden_out_host,
+                           int32_t* selected_ids_host, float* gate_weights_host);
+
+/* Cache trace of the most recent step, to host arrays (any may be NULL).  Per layer the
+ * distinct requests U in first-occurrence order (App. E.2.3), padded to B*K entries:
+ *   requests/hit/slot/evicted [L, B*K] int32 (evicted = -1 when nothing was displaced),
+ *   n_unique [L].  Waits for the stack's stream. */
+int remoe_last_step_trace(remoe_stack*, int32_t* requests, int32_t* hit, int32_t* slot,
+                          int32_t* evicted, int32_t* n_unique);
+
+/* Counters for one layer, or summed over layers with layer = -1 (App. E.2.4: #uMiss, uHR =
+ * uniq_hits / (uniq_hits + uniq_misses), tHR likewise).  Waits for the stack's stream. */
+int remoe_cache_stats(remoe_stack*, int32_t layer, remoe_cache_counters* out);
+
+/* Reuse statistic (Eq. 1): overlap_sum = sum over counted (step, sequence) pairs of
+ * |E_t n E_{t-1}|, pairs_counted = number of such pairs (steps t >= 2 since the last
+ * reset), so EOR = overlap_sum / (K * pairs_counted).  `last_ir` (host, [L, B] or NULL; with
+ * layer >= 0: [B]) receives IR_t of the most recent step, -1 where t = 1.  layer = -1 sums. */
+int remoe_reuse_stats(remoe_stack*, int32_t layer, uint64_t* overlap_sum,
+                      uint64_t* pairs_counted, float* last_ir);
+
+/* Empty every layer's cache, forget E_{t-1} and zero all counters (Sec. 3: each request
+ * starts from a cold expert cache). */
+int remoe_cache_reset(remoe_stack*);
+
+/* Replacement policy for subsequent steps (App. A.5 names LRU, LFU, FIFO); resets the cache. */
+int remoe_set_policy(remoe_stack*, int32_t policy);
+
+/* Cache-aware rerouting (App. F.2): add `beta` to the pre-top-K logits of experts resident
+ * before the step; 0 (default) leaves routing untouched.  Gate weights still come from the
+ * unbiased softmax. */
+int remoe_set_reroute_beta(remoe_stack*, float beta);
+
+/* Kernel timing aid: with `on` != 0 every expert-streaming kernel launch is bracketed by
+ * CUDA events on its own stream.  remoe_kernel_time returns the summed duration (ms), the
+ * number of launches and the weight bytes they streamed since profiling was switched on. */
+int remoe_set_profiling(remoe_stack*, int32_t on);
+int remoe_kernel_time(remoe_stack*, double* ms_sum, uint64_t* launches, uint64_t* weight_bytes);
+
+/* Text of the last CUDA runtime error seen by this stack ("" if none). */
+const char* remoe_last_cuda_error(const remoe_stack*);
+
+void remoe_stack_destroy(remoe_stack*);
+const char* remoe_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* REMOE_H_ */

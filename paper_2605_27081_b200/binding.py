@@ -1,0 +1,270 @@
+"""ctypes binding of libremoe.so: argument marshalling only, same names as the C ABI.
+
+Every step of the decode path runs inside the library's CUDA kernels; nothing here
+computes.  PyTorch is used by callers for device memory and streams; this module only
+needs raw pointers (``tensor.data_ptr()``) and, for host arrays, numpy buffers.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libremoe.so")
+
+REMOE_OK = 0
+REMOE_E_ARG, REMOE_E_CAPACITY, REMOE_E_NOT_LOADED, REMOE_E_NOT_PINNED = -1, -2, -3, -4
+REMOE_E_CUDA, REMOE_E_DEVICE_FLAG, REMOE_E_UNSUPPORTED, REMOE_E_NOMEM = -5, -6, -7, -8
+REMOE_F32, REMOE_BF16 = 0, 1
+REMOE_POLICY_LRU, REMOE_POLICY_FIFO, REMOE_POLICY_LFU = 0, 1, 2
+
+EXPORTS = [
+    "remoe_stack_create", "remoe_load_router", "remoe_load_shared", "remoe_load_experts_host",
+    "remoe_decode_step", "remoe_decode_step_host", "remoe_last_step_trace", "remoe_cache_stats",
+    "remoe_reuse_stats", "remoe_cache_reset", "remoe_set_policy", "remoe_set_reroute_beta",
+    "remoe_set_profiling", "remoe_kernel_time", "remoe_last_cuda_error", "remoe_stack_destroy",
+    "remoe_strerror",
+]
+
+
+class remoe_shape(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in (
+        "n_layers", "hidden", "n_routed", "top_k", "inter_routed", "n_shared", "inter_shared",
+        "shared_gate", "renorm_topk", "weight_dtype", "batch")]
+
+
+class remoe_cache_counters(C.Structure):
+    _fields_ = [(n, C.c_uint64) for n in (
+        "tok_hits", "tok_misses", "uniq_hits", "uniq_misses", "h2d_bytes", "steps")]
+
+
+class RemoeError(RuntimeError):
+    def __init__(self, code, what, detail=""):
+        self.code = code
+        super().__init__(f"{what}: {code} ({strerror(code)}){' -- ' + detail if detail else ''}")
+
+
+_lib = None
+
+
+def lib():
+    """The loaded shared library.  There is no fallback: a missing build is an error."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2605_27081_b200.build` "
+                "(there is no CPU or PyTorch fallback for this path)")
+        L = C.CDLL(LIB_PATH)
+        vp, i32, f32p, i32p = C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p
+        L.remoe_stack_create.argtypes = [C.POINTER(remoe_shape), i32, vp, C.POINTER(vp)]
+        L.remoe_load_router.argtypes = [vp, i32, vp, vp]
+        L.remoe_load_shared.argtypes = [vp, i32, i32, vp]
+        L.remoe_load_experts_host.argtypes = [vp, i32, i32, i32, C.POINTER(vp)]
+        L.remoe_decode_step.argtypes = [vp, f32p, f32p, i32p, f32p]
+        L.remoe_decode_step_host.argtypes = [vp, f32p, f32p, i32p, f32p]
+        L.remoe_last_step_trace.argtypes = [vp, i32p, i32p, i32p, i32p, i32p]
+        L.remoe_cache_stats.argtypes = [vp, i32, C.POINTER(remoe_cache_counters)]
+        L.remoe_reuse_stats.argtypes = [vp, i32, C.POINTER(C.c_uint64), C.POINTER(C.c_uint64), vp]
+        L.remoe_cache_reset.argtypes = [vp]
+        L.remoe_set_policy.argtypes = [vp, i32]
+        L.remoe_set_reroute_beta.argtypes = [vp, C.c_float]
+        L.remoe_set_profiling.argtypes = [vp, i32]
+        L.remoe_kernel_time.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
+        L.remoe_last_cuda_error.argtypes = [vp]
+        L.remoe_last_cuda_error.restype = C.c_char_p
+        L.remoe_stack_destroy.argtypes = [vp]
+        L.remoe_stack_destroy.restype = None
+        L.remoe_strerror.argtypes = [C.c_int]
+        L.remoe_strerror.restype = C.c_char_p
+        for name in EXPORTS:
+            if name not in ("remoe_last_cuda_error", "remoe_stack_destroy", "remoe_strerror"):
+                getattr(L, name).restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def strerror(code: int) -> str:
+    return lib().remoe_strerror(int(code)).decode()
+
+
+def _ptr(x):
+    """Raw address of a torch tensor, numpy array, int or None."""
+    if x is None:
+        return None
+    if isinstance(x, int):
+        return x
+    if hasattr(x, "data_ptr"):
+        return x.data_ptr()
+    if isinstance(x, np.ndarray):
+        return x.ctypes.data
+    raise TypeError(type(x))
+
+
+def _shape_struct(shape) -> remoe_shape:
+    if isinstance(shape, remoe_shape):
+        return shape
+    get = (lambda k: shape[k]) if isinstance(shape, dict) else (lambda k: getattr(shape, k))
+    return remoe_shape(*[int(get(n)) for n, _ in remoe_shape._fields_])
+
+
+# ---- thin wrappers with the C names; each returns the status code (and outputs) ----------
+
+def remoe_stack_create(shape, cache_slots_per_layer: int, cuda_stream: int | None = None):
+    h = C.c_void_p()
+    st = _shape_struct(shape)
+    rc = lib().remoe_stack_create(C.byref(st), int(cache_slots_per_layer), cuda_stream, C.byref(h))
+    return rc, h
+
+
+def remoe_load_router(h, layer, w_router_host, w_shared_gate_host=None):
+    return lib().remoe_load_router(h, int(layer), _ptr(w_router_host), _ptr(w_shared_gate_host))
+
+
+def remoe_load_shared(h, layer, idx, block_host):
+    return lib().remoe_load_shared(h, int(layer), int(idx), _ptr(block_host))
+
+
+def remoe_load_experts_host(h, layer, first_expert, pinned_ptrs):
+    n = len(pinned_ptrs)
+    arr = (C.c_void_p * n)(*[_ptr(p) for p in pinned_ptrs])
+    return lib().remoe_load_experts_host(h, int(layer), int(first_expert), n, arr)
+
+
+def remoe_decode_step(h, hidden_in, hidden_out, selected_ids, gate_weights):
+    return lib().remoe_decode_step(h, _ptr(hidden_in), _ptr(hidden_out), _ptr(selected_ids), _ptr(gate_weights))
+
+
+def remoe_decode_step_host(h, hidden_in, hidden_out, selected_ids, gate_weights):
+    return lib().remoe_decode_step_host(h, _ptr(hidden_in), _ptr(hidden_out), _ptr(selected_ids),
+                                        _ptr(gate_weights))
+
+
+def remoe_last_step_trace(h, requests, hit, slot, evicted, n_unique):
+    return lib().remoe_last_step_trace(h, _ptr(requests), _ptr(hit), _ptr(slot), _ptr(evicted), _ptr(n_unique))
+
+
+def remoe_cache_stats(h, layer=-1):
+    out = remoe_cache_counters()
+    rc = lib().remoe_cache_stats(h, int(layer), C.byref(out))
+    return rc, {n: int(getattr(out, n)) for n, _ in remoe_cache_counters._fields_}
+
+
+def remoe_reuse_stats(h, layer=-1, last_ir=None):
+    o, p = C.c_uint64(), C.c_uint64()
+    rc = lib().remoe_reuse_stats(h, int(layer), C.byref(o), C.byref(p), _ptr(last_ir))
+    return rc, int(o.value), int(p.value)
+
+
+def remoe_cache_reset(h):
+    return lib().remoe_cache_reset(h)
+
+
+def remoe_set_policy(h, policy):
+    return lib().remoe_set_policy(h, int(policy))
+
+
+def remoe_set_reroute_beta(h, beta):
+    return lib().remoe_set_reroute_beta(h, float(beta))
+
+
+def remoe_set_profiling(h, on):
+    return lib().remoe_set_profiling(h, int(bool(on)))
+
+
+def remoe_kernel_time(h):
+    ms, n, b = C.c_double(), C.c_uint64(), C.c_uint64()
+    rc = lib().remoe_kernel_time(h, C.byref(ms), C.byref(n), C.byref(b))
+    return rc, float(ms.value), int(n.value), int(b.value)
+
+
+def remoe_last_cuda_error(h) -> str:
+    return lib().remoe_last_cuda_error(h).decode()
+
+
+def remoe_stack_destroy(h):
+    lib().remoe_stack_destroy(h)
+
+
+class Stack:
+    """Owning convenience wrapper: raises RemoeError on any non-zero status."""
+
+    def __init__(self, shape, cache_slots_per_layer, cuda_stream: int | None = None):
+        self.shape = _shape_struct(shape)
+        self.cache_slots = int(cache_slots_per_layer)
+        rc, self.h = remoe_stack_create(self.shape, cache_slots_per_layer, cuda_stream)
+        if rc != REMOE_OK:
+            self.h = None
+            raise RemoeError(rc, "remoe_stack_create")
+        self._keep = []          # references that keep borrowed host blocks alive
+
+    def _ck(self, rc, what):
+        if rc != REMOE_OK:
+            raise RemoeError(rc, what, remoe_last_cuda_error(self.h) if rc == REMOE_E_CUDA else "")
+
+    def load_router(self, layer, w_router, w_shared_gate=None):
+        self._ck(remoe_load_router(self.h, layer, w_router, w_shared_gate), "remoe_load_router")
+
+    def load_shared(self, layer, idx, block):
+        self._ck(remoe_load_shared(self.h, layer, idx, block), "remoe_load_shared")
+
+    def load_experts_host(self, layer, first_expert, blocks, keep=None):
+        self._ck(remoe_load_experts_host(self.h, layer, first_expert, blocks), "remoe_load_experts_host")
+        self._keep.append(blocks if keep is None else keep)
+
+    def decode_step(self, hidden_in, hidden_out, selected_ids, gate_weights):
+        self._ck(remoe_decode_step(self.h, hidden_in, hidden_out, selected_ids, gate_weights), "remoe_decode_step")
+
+    def decode_step_host(self, hidden_in, hidden_out, selected_ids, gate_weights):
+        self._ck(remoe_decode_step_host(self.h, hidden_in, hidden_out, selected_ids, gate_weights),
+                 "remoe_decode_step_host")
+
+    def last_step_trace(self):
+        L, BK = self.shape.n_layers, self.shape.batch * self.shape.top_k
+        req, hit, slot, ev = (np.empty((L, BK), np.int32) for _ in range(4))
+        nu = np.empty(L, np.int32)
+        self._ck(remoe_last_step_trace(self.h, req, hit, slot, ev, nu), "remoe_last_step_trace")
+        return dict(requests=req, hit=hit, slot=slot, evicted=ev, n_unique=nu)
+
+    def cache_stats(self, layer=-1):
+        rc, out = remoe_cache_stats(self.h, layer)
+        self._ck(rc, "remoe_cache_stats")
+        return out
+
+    def reuse_stats(self, layer=-1, want_last_ir=False):
+        n = self.shape.batch * (self.shape.n_layers if layer < 0 else 1)
+        ir = np.empty(n, np.float32) if want_last_ir else None
+        rc, o, p = remoe_reuse_stats(self.h, layer, ir)
+        self._ck(rc, "remoe_reuse_stats")
+        return (o, p, ir) if want_last_ir else (o, p)
+
+    def cache_reset(self):
+        self._ck(remoe_cache_reset(self.h), "remoe_cache_reset")
+
+    def set_policy(self, policy):
+        self._ck(remoe_set_policy(self.h, policy), "remoe_set_policy")
+
+    def set_reroute_beta(self, beta):
+        self._ck(remoe_set_reroute_beta(self.h, beta), "remoe_set_reroute_beta")
+
+    def set_profiling(self, on):
+        self._ck(remoe_set_profiling(self.h, on), "remoe_set_profiling")
+
+    def kernel_time(self):
+        rc, ms, n, b = remoe_kernel_time(self.h)
+        self._ck(rc, "remoe_kernel_time")
+        return ms, n, b
+
+    def close(self):
+        if self.h is not None:
+            remoe_stack_destroy(self.h)
+            self.h = None
+            self._keep = []
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

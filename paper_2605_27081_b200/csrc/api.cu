@@ -1,0 +1,532 @@
+// Host side of libremoe: stack state, the per-step scheduler with its miss-fetch engine,
+// statistics, and the extern "C" boundary declared in remoe.h.
+//
+// Per decode step (batch 1):
+//   compute stream : route+resolve kernel -> copy of the step trace to pinned host memory
+//                    -> resident-phase streaming kernel (hits + shared experts, all layers)
+//   host           : waits only for the trace, then walks it: for each layer, one
+//                    cudaMemcpyAsync per missing expert from its pinned host block into the
+//                    victim slot on the copy stream, an event after the layer's last copy
+//   compute stream : per layer with misses: wait for that event, miss-phase streaming kernel
+//                    over the freshly filled slots; finally the combine kernel.
+// Copies of later layers overlap the compute of earlier ones; nothing is ever inserted into a
+// slot except the misses of an already routed step (no speculative prefetch, which would
+// break the fetch bound of Prop. 3.1).
+#include "remoe_internal.cuh"
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+using namespace remoe;
+
+struct EvPair {
+  cudaEvent_t a, b;
+  uint64_t bytes;
+};
+
+struct remoe_stack {
+  remoe_shape shape{};
+  int C = 0, device = 0, grid = 0, BK = 0;
+  cudaStream_t stream = nullptr, copy_stream = nullptr;
+  DevStack d{};
+  std::vector<void*> dev_allocs;
+  std::vector<void*> host_allocs;
+  std::vector<const void*> host_ptrs;      // [L*N] borrowed pinned expert blocks
+  std::vector<char> router_loaded, shared_loaded;
+  int* dev_block = nullptr;                // [err | trace]
+  int* host_block = nullptr;               // pinned mirror of dev_block
+  size_t block_ints = 0;
+  float* partial = nullptr;
+  int* contrib = nullptr;
+  cudaEvent_t ev_trace = nullptr;
+  std::vector<cudaEvent_t> ev_layer;
+  uint64_t steps = 0, steps_since_reset = 0;
+  std::vector<uint64_t> h2d_bytes;         // per layer
+  // staging for the host-buffer entry point
+  float *st_in_d = nullptr, *st_out_d = nullptr, *st_g_d = nullptr;
+  int* st_ids_d = nullptr;
+  float *st_in_h = nullptr, *st_out_h = nullptr, *st_g_h = nullptr;
+  int* st_ids_h = nullptr;
+  // profiling
+  bool profiling = false;
+  std::vector<EvPair> ev_used, ev_free;
+  double prof_ms = 0.0;
+  uint64_t prof_launches = 0, prof_bytes = 0;
+  std::string cuda_err;
+  int policy = REMOE_POLICY_LRU;
+  float beta = 0.f;
+};
+
+namespace {
+
+int fail_cuda(remoe_stack* s, cudaError_t e, const char* what) {
+  if (s) {
+    s->cuda_err = std::string(what) + ": " + cudaGetErrorString(e);
+  }
+  return REMOE_E_CUDA;
+}
+
+#define CK(call)                                                    \
+  do {                                                              \
+    cudaError_t e_ = (call);                                        \
+    if (e_ != cudaSuccess) return fail_cuda(s, e_, #call);          \
+  } while (0)
+
+template <typename T>
+int dev_alloc(remoe_stack* s, T** p, size_t count) {
+  void* q = nullptr;
+  cudaError_t e = cudaMalloc(&q, count * sizeof(T) > 0 ? count * sizeof(T) : 16);
+  if (e != cudaSuccess) {
+    fail_cuda(s, e, "cudaMalloc");
+    return e == cudaErrorMemoryAllocation ? REMOE_E_NOMEM : REMOE_E_CUDA;
+  }
+  s->dev_allocs.push_back(q);
+  *p = static_cast<T*>(q);
+  return REMOE_OK;
+}
+
+template <typename T>
+int host_alloc(remoe_stack* s, T** p, size_t count) {
+  void* q = nullptr;
+  cudaError_t e = cudaMallocHost(&q, count * sizeof(T) > 0 ? count * sizeof(T) : 16);
+  if (e != cudaSuccess) {
+    fail_cuda(s, e, "cudaMallocHost");
+    return REMOE_E_NOMEM;
+  }
+  s->host_allocs.push_back(q);
+  *p = static_cast<T*>(q);
+  return REMOE_OK;
+}
+
+int reset_state(remoe_stack* s) {
+  const DevStack& d = s->d;
+  const size_t L = d.L;
+  CK(cudaMemsetAsync(d.expert_of_slot, 0xff, L * d.C * sizeof(int), s->stream));
+  CK(cudaMemsetAsync(d.slot_of_expert, 0xff, L * d.N * sizeof(int), s->stream));
+  CK(cudaMemsetAsync(d.stamp, 0, L * d.C * sizeof(unsigned long long), s->stream));
+  CK(cudaMemsetAsync(d.freq, 0, L * d.C * sizeof(unsigned), s->stream));
+  CK(cudaMemsetAsync(d.clock, 0, L * sizeof(unsigned long long), s->stream));
+  CK(cudaMemsetAsync(d.prev_mask, 0, L * d.B * kMaskWords * sizeof(unsigned), s->stream));
+  CK(cudaMemsetAsync(d.counters, 0, L * kCounters * sizeof(unsigned long long), s->stream));
+  CK(cudaMemsetAsync(d.last_overlap, 0xff, L * d.B * sizeof(int), s->stream));
+  CK(cudaMemsetAsync(s->dev_block, 0, s->block_ints * sizeof(int), s->stream));
+  CK(cudaStreamSynchronize(s->stream));
+  s->steps = 0;
+  s->steps_since_reset = 0;
+  std::fill(s->h2d_bytes.begin(), s->h2d_bytes.end(), 0);
+  return REMOE_OK;
+}
+
+bool everything_loaded(const remoe_stack* s) {
+  for (char c : s->router_loaded) if (!c) return false;
+  for (char c : s->shared_loaded) if (!c) return false;
+  for (const void* p : s->host_ptrs) if (!p) return false;
+  return true;
+}
+
+int prof_begin(remoe_stack* s, cudaStream_t st, uint64_t bytes) {
+  if (!s->profiling) return REMOE_OK;
+  EvPair p;
+  if (!s->ev_free.empty()) {
+    p = s->ev_free.back();
+    s->ev_free.pop_back();
+  } else {
+    CK(cudaEventCreate(&p.a));
+    CK(cudaEventCreate(&p.b));
+  }
+  p.bytes = bytes;
+  CK(cudaEventRecord(p.a, st));
+  s->ev_used.push_back(p);
+  return REMOE_OK;
+}
+
+int prof_end(remoe_stack* s, cudaStream_t st) {
+  if (!s->profiling) return REMOE_OK;
+  CK(cudaEventRecord(s->ev_used.back().b, st));
+  return REMOE_OK;
+}
+
+int prof_collect(remoe_stack* s) {
+  for (EvPair& p : s->ev_used) {
+    float ms = 0.f;
+    CK(cudaEventSynchronize(p.b));
+    CK(cudaEventElapsedTime(&ms, p.a, p.b));
+    s->prof_ms += ms;
+    s->prof_launches += 1;
+    s->prof_bytes += p.bytes;
+    s->ev_free.push_back(p);
+  }
+  s->ev_used.clear();
+  return REMOE_OK;
+}
+
+int check_device_flag(remoe_stack* s) {
+  return s->host_block[0] != kErrNone ? REMOE_E_DEVICE_FLAG : REMOE_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* remoe_strerror(int code) {
+  switch (code) {
+    case REMOE_OK: return "ok";
+    case REMOE_E_ARG: return "invalid argument";
+    case REMOE_E_CAPACITY: return "cache capacity below top_k";
+    case REMOE_E_NOT_LOADED: return "weights not loaded";
+    case REMOE_E_NOT_PINNED: return "expert pointer is not page-locked host memory";
+    case REMOE_E_CUDA: return "CUDA runtime error";
+    case REMOE_E_DEVICE_FLAG: return "device-side error flag set";
+    case REMOE_E_UNSUPPORTED: return "unsupported shape";
+    case REMOE_E_NOMEM: return "out of memory";
+    default: return "unknown error";
+  }
+}
+
+const char* remoe_last_cuda_error(const remoe_stack* s) { return s ? s->cuda_err.c_str() : ""; }
+
+void remoe_stack_destroy(remoe_stack* s) {
+  if (!s) return;
+  cudaSetDevice(s->device);
+  cudaStreamSynchronize(s->stream);
+  if (s->copy_stream) {
+    cudaStreamSynchronize(s->copy_stream);
+    cudaStreamDestroy(s->copy_stream);
+  }
+  for (EvPair& p : s->ev_used) { cudaEventDestroy(p.a); cudaEventDestroy(p.b); }
+  for (EvPair& p : s->ev_free) { cudaEventDestroy(p.a); cudaEventDestroy(p.b); }
+  if (s->ev_trace) cudaEventDestroy(s->ev_trace);
+  for (cudaEvent_t e : s->ev_layer) cudaEventDestroy(e);
+  for (void* p : s->dev_allocs) cudaFree(p);
+  for (void* p : s->host_allocs) cudaFreeHost(p);
+  delete s;
+}
+
+int remoe_stack_create(const remoe_shape* sh, int32_t cache_slots, void* cuda_stream, remoe_stack** out) {
+  if (!sh || !out) return REMOE_E_ARG;
+  *out = nullptr;
+  if (sh->n_layers < 1 || sh->hidden < 1 || sh->n_routed < 1 || sh->top_k < 1 || sh->inter_routed < 1 ||
+      sh->batch < 1 || sh->n_shared < 0 || cache_slots < 1 || sh->top_k > sh->n_routed ||
+      (sh->n_shared > 0 && sh->inter_shared < 1) || (sh->weight_dtype != REMOE_F32 && sh->weight_dtype != REMOE_BF16))
+    return REMOE_E_ARG;
+  if (sh->batch == 1 && cache_slots < sh->top_k) return REMOE_E_CAPACITY;
+  const int wbytes = sh->weight_dtype == REMOE_BF16 ? 2 : 4;
+  const long pairs = (long)sh->n_layers * (sh->top_k + sh->n_shared);
+  if (sh->n_routed > kMaxRouted || sh->top_k > 32 || cache_slots > kMaxSlots || cache_slots > sh->n_routed ||
+      (long)sh->batch * sh->top_k > kMaxRequests || pairs > kMaxPairs || !ffn_stream_supported(sh->hidden, wbytes))
+    return REMOE_E_UNSUPPORTED;
+
+  remoe_stack* s = new (std::nothrow) remoe_stack();
+  if (!s) return REMOE_E_NOMEM;
+  s->shape = *sh;
+  s->C = cache_slots;
+  s->stream = static_cast<cudaStream_t>(cuda_stream);
+  s->BK = sh->batch * sh->top_k;
+  int rc = REMOE_OK;
+  auto bail = [&](int code) {
+    remoe_stack_destroy(s);
+    return code;
+  };
+  if (cudaGetDevice(&s->device) != cudaSuccess) return bail(REMOE_E_CUDA);
+  int sms = 0;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, s->device) != cudaSuccess || sms < 1)
+    return bail(REMOE_E_CUDA);
+  s->grid = sms;
+  if (cudaStreamCreateWithFlags(&s->copy_stream, cudaStreamNonBlocking) != cudaSuccess) return bail(REMOE_E_CUDA);
+  if (cudaEventCreateWithFlags(&s->ev_trace, cudaEventDisableTiming) != cudaSuccess) return bail(REMOE_E_CUDA);
+  s->ev_layer.resize(sh->n_layers, nullptr);
+  for (auto& e : s->ev_layer)
+    if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return bail(REMOE_E_CUDA);
+
+  DevStack& d = s->d;
+  d.L = sh->n_layers; d.H = sh->hidden; d.N = sh->n_routed; d.K = sh->top_k; d.I = sh->inter_routed;
+  d.S = sh->n_shared; d.Is = sh->n_shared ? sh->inter_shared : 0; d.B = sh->batch; d.C = cache_slots;
+  d.shared_gate = sh->shared_gate ? 1 : 0; d.renorm = sh->renorm_topk ? 1 : 0; d.wbytes = wbytes;
+  d.policy = REMOE_POLICY_LRU; d.beta = 0.f; d.has_prev = 0;
+  d.slot_bytes = (size_t)3 * d.I * d.H * wbytes;
+  d.shared_bytes = (size_t)3 * d.Is * d.H * wbytes;
+  const size_t L = d.L;
+  char *router = nullptr, *sgw = nullptr, *shared = nullptr, *slots = nullptr;
+#define TRY(x) do { rc = (x); if (rc != REMOE_OK) return bail(rc); } while (0)
+  TRY(dev_alloc(s, &router, L * d.N * d.H * wbytes));
+  TRY(dev_alloc(s, &sgw, L * d.H * wbytes));
+  TRY(dev_alloc(s, &shared, L * d.S * d.shared_bytes));
+  TRY(dev_alloc(s, &slots, L * d.C * d.slot_bytes));
+  d.router = router; d.shared_gate_w = sgw; d.shared_blocks = shared; d.slots = slots;
+  TRY(dev_alloc(s, &d.expert_of_slot, L * d.C));
+  TRY(dev_alloc(s, &d.slot_of_expert, L * d.N));
+  TRY(dev_alloc(s, &d.stamp, L * d.C));
+  TRY(dev_alloc(s, &d.freq, L * d.C));
+  TRY(dev_alloc(s, &d.clock, L));
+  TRY(dev_alloc(s, &d.prev_mask, L * d.B * kMaskWords));
+  TRY(dev_alloc(s, &d.counters, L * kCounters));
+  TRY(dev_alloc(s, &d.shared_scale, L * d.B));
+  TRY(dev_alloc(s, &d.last_overlap, L * d.B));
+  s->block_ints = 1 + (size_t)trace_ints(d.L, s->BK);
+  TRY(dev_alloc(s, &s->dev_block, s->block_ints));
+  TRY(host_alloc(s, &s->host_block, s->block_ints));
+  std::memset(s->host_block, 0, s->block_ints * sizeof(int));
+  d.err = s->dev_block;
+  d.trace = s->dev_block + 1;
+  TRY(dev_alloc(s, &s->partial, (size_t)2 * L * s->grid * d.H));
+  TRY(dev_alloc(s, &s->contrib, (size_t)2 * L * 2));
+  const size_t io = L * d.B * d.H, kk = L * (size_t)s->BK;
+  TRY(dev_alloc(s, &s->st_in_d, io));
+  TRY(dev_alloc(s, &s->st_out_d, io));
+  TRY(dev_alloc(s, &s->st_g_d, kk));
+  TRY(dev_alloc(s, &s->st_ids_d, kk));
+  TRY(host_alloc(s, &s->st_in_h, io));
+  TRY(host_alloc(s, &s->st_out_h, io));
+  TRY(host_alloc(s, &s->st_g_h, kk));
+  TRY(host_alloc(s, &s->st_ids_h, kk));
+#undef TRY
+  s->host_ptrs.assign(L * d.N, nullptr);
+  s->router_loaded.assign(L, 0);
+  s->shared_loaded.assign(L * d.S, 0);
+  s->h2d_bytes.assign(L, 0);
+  rc = reset_state(s);
+  if (rc != REMOE_OK) return bail(rc);
+  *out = s;
+  return REMOE_OK;
+}
+
+int remoe_load_router(remoe_stack* s, int32_t layer, const void* w, const void* wsg) {
+  if (!s || !w || layer < 0 || layer >= s->d.L) return REMOE_E_ARG;
+  if (s->d.shared_gate && !wsg) return REMOE_E_ARG;
+  const size_t row = (size_t)s->d.H * s->d.wbytes;
+  CK(cudaMemcpyAsync(const_cast<char*>(s->d.router) + (size_t)layer * s->d.N * row, w, s->d.N * row,
+                     cudaMemcpyHostToDevice, s->stream));
+  if (s->d.shared_gate)
+    CK(cudaMemcpyAsync(const_cast<char*>(s->d.shared_gate_w) + (size_t)layer * row, wsg, row,
+                       cudaMemcpyHostToDevice, s->stream));
+  CK(cudaStreamSynchronize(s->stream));
+  s->router_loaded[layer] = 1;
+  return REMOE_OK;
+}
+
+int remoe_load_shared(remoe_stack* s, int32_t layer, int32_t idx, const void* block) {
+  if (!s || !block || layer < 0 || layer >= s->d.L || idx < 0 || idx >= s->d.S) return REMOE_E_ARG;
+  CK(cudaMemcpyAsync(const_cast<char*>(s->d.shared_blocks) + ((size_t)layer * s->d.S + idx) * s->d.shared_bytes,
+                     block, s->d.shared_bytes, cudaMemcpyHostToDevice, s->stream));
+  CK(cudaStreamSynchronize(s->stream));
+  s->shared_loaded[(size_t)layer * s->d.S + idx] = 1;
+  return REMOE_OK;
+}
+
+int remoe_load_experts_host(remoe_stack* s, int32_t layer, int32_t first, int32_t count,
+                            const void* const* ptrs) {
+  if (!s || !ptrs || layer < 0 || layer >= s->d.L || first < 0 || count < 0 || first + count > s->d.N)
+    return REMOE_E_ARG;
+  for (int i = 0; i < count; ++i) {
+    if (!ptrs[i] || (reinterpret_cast<uintptr_t>(ptrs[i]) & 15u)) return REMOE_E_ARG;
+    cudaPointerAttributes at{};
+    cudaError_t e = cudaPointerGetAttributes(&at, ptrs[i]);
+    if (e != cudaSuccess) {
+      cudaGetLastError();
+      return REMOE_E_NOT_PINNED;
+    }
+    if (at.type != cudaMemoryTypeHost) return REMOE_E_NOT_PINNED;
+  }
+  for (int i = 0; i < count; ++i) s->host_ptrs[(size_t)layer * s->d.N + first + i] = ptrs[i];
+  return REMOE_OK;
+}
+
+int remoe_decode_step(remoe_stack* s, const float* hin, float* hout, int32_t* ids, float* gates) {
+  if (!s || !hin || !hout || !ids || !gates) return REMOE_E_ARG;
+  if ((reinterpret_cast<uintptr_t>(hin) | reinterpret_cast<uintptr_t>(hout)) & 15u) return REMOE_E_ARG;
+  if (!everything_loaded(s)) return REMOE_E_NOT_LOADED;
+  if (s->d.B != 1) return REMOE_E_UNSUPPORTED;
+  DevStack& d = s->d;
+  d.has_prev = s->steps_since_reset > 0 ? 1 : 0;
+  d.policy = s->policy;
+  d.beta = s->beta;
+
+  CK(launch_route(d, hin, ids, gates, s->contrib, s->stream));
+  CK(cudaMemcpyAsync(s->host_block, s->dev_block, s->block_ints * sizeof(int), cudaMemcpyDeviceToHost, s->stream));
+  CK(cudaEventRecord(s->ev_trace, s->stream));
+
+  FfnArgs a{};
+  a.d = d;
+  a.hidden_in = hin;
+  a.gates = gates;
+  a.partial = s->partial;
+  a.contrib = s->contrib;
+  a.grid_cap = s->grid;
+  a.phase = 0;
+  a.layer = -1;
+  // The resident phase needs no host decision: enqueue it before waiting for the trace.
+  int rc = prof_begin(s, s->stream, 0);
+  if (rc != REMOE_OK) return rc;
+  CK(launch_ffn_stream(a, s->grid, s->stream));
+  rc = prof_end(s, s->stream);
+  if (rc != REMOE_OK) return rc;
+  const size_t prof_slot = s->profiling ? s->ev_used.size() - 1 : 0;
+
+  CK(cudaEventSynchronize(s->ev_trace));
+  s->steps += 1;
+  s->steps_since_reset += 1;
+  if (check_device_flag(s) != REMOE_OK) return REMOE_E_DEVICE_FLAG;
+
+  int* tr = s->host_block + 1;
+  const int* t_req = trace_requests(tr, d.L, s->BK);
+  const int* t_hit = trace_hit(tr, d.L, s->BK);
+  const int* t_slot = trace_slot(tr, d.L, s->BK);
+  uint64_t resident_bytes = 0;
+  bool copy_ordered = false;
+  for (int l = 0; l < d.L; ++l) {
+    int misses = 0;
+    for (int k = 0; k < d.K; ++k) {
+      const int i = l * s->BK + k;
+      if (t_hit[i]) { resident_bytes += d.slot_bytes; continue; }
+      const int e = t_req[i], slot = t_slot[i];
+      if (e < 0 || e >= d.N || slot < 0 || slot >= d.C) return REMOE_E_DEVICE_FLAG;
+      if (!copy_ordered) {
+        // Victim slots may still be read by the previous step's kernels, all of which precede
+        // this step's route kernel on the compute stream.
+        CK(cudaStreamWaitEvent(s->copy_stream, s->ev_trace, 0));
+        copy_ordered = true;
+      }
+      CK(cudaMemcpyAsync(d.slots + ((size_t)l * d.C + slot) * d.slot_bytes, s->host_ptrs[(size_t)l * d.N + e],
+                         d.slot_bytes, cudaMemcpyHostToDevice, s->copy_stream));
+      ++misses;
+    }
+    resident_bytes += (uint64_t)d.S * d.shared_bytes;
+    if (misses) {
+      s->h2d_bytes[l] += (uint64_t)misses * d.slot_bytes;
+      CK(cudaEventRecord(s->ev_layer[l], s->copy_stream));
+      CK(cudaStreamWaitEvent(s->stream, s->ev_layer[l], 0));
+      a.phase = 1;
+      a.layer = l;
+      rc = prof_begin(s, s->stream, (uint64_t)misses * d.slot_bytes);
+      if (rc != REMOE_OK) return rc;
+      CK(launch_ffn_stream(a, s->grid, s->stream));
+      rc = prof_end(s, s->stream);
+      if (rc != REMOE_OK) return rc;
+    }
+  }
+  if (s->profiling) s->ev_used[prof_slot].bytes = resident_bytes;
+  CK(launch_combine(a, hout, s->stream));
+  return REMOE_OK;
+}
+
+int remoe_decode_step_host(remoe_stack* s, const float* hin, float* hout, int32_t* ids, float* gates) {
+  if (!s || !hin || !hout || !ids || !gates) return REMOE_E_ARG;
+  const size_t io = (size_t)s->d.L * s->d.B * s->d.H, kk = (size_t)s->d.L * s->BK;
+  std::memcpy(s->st_in_h, hin, io * sizeof(float));
+  CK(cudaMemcpyAsync(s->st_in_d, s->st_in_h, io * sizeof(float), cudaMemcpyHostToDevice, s->stream));
+  int rc = remoe_decode_step(s, s->st_in_d, s->st_out_d, s->st_ids_d, s->st_g_d);
+  if (rc != REMOE_OK) return rc;
+  CK(cudaMemcpyAsync(s->st_out_h, s->st_out_d, io * sizeof(float), cudaMemcpyDeviceToHost, s->stream));
+  CK(cudaMemcpyAsync(s->st_ids_h, s->st_ids_d, kk * sizeof(int), cudaMemcpyDeviceToHost, s->stream));
+  CK(cudaMemcpyAsync(s->st_g_h, s->st_g_d, kk * sizeof(float), cudaMemcpyDeviceToHost, s->stream));
+  CK(cudaStreamSynchronize(s->stream));
+  std::memcpy(hout, s->st_out_h, io * sizeof(float));
+  std::memcpy(ids, s->st_ids_h, kk * sizeof(int));
+  std::memcpy(gates, s->st_g_h, kk * sizeof(float));
+  return REMOE_OK;
+}
+
+int remoe_last_step_trace(remoe_stack* s, int32_t* req, int32_t* hit, int32_t* slot, int32_t* ev, int32_t* nu) {
+  if (!s) return REMOE_E_ARG;
+  if (s->steps == 0) return REMOE_E_ARG;
+  CK(cudaStreamSynchronize(s->stream));
+  CK(cudaMemcpy(s->host_block, s->dev_block, s->block_ints * sizeof(int), cudaMemcpyDeviceToHost));
+  int* tr = s->host_block + 1;
+  const size_t n = (size_t)s->d.L * s->BK * sizeof(int);
+  if (req) std::memcpy(req, trace_requests(tr, s->d.L, s->BK), n);
+  if (hit) std::memcpy(hit, trace_hit(tr, s->d.L, s->BK), n);
+  if (slot) std::memcpy(slot, trace_slot(tr, s->d.L, s->BK), n);
+  if (ev) std::memcpy(ev, trace_evicted(tr, s->d.L, s->BK), n);
+  if (nu) std::memcpy(nu, trace_n_unique(tr), (size_t)s->d.L * sizeof(int));
+  return check_device_flag(s);
+}
+
+int remoe_cache_stats(remoe_stack* s, int32_t layer, remoe_cache_counters* out) {
+  if (!s || !out || layer < -1 || layer >= s->d.L) return REMOE_E_ARG;
+  CK(cudaStreamSynchronize(s->stream));
+  std::vector<unsigned long long> c((size_t)s->d.L * kCounters);
+  CK(cudaMemcpy(c.data(), s->d.counters, c.size() * sizeof(unsigned long long), cudaMemcpyDeviceToHost));
+  std::memset(out, 0, sizeof(*out));
+  for (int l = 0; l < s->d.L; ++l) {
+    if (layer >= 0 && l != layer) continue;
+    out->tok_hits += c[(size_t)l * kCounters + 0];
+    out->tok_misses += c[(size_t)l * kCounters + 1];
+    out->uniq_hits += c[(size_t)l * kCounters + 2];
+    out->uniq_misses += c[(size_t)l * kCounters + 3];
+    out->h2d_bytes += s->h2d_bytes[l];
+  }
+  out->steps = s->steps;
+  return REMOE_OK;
+}
+
+int remoe_reuse_stats(remoe_stack* s, int32_t layer, uint64_t* overlap_sum, uint64_t* pairs, float* last_ir) {
+  if (!s || layer < -1 || layer >= s->d.L) return REMOE_E_ARG;
+  CK(cudaStreamSynchronize(s->stream));
+  std::vector<unsigned long long> c((size_t)s->d.L * kCounters);
+  CK(cudaMemcpy(c.data(), s->d.counters, c.size() * sizeof(unsigned long long), cudaMemcpyDeviceToHost));
+  uint64_t o = 0, p = 0;
+  for (int l = 0; l < s->d.L; ++l) {
+    if (layer >= 0 && l != layer) continue;
+    o += c[(size_t)l * kCounters + 4];
+    p += c[(size_t)l * kCounters + 5];
+  }
+  if (overlap_sum) *overlap_sum = o;
+  if (pairs) *pairs = p;
+  if (last_ir) {
+    std::vector<int> ov((size_t)s->d.L * s->d.B);
+    CK(cudaMemcpy(ov.data(), s->d.last_overlap, ov.size() * sizeof(int), cudaMemcpyDeviceToHost));
+    const int l0 = layer < 0 ? 0 : layer, l1 = layer < 0 ? s->d.L : layer + 1;
+    size_t j = 0;
+    for (int l = l0; l < l1; ++l)
+      for (int b = 0; b < s->d.B; ++b) {
+        const int v = ov[(size_t)l * s->d.B + b];
+        last_ir[j++] = v < 0 ? -1.f : (float)v / (float)s->d.K;
+      }
+  }
+  return REMOE_OK;
+}
+
+int remoe_cache_reset(remoe_stack* s) {
+  if (!s) return REMOE_E_ARG;
+  CK(cudaStreamSynchronize(s->stream));
+  CK(cudaStreamSynchronize(s->copy_stream));
+  return reset_state(s);
+}
+
+int remoe_set_policy(remoe_stack* s, int32_t policy) {
+  if (!s || policy < REMOE_POLICY_LRU || policy > REMOE_POLICY_LFU) return REMOE_E_ARG;
+  s->policy = policy;
+  return remoe_cache_reset(s);
+}
+
+int remoe_set_reroute_beta(remoe_stack* s, float beta) {
+  if (!s || !(beta == beta)) return REMOE_E_ARG;
+  s->beta = beta;
+  return REMOE_OK;
+}
+
+int remoe_set_profiling(remoe_stack* s, int32_t on) {
+  if (!s) return REMOE_E_ARG;
+  int rc = prof_collect(s);
+  if (rc != REMOE_OK) return rc;
+  s->profiling = on != 0;
+  s->prof_ms = 0.0;
+  s->prof_launches = 0;
+  s->prof_bytes = 0;
+  return REMOE_OK;
+}
+
+int remoe_kernel_time(remoe_stack* s, double* ms_sum, uint64_t* launches, uint64_t* bytes) {
+  if (!s) return REMOE_E_ARG;
+  int rc = prof_collect(s);
+  if (rc != REMOE_OK) return rc;
+  if (ms_sum) *ms_sum = s->prof_ms;
+  if (launches) *launches = s->prof_launches;
+  if (bytes) *bytes = s->prof_bytes;
+  return REMOE_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,401 @@
+// Streaming SwiGLU expert GEMV with fused gate-weighted combine, batch 1, sm_100a.
+//
+// An expert block is stored channel-major: for intermediate channel i the rows W_gate[i,:],
+// W_up[i,:] and W_down[:,i] are contiguous (3*H elements).  One such triple is all the data
+// needed for
+//     a_i = silu(W_gate[i,:] . h) * (W_up[i,:] . h) * g          (g: gate weight / shared scale)
+//     out += a_i * W_down[:, i]
+// so the whole layer -- K routed experts in their cache slots plus the shared experts -- is one
+// linear stream of triples with no intermediate vector in memory and no dependency between
+// CTAs.  The kernel therefore treats every active (layer, expert) of the launch as one long
+// row list, cuts it into equal contiguous ranges, one per CTA, and in each CTA
+//   - a producer thread moves triples HBM -> shared memory with bulk async copies (TMA,
+//     non-tensor form) into a ring of stages guarded by full/empty mbarriers;
+//   - eight consumer warps take triples round-robin; a warp owns a whole triple: two dot
+//     products by 128-bit shared loads and shuffle reduction, SiLU, then an AXPY into its
+//     private fp32 copy of out[H] held in registers;
+//   - at a layer boundary and at the end the eight private copies are added in a fixed order
+//     and written as this CTA's partial for that layer.
+// A second tiny kernel adds the partials of each layer in a fixed order (resident phase by
+// ascending CTA, then miss phase by ascending CTA), so results are deterministic and no float
+// atomics are used.  HBM traffic is the weight bytes once plus O(grid * H) partials.
+#include "remoe_internal.cuh"
+
+namespace remoe {
+
+namespace {
+
+constexpr int kConsumerWarps = 8;
+constexpr int kThreads = (kConsumerWarps + 1) * 32;
+constexpr int kMaxStages = 16;
+constexpr unsigned kSpinLimit = 1u << 20;
+constexpr unsigned kFull = 0xffffffffu;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: false if the phase did not complete within the spin limit.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+  for (unsigned it = 0; it < kSpinLimit; ++it)
+    if (mbar_try_wait(bar, parity)) return true;
+  return false;
+}
+__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+          smem_u32(dst)),
+      "l"(__cvta_generic_to_global(src)), "r"(bytes), "r"(smem_u32(bar))
+      : "memory");
+}
+__device__ __forceinline__ void consumer_bar() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+
+template <int WB>
+struct Elems;
+template <>
+struct Elems<4> {
+  static constexpr int kVec = 4;
+  __device__ static __forceinline__ void load(const char* p, float* f) {
+    const float4 v = *reinterpret_cast<const float4*>(p);
+    f[0] = v.x; f[1] = v.y; f[2] = v.z; f[3] = v.w;
+  }
+};
+template <>
+struct Elems<2> {
+  static constexpr int kVec = 8;
+  __device__ static __forceinline__ void load(const char* p, float* f) {
+    const uint4 v = *reinterpret_cast<const uint4*>(p);
+    f[0] = __uint_as_float(v.x << 16); f[1] = __uint_as_float(v.x & 0xffff0000u);
+    f[2] = __uint_as_float(v.y << 16); f[3] = __uint_as_float(v.y & 0xffff0000u);
+    f[4] = __uint_as_float(v.z << 16); f[5] = __uint_as_float(v.z & 0xffff0000u);
+    f[6] = __uint_as_float(v.w << 16); f[7] = __uint_as_float(v.w & 0xffff0000u);
+  }
+};
+
+// Shared-memory carve-up (dynamic): barriers | row prefix table | reduce buffer | stage ring.
+struct Layout {
+  size_t bars, prefix, red, stages, total;
+  int n_stages;
+};
+__host__ __device__ inline Layout make_layout(int H, int wbytes) {
+  Layout y;
+  y.bars = 0;
+  y.prefix = 2 * kMaxStages * sizeof(uint64_t);
+  y.red = y.prefix + (size_t)(kMaxPairs + 1) * sizeof(int) + 12;           // keep 16-byte alignment
+  y.red = (y.red + 127) / 128 * 128;
+  y.stages = y.red + (size_t)kConsumerWarps * H * sizeof(float);
+  const size_t stage = (size_t)3 * H * wbytes;
+  const size_t budget = 227 * 1024;
+  int n = (int)((budget - y.stages) / stage);
+  if (n > kMaxStages) n = kMaxStages;
+  y.n_stages = n;
+  y.total = y.stages + (size_t)n * stage;
+  return y;
+}
+
+// Rows (channel triples) a (layer, position) pair contributes to this launch.
+__device__ __forceinline__ int pair_rows(const FfnArgs& a, int pair) {
+  const DevStack& d = a.d;
+  const int P = d.K + d.S;
+  const int l = pair / P, p = pair % P;
+  if (p >= d.K) return a.phase == 0 ? d.Is : 0;
+  const int hit = trace_hit(d.trace, d.L, d.K)[l * d.K + p];
+  if (a.phase == 0) return hit ? d.I : 0;
+  return (l == a.layer && !hit) ? d.I : 0;
+}
+
+template <int WB, int H>
+__global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(const __grid_constant__ FfnArgs a) {
+  using E = Elems<WB>;
+  constexpr int kVec = E::kVec;
+  constexpr int kIter = H / (32 * kVec);
+  constexpr int kCols = kIter * kVec;                  // columns of h / out owned by one lane
+  constexpr uint32_t kStageBytes = 3u * H * WB;
+  constexpr uint32_t kRowBytes = (uint32_t)H * WB;
+
+  extern __shared__ __align__(128) unsigned char smem[];
+  const Layout lay = make_layout(H, WB);
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + lay.bars);
+  uint64_t* empty = full + kMaxStages;
+  int* prefix = reinterpret_cast<int*>(smem + lay.prefix);
+  float* red = reinterpret_cast<float*>(smem + lay.red);
+  unsigned char* stages = smem + lay.stages;
+  const int NS = lay.n_stages;
+  __shared__ int s_abort;
+
+  const DevStack& d = a.d;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int P = d.K + d.S, n_pairs = d.L * P;
+
+  // Work table: exclusive prefix of rows per pair.
+  for (int i = tid; i < n_pairs; i += kThreads) prefix[i + 1] = pair_rows(a, i);
+  if (tid == 0) {
+    prefix[0] = 0;
+    s_abort = 0;
+    for (int s = 0; s < NS; ++s) { mbar_init(full + s, 1); mbar_init(empty + s, 1); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (warp == 0) {
+    int carry = 0;
+    for (int base = 0; base < n_pairs; base += 32) {
+      const int i = base + lane;
+      int v = i < n_pairs ? prefix[i + 1] : 0;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(kFull, v, o);
+        if (lane >= o) v += t;
+      }
+      if (i < n_pairs) prefix[i + 1] = v + carry;
+      carry += __shfl_sync(kFull, v, 31);
+    }
+  }
+  __syncthreads();
+
+  const int M = prefix[n_pairs];
+  const int G = gridDim.x;
+  const int q = (M + G - 1) / G;                       // rows per CTA
+  const int r0 = min(M, (int)blockIdx.x * q), r1 = min(M, r0 + q);
+
+  if (blockIdx.x == 0) {
+    for (int l = tid; l < d.L; l += kThreads) {
+      if (a.phase != 0 && l != a.layer) continue;
+      const int lo = prefix[l * P], hi = prefix[(l + 1) * P];
+      int* c = a.contrib + ((size_t)a.phase * d.L + l) * 2;
+      if (hi > lo) { c[0] = lo / q; c[1] = (hi - 1) / q; } else { c[0] = 1; c[1] = 0; }
+    }
+  }
+  if (r0 >= r1) return;
+
+  const int* t_slot = trace_slot(d.trace, d.L, d.K);
+
+  if (warp == kConsumerWarps) {
+    // ------------------------------------------------------------------ producer
+    if (lane == 0) {
+      int pair = 0;
+      const char* base = nullptr;
+      int pair_of_base = -1;
+      int issued = 0;
+      bool ok = true;
+      for (int r = r0; r < r1 && ok; ++r, ++issued) {
+        while (prefix[pair + 1] <= r) ++pair;
+        if (pair != pair_of_base) {
+          const int l = pair / P, p = pair % P;
+          if (p < d.K) {
+            const int slot = t_slot[l * d.K + p];
+            if (slot < 0 || slot >= d.C) { atomicCAS(d.err, kErrNone, kErrBadIndex); ok = false; break; }
+            base = d.slots + ((size_t)l * d.C + slot) * d.slot_bytes;
+          } else {
+            base = d.shared_blocks + ((size_t)l * d.S + (p - d.K)) * d.shared_bytes;
+          }
+          pair_of_base = pair;
+        }
+        const int i = r - prefix[pair];
+        const int n = r - r0, s = n % NS;
+        if (n >= NS) {
+          if (*(volatile int*)&s_abort) { ok = false; break; }
+          if (!mbar_wait(empty + s, ((n / NS) - 1) & 1)) {
+            atomicCAS(d.err, kErrNone, kErrWaitEmpty);
+            ok = false;
+            break;
+          }
+        }
+        mbar_expect_tx(full + s, kStageBytes);
+        bulk_g2s(stages + (size_t)s * kStageBytes, base + (size_t)i * kStageBytes, kStageBytes, full + s);
+      }
+      if (!ok) {
+        // Let the consumers leave, then wait (bounded) for copies that are still landing.
+        atomicExch(&s_abort, 1);
+        for (int n = max(0, issued - NS); n < issued; ++n)
+          if (!mbar_wait(full + (n % NS), (n / NS) & 1)) atomicCAS(d.err, kErrNone, kErrDrain);
+      }
+    }
+  } else {
+    // ----------------------------------------------------------------- consumers
+    float hreg[kCols], acc[kCols];
+    int pair = 0;
+    while (prefix[pair + 1] <= r0) ++pair;
+    int l_first = pair / P;
+    int pair_last = pair;
+    while (prefix[pair_last + 1] < r1) ++pair_last;
+    const int l_last = pair_last / P;
+    bool aborted = false;
+
+    for (int l = l_first; l <= l_last; ++l) {
+      const int lo = max(r0, prefix[l * P]), hi = min(r1, prefix[(l + 1) * P]);
+      if (lo >= hi) continue;
+      const float* h = a.hidden_in + (size_t)l * H;
+#pragma unroll
+      for (int it = 0; it < kIter; ++it) {
+#pragma unroll
+        for (int v4 = 0; v4 < kVec / 4; ++v4) {
+          const float4 x = __ldg(reinterpret_cast<const float4*>(h + (it * 32 + lane) * kVec) + v4);
+          hreg[it * kVec + v4 * 4 + 0] = x.x; hreg[it * kVec + v4 * 4 + 1] = x.y;
+          hreg[it * kVec + v4 * 4 + 2] = x.z; hreg[it * kVec + v4 * 4 + 3] = x.w;
+        }
+      }
+#pragma unroll
+      for (int c = 0; c < kCols; ++c) acc[c] = 0.f;
+
+      // first row of this layer handled by this warp: local index n = r - r0 with n % 8 == warp
+      int r = lo + ((warp - (lo - r0)) % kConsumerWarps + kConsumerWarps) % kConsumerWarps;
+      float scale = 0.f;
+      int pair_of_scale = -1;
+      for (; r < hi && !aborted; r += kConsumerWarps) {
+        while (prefix[pair + 1] <= r) ++pair;
+        if (pair != pair_of_scale) {
+          const int p = pair % P;
+          scale = p < d.K ? a.gates[l * d.K + p] : d.shared_scale[l];
+          pair_of_scale = pair;
+        }
+        const int n = r - r0, s = n % NS;
+        if (*(volatile int*)&s_abort || !mbar_wait(full + s, (n / NS) & 1)) {
+          if (!*(volatile int*)&s_abort) { atomicCAS(d.err, kErrNone, kErrWaitFull); atomicExch(&s_abort, 1); }
+          aborted = true;
+          break;
+        }
+        const char* st = reinterpret_cast<const char*>(stages) + (size_t)s * kStageBytes;
+        float g = 0.f, u = 0.f;
+#pragma unroll
+        for (int it = 0; it < kIter; ++it) {
+          float w[kVec];
+          E::load(st + (it * 32 + lane) * 16, w);
+#pragma unroll
+          for (int j = 0; j < kVec; ++j) g = fmaf(w[j], hreg[it * kVec + j], g);
+        }
+#pragma unroll
+        for (int it = 0; it < kIter; ++it) {
+          float w[kVec];
+          E::load(st + kRowBytes + (it * 32 + lane) * 16, w);
+#pragma unroll
+          for (int j = 0; j < kVec; ++j) u = fmaf(w[j], hreg[it * kVec + j], u);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          g += __shfl_xor_sync(kFull, g, o);
+          u += __shfl_xor_sync(kFull, u, o);
+        }
+        const float av = g / (1.f + __expf(-g)) * u * scale;
+#pragma unroll
+        for (int it = 0; it < kIter; ++it) {
+          float w[kVec];
+          E::load(st + 2 * kRowBytes + (it * 32 + lane) * 16, w);
+#pragma unroll
+          for (int j = 0; j < kVec; ++j) acc[it * kVec + j] = fmaf(av, w[j], acc[it * kVec + j]);
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty + s);
+      }
+
+      // Layer flush: add the eight private copies in warp order, write this CTA's partial.
+      float* mine = red + (size_t)warp * H;
+#pragma unroll
+      for (int it = 0; it < kIter; ++it)
+#pragma unroll
+        for (int v4 = 0; v4 < kVec / 4; ++v4)
+          *reinterpret_cast<float4*>(mine + (it * 32 + lane) * kVec + v4 * 4) =
+              make_float4(acc[it * kVec + v4 * 4], acc[it * kVec + v4 * 4 + 1], acc[it * kVec + v4 * 4 + 2],
+                          acc[it * kVec + v4 * 4 + 3]);
+      consumer_bar();
+      float* dst = a.partial + (((size_t)a.phase * d.L + l) * a.grid_cap + blockIdx.x) * H;
+      for (int c = tid; c < H; c += kConsumerWarps * 32) {
+        float t = 0.f;
+#pragma unroll
+        for (int w = 0; w < kConsumerWarps; ++w) t += red[(size_t)w * H + c];
+        dst[c] = t;
+      }
+      consumer_bar();
+    }
+  }
+}
+
+__global__ void __launch_bounds__(256) combine_kernel(FfnArgs a, float* __restrict__ hidden_out) {
+  const DevStack& d = a.d;
+  const int l = blockIdx.y;
+  const int c = blockIdx.x * 256 + threadIdx.x;
+  if (c >= d.H) return;
+  float t = 0.f;
+  for (int phase = 0; phase < 2; ++phase) {
+    const int* cb = a.contrib + ((size_t)phase * d.L + l) * 2;
+    const int lo = cb[0], hi = cb[1];
+    const float* p = a.partial + (((size_t)phase * d.L + l) * a.grid_cap) * d.H + c;
+    for (int b = lo; b <= hi; ++b) t += p[(size_t)b * d.H];
+  }
+  hidden_out[(size_t)l * d.H + c] = t;
+}
+
+template <int WB, int H>
+cudaError_t launch_one(const FfnArgs& a, int grid, cudaStream_t st) {
+  const Layout lay = make_layout(H, WB);
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(ffn_stream_kernel<WB, H>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)lay.total);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  ffn_stream_kernel<WB, H><<<grid, kThreads, lay.total, st>>>(a);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+bool ffn_stream_supported(int H, int wbytes) {
+  if (wbytes == 4) return H == 128 || H == 256 || H == 512 || H == 1024;
+  if (wbytes == 2) return H == 256 || H == 512 || H == 1024 || H == 2048;
+  return false;
+}
+
+size_t ffn_stream_smem_bytes(int H, int wbytes, int* stages_out) {
+  const Layout lay = make_layout(H, wbytes);
+  if (stages_out) *stages_out = lay.n_stages;
+  return lay.total;
+}
+
+cudaError_t launch_ffn_stream(const FfnArgs& a, int grid, cudaStream_t st) {
+  const int H = a.d.H;
+  if (a.d.wbytes == 4) {
+    switch (H) {
+      case 128: return launch_one<4, 128>(a, grid, st);
+      case 256: return launch_one<4, 256>(a, grid, st);
+      case 512: return launch_one<4, 512>(a, grid, st);
+      case 1024: return launch_one<4, 1024>(a, grid, st);
+    }
+  } else {
+    switch (H) {
+      case 256: return launch_one<2, 256>(a, grid, st);
+      case 512: return launch_one<2, 512>(a, grid, st);
+      case 1024: return launch_one<2, 1024>(a, grid, st);
+      case 2048: return launch_one<2, 2048>(a, grid, st);
+    }
+  }
+  return cudaErrorInvalidValue;
+}
+
+cudaError_t launch_combine(const FfnArgs& a, float* hidden_out, cudaStream_t st) {
+  dim3 grid((a.d.H + 255) / 256, a.d.L);
+  combine_kernel<<<grid, 256, 0, st>>>(a, hidden_out);
+  return cudaGetLastError();
+}
+
+}  // namespace remoe

@@ -1,0 +1,83 @@
+// Internal declarations shared by the kernels and the host scheduler of libremoe.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "remoe.h"
+
+namespace remoe {
+
+constexpr int kMaxRouted = 256;        // N_r limit: 8 logits per lane in the top-K warp
+constexpr int kMaskWords = kMaxRouted / 32;
+constexpr int kMaxSlots = 256;         // C limit of the shared-memory directory image
+constexpr int kMaxRequests = 1024;     // B*K limit of one layer-step
+constexpr int kMaxPairs = 1024;        // L*(K+S) limit of the streaming kernel's work table
+constexpr int kCounters = 6;           // tok_hits, tok_misses, uniq_hits, uniq_misses, overlap, pairs
+
+// Device-side error codes written to DevStack::err (first writer wins).
+enum : int {
+  kErrNone = 0,
+  kErrWaitFull = 1,     // consumer gave up waiting for a weight row
+  kErrWaitEmpty = 2,    // producer gave up waiting for a free stage
+  kErrBadIndex = 3,     // an expert id or slot index outside its range
+  kErrDrain = 4         // copies still in flight when a kernel bailed out
+};
+
+// Everything the kernels need, passed by value.
+struct DevStack {
+  int L, H, N, K, I, S, Is, B, C;
+  int shared_gate, renorm, wbytes;     // wbytes: 4 (float32) or 2 (bfloat16)
+  int policy;
+  float beta;
+  int has_prev;                        // 0 on the first step after a reset
+  size_t slot_bytes, shared_bytes;     // bytes of one routed / shared expert block
+
+  const char* router;                  // [L][N][H]
+  const char* shared_gate_w;           // [L][H]
+  const char* shared_blocks;           // [L][S][shared_bytes]
+  char* slots;                         // [L][C][slot_bytes]
+
+  int* expert_of_slot;                 // [L][C]   -1 = empty
+  int* slot_of_expert;                 // [L][N]   -1 = not resident
+  unsigned long long* stamp;           // [L][C]
+  unsigned* freq;                      // [L][C]
+  unsigned long long* clock;           // [L]
+  unsigned* prev_mask;                 // [L][B][kMaskWords]
+  unsigned long long* counters;        // [L][kCounters]
+
+  float* shared_scale;                 // [L][B]
+  int* last_overlap;                   // [L][B]   -1 when not counted
+  // Step trace, one block so that a single copy brings it to the host:
+  // n_unique[L] | requests[L][B*K] | hit[L][B*K] | slot[L][B*K] | evicted[L][B*K]
+  int* trace;
+  int* err;
+};
+
+__host__ __device__ inline int trace_ints(int L, int BK) { return L + 4 * L * BK; }
+__host__ __device__ inline int* trace_n_unique(int* t) { return t; }
+__host__ __device__ inline int* trace_requests(int* t, int L, int BK) { return t + L; }
+__host__ __device__ inline int* trace_hit(int* t, int L, int BK) { return t + L + L * BK; }
+__host__ __device__ inline int* trace_slot(int* t, int L, int BK) { return t + L + 2 * L * BK; }
+__host__ __device__ inline int* trace_evicted(int* t, int L, int BK) { return t + L + 3 * L * BK; }
+
+// Streaming FFN launch description (batch 1).
+struct FfnArgs {
+  DevStack d;
+  const float* hidden_in;              // [L][1][H]
+  const float* gates;                  // [L][1][K]
+  int phase;                           // 0: resident (hits + shared), all layers; 1: misses of `layer`
+  int layer;
+  float* partial;                      // [2][L][grid][H]
+  int* contrib;                        // [2][L][2]  (first CTA, last CTA) contributing; first > last = none
+  int grid_cap;                        // CTAs per phase the partial buffer is laid out for
+};
+
+cudaError_t launch_route(const DevStack& d, const float* hidden_in, int* ids, float* gates,
+                         int* contrib, cudaStream_t st);
+cudaError_t launch_ffn_stream(const FfnArgs& a, int grid, cudaStream_t st);
+cudaError_t launch_combine(const FfnArgs& a, float* hidden_out, cudaStream_t st);
+size_t ffn_stream_smem_bytes(int H, int wbytes, int* stages_out);
+bool ffn_stream_supported(int H, int wbytes);
+
+}  // namespace remoe

@@ -1,0 +1,329 @@
+// Router GEMV, softmax, top-K gating, reuse statistic and cache directory update.
+//
+// One CTA per (layer, sequence) computes the N router logits (Sec. 3.1: h^T theta_gate) with
+// one warp per expert row, 128-bit loads and shuffle reductions.  Warp 0 then takes the
+// softmax over all N logits, selects the K largest logits (equal logits: lower index first),
+// emits ids and gate weights, and updates the reuse statistic |E_t n E_{t-1}| (Eq. 1) from
+// N-bit selection masks.  The directory update (App. A.1-A.2: hits and misses judged against
+// the state before the step, then serve-and-admit with LRU/FIFO/LFU victims) is integer
+// work done by one warp per layer, with one cache slot per lane during victim search.
+#include "remoe_internal.cuh"
+
+#include <math_constants.h>
+
+namespace remoe {
+
+namespace {
+
+constexpr unsigned kFull = 0xffffffffu;
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(kFull, v, o);
+  return v;
+}
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(kFull, v, o));
+  return v;
+}
+
+// Dot product of one weight row (H elements, 16-byte aligned) with h, by one warp.
+__device__ __forceinline__ float row_dot(const char* row, const float* __restrict__ h, int H,
+                                         int wbytes, int lane) {
+  float acc = 0.f;
+  if (wbytes == 4) {
+    const float4* r4 = reinterpret_cast<const float4*>(row);
+    const float4* h4 = reinterpret_cast<const float4*>(h);
+    for (int c = lane; c < H / 4; c += 32) {
+      float4 w = __ldg(r4 + c);
+      float4 x = __ldg(h4 + c);
+      acc = fmaf(w.x, x.x, acc);
+      acc = fmaf(w.y, x.y, acc);
+      acc = fmaf(w.z, x.z, acc);
+      acc = fmaf(w.w, x.w, acc);
+    }
+  } else {
+    const uint4* r4 = reinterpret_cast<const uint4*>(row);
+    const float4* h4 = reinterpret_cast<const float4*>(h);
+    for (int c = lane; c < H / 8; c += 32) {
+      uint4 w = __ldg(r4 + c);
+      float4 x0 = __ldg(h4 + 2 * c);
+      float4 x1 = __ldg(h4 + 2 * c + 1);
+      acc = fmaf(__uint_as_float(w.x << 16), x0.x, acc);
+      acc = fmaf(__uint_as_float(w.x & 0xffff0000u), x0.y, acc);
+      acc = fmaf(__uint_as_float(w.y << 16), x0.z, acc);
+      acc = fmaf(__uint_as_float(w.y & 0xffff0000u), x0.w, acc);
+      acc = fmaf(__uint_as_float(w.z << 16), x1.x, acc);
+      acc = fmaf(__uint_as_float(w.z & 0xffff0000u), x1.y, acc);
+      acc = fmaf(__uint_as_float(w.w << 16), x1.z, acc);
+      acc = fmaf(__uint_as_float(w.w & 0xffff0000u), x1.w, acc);
+    }
+  }
+  return warp_sum(acc);
+}
+
+struct DirSmem {
+  unsigned long long stamp[kMaxSlots];
+  int eos[kMaxSlots];
+  unsigned freq[kMaxSlots];
+  int soe[kMaxRouted];
+  int uniq[kMaxRequests];
+  unsigned char hitf[kMaxRequests];
+  unsigned seen[kMaskWords];
+};
+
+// Cache resolution for one layer by one warp.  `flat` holds the step's B*K requested ids in
+// (sequence, rank) order (App. E.2.3: R); U = Unique(R) keeps first occurrences.
+__device__ void resolve_layer(const DevStack& d, int l, const int* flat, int n_flat, DirSmem& sm,
+                              int lane, int* contrib) {
+  const int C = d.C, N = d.N, BK = d.B * d.K;
+  for (int s = lane; s < C; s += 32) {
+    sm.eos[s] = d.expert_of_slot[l * C + s];
+    sm.stamp[s] = d.stamp[l * C + s];
+    sm.freq[s] = d.freq[l * C + s];
+  }
+  for (int e = lane; e < N; e += 32) sm.soe[e] = d.slot_of_expert[l * N + e];
+  if (lane < kMaskWords) sm.seen[lane] = 0u;
+  __syncwarp();
+
+  const unsigned lt = (1u << lane) - 1u;
+  int n_u = 0, tok_h = 0;
+  for (int base = 0; base < n_flat; base += 32) {
+    const int i = base + lane;
+    const bool valid = i < n_flat;
+    int e = valid ? flat[i] : -1 - lane;
+    if (valid && (e < 0 || e >= N)) { atomicCAS(d.err, kErrNone, kErrBadIndex); e = 0; }
+    const bool resident = valid && sm.soe[e] >= 0;
+    tok_h += __popc(__ballot_sync(kFull, resident));
+    const unsigned same = __match_any_sync(kFull, e);
+    const bool first_here = valid && (__ffs(same) - 1 == lane);
+    const bool seen_before = valid && ((sm.seen[e >> 5] >> (e & 31)) & 1u);
+    const bool is_new = first_here && !seen_before;
+    const unsigned newmask = __ballot_sync(kFull, is_new);
+    if (is_new) {
+      sm.uniq[n_u + __popc(newmask & lt)] = e;
+      atomicOr(&sm.seen[e >> 5], 1u << (e & 31));
+    }
+    n_u += __popc(newmask);
+    __syncwarp();
+  }
+
+  int* t_req = trace_requests(d.trace, d.L, BK) + l * BK;
+  int* t_hit = trace_hit(d.trace, d.L, BK) + l * BK;
+  int* t_slot = trace_slot(d.trace, d.L, BK) + l * BK;
+  int* t_ev = trace_evicted(d.trace, d.L, BK) + l * BK;
+
+  // Classification against the pre-step state, then phase 1: touch hits in request order.
+  unsigned long long clock = d.clock[l];
+  int uniq_h = 0;
+  for (int base = 0; base < BK; base += 32) {
+    const int i = base + lane;
+    const bool valid = i < n_u;
+    const int e = valid ? sm.uniq[i] : -1;
+    const int s = valid ? sm.soe[e] : -1;
+    const bool hit = s >= 0;
+    const unsigned hm = __ballot_sync(kFull, hit);
+    if (hit) {
+      if (d.policy != REMOE_POLICY_FIFO) sm.stamp[s] = clock + 1 + __popc(hm & lt);
+      sm.freq[s] += 1u;
+    }
+    clock += __popc(hm);
+    uniq_h += __popc(hm);
+    if (i < BK) {
+      t_req[i] = e;
+      t_hit[i] = valid ? (hit ? 1 : 0) : 0;
+      t_slot[i] = s;
+      t_ev[i] = -1;
+      sm.hitf[i] = hit ? 1 : 0;
+    }
+    __syncwarp();
+  }
+
+  // Phase 2: admit misses in request order.  Victim: lowest empty slot; else the oldest
+  // (LFU: least used, then oldest) occupant that is not part of this step's request; only if
+  // every slot holds one of this step's experts, the oldest of all.
+  for (int i = 0; i < n_u; ++i) {
+    if (sm.hitf[i]) continue;
+    const int e = sm.uniq[i];
+    unsigned long long best = ~0ull;
+    int best_s = -1;
+    for (int s = lane; s < C; s += 32) {
+      const int occ = sm.eos[s];
+      unsigned long long key;
+      if (occ < 0) {
+        key = (unsigned long long)s;
+      } else {
+        const unsigned long long cls = ((sm.seen[occ >> 5] >> (occ & 31)) & 1u) ? 2ull : 1ull;
+        const unsigned long long f =
+            d.policy == REMOE_POLICY_LFU ? (unsigned long long)min(sm.freq[s], 0x3fffffu) : 0ull;
+        key = (cls << 62) | (f << 40) | (sm.stamp[s] & ((1ull << 40) - 1ull));
+      }
+      if (key < best) { best = key; best_s = s; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const unsigned long long ok = __shfl_xor_sync(kFull, best, o);
+      const int os = __shfl_xor_sync(kFull, best_s, o);
+      if (os >= 0 && (best_s < 0 || ok < best || (ok == best && os < best_s))) { best = ok; best_s = os; }
+    }
+    if (lane == 0) {
+      const int ev = sm.eos[best_s];
+      if (ev >= 0) sm.soe[ev] = -1;
+      sm.eos[best_s] = e;
+      sm.soe[e] = best_s;
+      clock += 1;
+      sm.stamp[best_s] = clock;
+      sm.freq[best_s] = 1u;
+      t_slot[i] = best_s;
+      t_ev[i] = ev;
+    }
+    __syncwarp();
+  }
+
+  for (int s = lane; s < C; s += 32) {
+    d.expert_of_slot[l * C + s] = sm.eos[s];
+    d.stamp[l * C + s] = sm.stamp[s];
+    d.freq[l * C + s] = sm.freq[s];
+  }
+  for (int e = lane; e < N; e += 32) d.slot_of_expert[l * N + e] = sm.soe[e];
+  if (lane == 0) {
+    d.clock[l] = clock;
+    unsigned long long* c = d.counters + (size_t)l * kCounters;
+    c[0] += (unsigned long long)tok_h;
+    c[1] += (unsigned long long)(n_flat - tok_h);
+    c[2] += (unsigned long long)uniq_h;
+    c[3] += (unsigned long long)(n_u - uniq_h);
+    trace_n_unique(d.trace)[l] = n_u;
+    contrib[(d.L + l) * 2 + 0] = 1;      // no miss-phase contribution yet for this layer
+    contrib[(d.L + l) * 2 + 1] = 0;
+  }
+}
+
+__global__ void __launch_bounds__(256) route_kernel(DevStack d, const float* __restrict__ hidden_in,
+                                                    int* __restrict__ ids, float* __restrict__ gates,
+                                                    int* contrib) {
+  __shared__ float z[kMaxRouted];
+  __shared__ int s_ids[32];
+  __shared__ float s_g[32];
+  __shared__ DirSmem dir;
+
+  const int lb = blockIdx.x;
+  const int l = lb / d.B;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const float* h = hidden_in + (size_t)lb * d.H;
+  const size_t row_bytes = (size_t)d.H * d.wbytes;
+
+  for (int e = warp; e < d.N; e += 8) {
+    const float acc = row_dot(d.router + ((size_t)l * d.N + e) * row_bytes, h, d.H, d.wbytes, lane);
+    if (lane == 0) z[e] = acc;
+  }
+  if (warp == 7) {
+    float sc = 1.f;
+    if (d.shared_gate) {
+      const float dot = row_dot(d.shared_gate_w + (size_t)l * row_bytes, h, d.H, d.wbytes, lane);
+      sc = 1.f / (1.f + expf(-dot));
+    }
+    if (lane == 0) d.shared_scale[lb] = sc;
+  }
+  __syncthreads();
+  if (warp != 0) return;
+
+  // Softmax over all N logits and top-K on the (optionally residency-biased) logits.
+  float v[kMaskWords], sc[kMaskWords];
+  float m = -CUDART_INF_F;
+#pragma unroll
+  for (int j = 0; j < kMaskWords; ++j) {
+    const int e = lane + 32 * j;
+    v[j] = e < d.N ? z[e] : -CUDART_INF_F;
+    sc[j] = v[j];
+    if (d.beta != 0.f && e < d.N && d.slot_of_expert[l * d.N + e] >= 0) sc[j] += d.beta;
+    m = fmaxf(m, v[j]);
+  }
+  m = warp_max(m);
+  float sum = 0.f;
+#pragma unroll
+  for (int j = 0; j < kMaskWords; ++j)
+    if (lane + 32 * j < d.N) sum += expf(v[j] - m);
+  sum = warp_sum(sum);
+
+  unsigned taken = 0u;
+  for (int k = 0; k < d.K; ++k) {
+    float best = -CUDART_INF_F;
+    int idx = INT_MAX;
+#pragma unroll
+    for (int j = 0; j < kMaskWords; ++j) {
+      const int e = lane + 32 * j;
+      if (e < d.N && !((taken >> j) & 1u) && (idx == INT_MAX || sc[j] > best)) { best = sc[j]; idx = e; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float ob = __shfl_xor_sync(kFull, best, o);
+      const int oi = __shfl_xor_sync(kFull, idx, o);
+      if (oi != INT_MAX && (idx == INT_MAX || ob > best || (ob == best && oi < idx))) { best = ob; idx = oi; }
+    }
+    if ((idx & 31) == lane) taken |= 1u << (idx >> 5);
+    if (lane == 0) {
+      s_ids[k] = idx;
+      s_g[k] = expf(z[idx] - m) / sum;
+    }
+  }
+  __syncwarp();
+  if (lane == 0 && d.renorm) {
+    float t = 0.f;
+    for (int k = 0; k < d.K; ++k) t += s_g[k];
+    for (int k = 0; k < d.K; ++k) s_g[k] /= t;
+  }
+  __syncwarp();
+  if (lane < d.K) {
+    ids[(size_t)lb * d.K + lane] = s_ids[lane];
+    gates[(size_t)lb * d.K + lane] = s_g[lane];
+  }
+
+  // Reuse: |E_t n E_{t-1}| from selection bit masks (Eq. 1); counted from the second step on.
+  int ov = 0;
+#pragma unroll
+  for (int j = 0; j < kMaskWords; ++j) {
+    const unsigned word = __ballot_sync(kFull, (taken >> j) & 1u);
+    if (lane == 0) {
+      unsigned* pm = d.prev_mask + (size_t)lb * kMaskWords + j;
+      if (d.has_prev) ov += __popc(word & *pm);
+      *pm = word;
+    }
+  }
+  if (lane == 0) {
+    d.last_overlap[lb] = d.has_prev ? ov : -1;
+    if (d.has_prev) {
+      atomicAdd(d.counters + (size_t)l * kCounters + 4, (unsigned long long)ov);
+      atomicAdd(d.counters + (size_t)l * kCounters + 5, 1ull);
+    }
+  }
+  if (d.B == 1) resolve_layer(d, l, s_ids, d.K, dir, lane, contrib);
+}
+
+__global__ void __launch_bounds__(32) resolve_kernel(DevStack d, const int* __restrict__ ids, int* contrib) {
+  __shared__ DirSmem dir;
+  __shared__ int flat[kMaxRequests];
+  const int l = blockIdx.x, lane = threadIdx.x;
+  const int BK = d.B * d.K;
+  for (int i = lane; i < BK; i += 32) flat[i] = ids[(size_t)l * BK + i];
+  __syncwarp();
+  resolve_layer(d, l, flat, BK, dir, lane, contrib);
+}
+
+}  // namespace
+
+cudaError_t launch_route(const DevStack& d, const float* hidden_in, int* ids, float* gates,
+                         int* contrib, cudaStream_t st) {
+  route_kernel<<<d.L * d.B, 256, 0, st>>>(d, hidden_in, ids, gates, contrib);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  if (d.B > 1) {
+    resolve_kernel<<<d.L, 32, 0, st>>>(d, ids, contrib);
+    e = cudaGetLastError();
+  }
+  return e;
+}
+
+}  // namespace remoe

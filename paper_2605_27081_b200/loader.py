@@ -1,0 +1,54 @@
+"""Put a seeded synthetic workload where the library expects it.
+
+Routed experts go to page-locked host memory (the library fetches misses from there),
+router and shared-expert weights are copied to the device once.  No arithmetic of the
+decode path happens here.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import synth
+from .binding import Stack
+
+
+class LoadedWorkload:
+    """A stack plus the host-side tensors it borrows.
+
+    ``distinct_experts``: generate only that many distinct routed blocks per layer and let
+    the remaining expert ids alias them (saves host memory and generation time when only
+    timing matters); ``None`` generates all N blocks per layer.
+    """
+
+    def __init__(self, shape: synth.Shape, cache_slots: int, seed: int = 0, stream: int | None = None,
+                 distinct_experts: int | None = None, threads: int | None = None):
+        self.shape, self.cache_slots, self.seed = shape, cache_slots, seed
+        L, N = shape.n_layers, shape.n_routed
+        nd = N if distinct_experts is None else min(N, int(distinct_experts))
+        self.n_distinct = nd
+        elems = synth.expert_block_elems(shape.hidden, shape.inter_routed)
+        np_dt = np.uint16 if shape.weight_dtype == 1 else np.float32
+        gen_shape = synth.Shape(**{**shape.asdict(), "n_routed": nd})
+        self._store_t = torch.empty(L * nd * elems * shape.elem_bytes, dtype=torch.uint8, pin_memory=True)
+        self.store = self._store_t.numpy().view(np_dt).reshape(L, nd, elems)
+        synth.fill_expert_store(seed, gen_shape, self.store, threads=threads)
+        self.routers = [synth.gen_router(seed, shape, l) for l in range(L)]
+        self.shared_gates = [synth.gen_shared_gate(seed, shape, l) for l in range(L)] if shape.shared_gate else None
+        self.shared = [[synth.gen_shared_block(seed, shape, l, i) for i in range(shape.n_shared)] for l in range(L)]
+
+        self.stack = Stack(shape, cache_slots, stream)
+        base = self._store_t.data_ptr()
+        blk = elems * shape.elem_bytes
+        for l in range(L):
+            self.stack.load_router(l, self.routers[l], None if self.shared_gates is None else self.shared_gates[l])
+            for i in range(shape.n_shared):
+                self.stack.load_shared(l, i, self.shared[l][i])
+            ptrs = [base + (l * nd + (e % nd)) * blk for e in range(N)]
+            self.stack.load_experts_host(l, 0, ptrs, keep=self._store_t)
+
+    def expert_block(self, layer: int, expert: int) -> np.ndarray:
+        return self.store[layer, expert % self.n_distinct]
+
+    def close(self):
+        self.stack.close()

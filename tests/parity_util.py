@@ -1,0 +1,122 @@
+"""Helpers that set the CUDA library beside the CPU oracle on the same seeded inputs."""
+from __future__ import annotations
+
+import numpy as np
+
+import synth
+from oracle import remoe_oracle as orc
+
+TOL = {0: 1e-4, 1: 2e-2}          # max|d| / max|ref| : float32 weights, bf16 weights
+NEAR_TIE = 1e-5                   # logit margin below which selected ids may differ
+
+
+def widen(shape, a):
+    return synth.bf16_bits_to_f32(a) if shape.weight_dtype == 1 else a
+
+
+def oracle_for(wl, policy="lru", reroute_beta=0.0):
+    """An OracleStack reading the very arrays the library was loaded from."""
+    s = wl.shape
+    routers = [widen(s, r) for r in wl.routers]
+    sg = None if wl.shared_gates is None else [widen(s, g) for g in wl.shared_gates]
+
+    def ew(l, e):
+        return synth.expert_matrices(widen(s, wl.expert_block(l, e)), s.hidden, s.inter_routed)
+
+    def sw(l, i):
+        return synth.expert_matrices(widen(s, wl.shared[l][i]), s.hidden, s.inter_shared)
+
+    return orc.OracleStack(s, wl.cache_slots, routers, ew, sw, shared_gates=sg, policy=policy,
+                           reroute_beta=reroute_beta)
+
+
+def rel_err(got, ref):
+    ref = np.asarray(ref, dtype=np.float64)
+    denom = np.max(np.abs(ref))
+    return float(np.max(np.abs(np.asarray(got, dtype=np.float64) - ref)) / (denom if denom > 0 else 1.0))
+
+
+class StepChecker:
+    """Feeds one step to both sides and compares ids, gates, cache trace and outputs.
+
+    Where the oracle's top-K margin is below NEAR_TIE and the library picked a different
+    (equally defensible) set, the difference is counted and the oracle is re-run for that
+    (layer, sequence) with the library's ids so that later cache states stay comparable.
+    """
+
+    def __init__(self, wl, oracle, torch, device="cuda:0"):
+        self.wl, self.o, self.torch = wl, oracle, torch
+        s = wl.shape
+        self.L, self.B, self.K, self.H = s.n_layers, s.batch, s.top_k, s.hidden
+        self.d_in = torch.empty((self.L, self.B, self.H), dtype=torch.float32, device=device)
+        self.d_out = torch.empty_like(self.d_in)
+        self.d_ids = torch.empty((self.L, self.B, self.K), dtype=torch.int32, device=device)
+        self.d_g = torch.empty((self.L, self.B, self.K), dtype=torch.float32, device=device)
+        self.near_ties = 0
+        self.max_out_err = 0.0
+        self.max_gate_err = 0.0
+
+    def gpu_step(self, h, host_api=False):
+        t = self.torch
+        if host_api:
+            out = np.empty((self.L, self.B, self.H), np.float32)
+            ids = np.empty((self.L, self.B, self.K), np.int32)
+            g = np.empty((self.L, self.B, self.K), np.float32)
+            self.wl.stack.decode_step_host(np.ascontiguousarray(h), out, ids, g)
+            return ids, g, out
+        self.d_in.copy_(t.from_numpy(np.ascontiguousarray(h)))
+        self.wl.stack.decode_step(self.d_in, self.d_out, self.d_ids, self.d_g)
+        t.cuda.synchronize()
+        return self.d_ids.cpu().numpy(), self.d_g.cpu().numpy(), self.d_out.cpu().numpy()
+
+    def step(self, h, ffn="selected", ffn_layers=None, host_api=False, check_trace=True):
+        ids, g, out = self.gpu_step(h, host_api)
+        # First pass of the oracle on a copy of nothing: we need margins before committing,
+        # so route without touching state.
+        override = {}
+        for l in range(self.L):
+            for b in range(self.B):
+                o_ids, _, margin, _, _ = self.o.route(l, h[l, b])
+                if list(o_ids) != list(ids[l, b]):
+                    assert margin < NEAR_TIE, (
+                        f"ids differ at layer {l} seq {b} with margin {margin}: {list(o_ids)} vs {list(ids[l, b])}")
+                    self.near_ties += 1
+                    override[(l, b)] = [int(e) for e in ids[l, b]]
+        r = self.o.step(h, ffn=ffn, id_override=override or None, ffn_layers=ffn_layers)
+        assert np.array_equal(r["ids"], ids)
+        ge = float(np.max(np.abs(r["gates"] - g) / np.maximum(np.abs(r["gates"]), 1e-30)))
+        self.max_gate_err = max(self.max_gate_err, ge)
+        assert ge <= 1e-4, f"gate weights off by {ge}"
+        if check_trace:
+            tr = self.wl.stack.last_step_trace()
+            for l in range(self.L):
+                n = len(r["requests"][l])
+                assert tr["n_unique"][l] == n
+                assert list(tr["requests"][l][:n]) == r["requests"][l]
+                assert [bool(x) for x in tr["hit"][l][:n]] == r["hit"][l]
+                assert list(tr["slot"][l][:n]) == r["slot"][l]
+                assert list(tr["evicted"][l][:n]) == r["evicted"][l]
+        if ffn is not None:
+            tol = TOL[self.wl.shape.weight_dtype]
+            for l in (range(self.L) if ffn_layers is None else ffn_layers):
+                e = rel_err(out[l], r["out"][l])
+                self.max_out_err = max(self.max_out_err, e)
+                assert e <= tol, f"layer {l}: output error {e} > {tol}"
+        return r, (ids, g, out)
+
+    def check_counters(self):
+        st = self.wl.stack
+        o = self.o
+        tot = st.cache_stats(-1)
+        assert tot["tok_hits"] == sum(o.tok_hits) and tot["tok_misses"] == sum(o.tok_misses)
+        assert tot["uniq_hits"] == sum(o.uniq_hits) and tot["uniq_misses"] == sum(o.uniq_misses)
+        assert tot["steps"] == o.steps
+        assert tot["h2d_bytes"] == sum(o.uniq_misses) * synth.expert_block_bytes(self.wl.shape)
+        for l in range(self.L):
+            c = st.cache_stats(l)
+            assert (c["tok_hits"], c["tok_misses"], c["uniq_hits"], c["uniq_misses"]) == (
+                o.tok_hits[l], o.tok_misses[l], o.uniq_hits[l], o.uniq_misses[l])
+            ov, pairs = st.reuse_stats(l)
+            assert (ov, pairs) == (o.overlap_sum[l], o.pairs_counted[l])
+        ov, pairs = st.reuse_stats(-1)
+        assert (ov, pairs) == (sum(o.overlap_sum), sum(o.pairs_counted))

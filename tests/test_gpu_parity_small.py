@@ -1,0 +1,111 @@
+"""GPU parity on small shapes: every step of the path against the CPU oracle, element by element."""
+import numpy as np
+import pytest
+
+import synth
+
+pytestmark = pytest.mark.gpu
+
+
+def _run(shape, cache_slots, rho, steps, seed=0, dense_steps=2, host_api_every=0, policy=None, beta=0.0):
+    import torch
+    from paper_2605_27081_b200.loader import LoadedWorkload
+    from parity_util import StepChecker, oracle_for
+
+    wl = LoadedWorkload(shape, cache_slots, seed)
+    try:
+        pol_name = "lru"
+        if policy is not None:
+            wl.stack.set_policy(policy)
+            pol_name = {0: "lru", 1: "fifo", 2: "lfu"}[policy]
+        if beta:
+            wl.stack.set_reroute_beta(beta)
+        chk = StepChecker(wl, oracle_for(wl, pol_name, beta), torch)
+        hs = synth.HiddenStream(seed, shape, rho)
+        last = None
+        for t in range(steps):
+            h = hs.step()
+            host = bool(host_api_every) and t % host_api_every == host_api_every - 1
+            last, _ = chk.step(h, ffn="dense" if t < dense_steps else "selected", host_api=host)
+        chk.check_counters()
+        o, p, ir = wl.stack.reuse_stats(-1, want_last_ir=True)
+        exp = last["overlap"].reshape(-1)
+        assert np.allclose(ir, np.where(exp < 0, -1.0, exp / shape.top_k))
+        return chk
+    finally:
+        wl.close()
+
+
+def test_tiny_fp32_config_full():
+    cfg = synth.config("tiny_fp32")
+    chk = _run(cfg["shape"], cfg["cache_slots"], cfg["rhos"][0], cfg["steps"], cfg["seed"], dense_steps=64,
+               host_api_every=5)
+    assert chk.max_out_err <= 1e-4
+
+
+@pytest.mark.parametrize("shape,c,rho", [
+    (synth.Shape(3, 256, 20, 3, 72, 2, 40, 0, 0, 1, 1), 5, 0.6),        # bf16, shared experts, ragged I
+    (synth.Shape(2, 512, 33, 4, 50, 1, 130, 1, 0, 1, 1), 4, 0.8),       # N not a multiple of 32, C = K, sigmoid gate
+    (synth.Shape(4, 1024, 128, 8, 24, 0, 0, 0, 1, 1, 1), 32, 0.5),      # renormalised top-8 of 128
+    (synth.Shape(2, 2048, 64, 6, 44, 2, 44, 0, 0, 1, 1), 16, 0.9),      # full hidden width
+    (synth.Shape(2, 128, 9, 9, 16, 0, 0, 0, 0, 0, 1), 9, 0.3),          # K = N = C, float32
+    (synth.Shape(1, 1024, 200, 5, 8, 1, 8, 1, 1, 0, 1), 200, 0.0),      # all resident, float32, N = 200
+])
+def test_small_shapes(shape, c, rho):
+    _run(shape, c, rho, steps=24, seed=1, dense_steps=2, host_api_every=7)
+
+
+def test_many_layers_span_ctas():
+    """Enough rows that CTAs cross expert and layer boundaries in the streaming kernel."""
+    shape = synth.Shape(12, 512, 16, 4, 300, 1, 300, 0, 0, 1, 1)
+    _run(shape, 6, 0.7, steps=12, seed=2, dense_steps=1)
+
+
+@pytest.mark.parametrize("policy", [1, 2])
+def test_other_policies(policy):
+    _run(synth.Shape(2, 256, 24, 3, 16, 0, 0, 0, 0, 0, 1), 5, 0.5, steps=60, seed=3, dense_steps=0, policy=policy)
+
+
+def test_reroute_beta():
+    _run(synth.Shape(2, 256, 24, 3, 16, 0, 0, 0, 0, 0, 1), 5, 0.3, steps=40, seed=4, dense_steps=0, beta=0.5)
+
+
+def test_reset_and_errors():
+    import torch
+    from paper_2605_27081_b200 import binding as B
+    from paper_2605_27081_b200.loader import LoadedWorkload
+    from parity_util import StepChecker, oracle_for
+
+    shape = synth.Shape(2, 256, 16, 2, 32, 0, 0, 0, 0, 0, 1)
+    rc, h = B.remoe_stack_create(shape, 1)
+    assert rc == B.REMOE_E_CAPACITY
+    rc, h = B.remoe_stack_create(synth.Shape(2, 250, 16, 2, 32), 4)
+    assert rc == B.REMOE_E_UNSUPPORTED
+    rc, h = B.remoe_stack_create(synth.Shape(0, 256, 16, 2, 32), 4)
+    assert rc == B.REMOE_E_ARG
+    rc, h = B.remoe_stack_create(shape, 4)
+    assert rc == 0
+    x = torch.zeros((2, 1, 256), device="cuda")
+    ids = torch.zeros((2, 1, 2), dtype=torch.int32, device="cuda")
+    g = torch.zeros((2, 1, 2), device="cuda")
+    assert B.remoe_decode_step(h, x, x.clone(), ids, g) == B.REMOE_E_NOT_LOADED
+    assert B.remoe_decode_step(h, None, x, ids, g) == B.REMOE_E_ARG
+    pageable = np.zeros(3 * 256 * 32, np.float32)
+    assert B.remoe_load_experts_host(h, 0, 0, [pageable]) == B.REMOE_E_NOT_PINNED
+    assert B.remoe_load_experts_host(h, 0, 15, [pageable, pageable]) == B.REMOE_E_ARG
+    assert B.remoe_load_router(h, 5, pageable) == B.REMOE_E_ARG
+    B.remoe_stack_destroy(h)
+
+    wl = LoadedWorkload(shape, 4, seed=5)
+    try:
+        chk = StepChecker(wl, oracle_for(wl), torch)
+        hs = synth.HiddenStream(5, shape, 0.5).take(10)
+        for t in range(6):
+            chk.step(hs[t])
+        wl.stack.cache_reset()
+        chk.o.reset()
+        for t in range(10):
+            chk.step(hs[t])
+        chk.check_counters()
+    finally:
+        wl.close()
