@@ -153,11 +153,17 @@ int remoe_set_policy(remoe_stack*, int32_t policy);
  * unbiased softmax. */
 int remoe_set_reroute_beta(remoe_stack*, float beta);
 
-/* Kernel timing aid: with `on` != 0 every expert-streaming kernel launch is bracketed by
- * CUDA events on its own stream.  remoe_kernel_time returns the summed duration (ms), the
- * number of launches and the weight bytes they streamed since profiling was switched on. */
+/* Kernel timing aid: with `on` != 0 every launch of the expert-streaming kernel is bracketed
+ * by CUDA events on the stream it runs on.  remoe_kernel_time returns, for phase 0 (resident
+ * experts: cache hits + shared, one launch per step) or phase 1 (just-fetched experts, one
+ * launch per layer with misses), the summed duration in ms, the number of launches and the
+ * expert-weight bytes they streamed since profiling was switched on.  Waits for the events. */
 int remoe_set_profiling(remoe_stack*, int32_t on);
-int remoe_kernel_time(remoe_stack*, double* ms_sum, uint64_t* launches, uint64_t* weight_bytes);
+int remoe_kernel_time(remoe_stack*, int32_t phase, double* ms_sum, uint64_t* launches,
+                      uint64_t* weight_bytes);
+
+/* Number of kernels this stack has launched since creation (all kinds). */
+int remoe_launch_count(remoe_stack*, uint64_t* launches);
 
 /* Text of the last CUDA runtime error seen by this stack ("" if none). */
 const char* remoe_last_cuda_error(const remoe_stack*);

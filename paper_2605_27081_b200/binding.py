@@ -24,7 +24,7 @@ EXPORTS = [
     "remoe_stack_create", "remoe_load_router", "remoe_load_shared", "remoe_load_experts_host",
     "remoe_decode_step", "remoe_decode_step_host", "remoe_last_step_trace", "remoe_cache_stats",
     "remoe_reuse_stats", "remoe_cache_reset", "remoe_set_policy", "remoe_set_reroute_beta",
-    "remoe_set_profiling", "remoe_kernel_time", "remoe_last_cuda_error", "remoe_stack_destroy",
+    "remoe_set_profiling", "remoe_kernel_time", "remoe_launch_count", "remoe_last_cuda_error", "remoe_stack_destroy",
     "remoe_strerror",
 ]
 
@@ -72,7 +72,8 @@ def lib():
         L.remoe_set_policy.argtypes = [vp, i32]
         L.remoe_set_reroute_beta.argtypes = [vp, C.c_float]
         L.remoe_set_profiling.argtypes = [vp, i32]
-        L.remoe_kernel_time.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
+        L.remoe_kernel_time.argtypes = [vp, i32, C.POINTER(C.c_double), C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
+        L.remoe_launch_count.argtypes = [vp, C.POINTER(C.c_uint64)]
         L.remoe_last_cuda_error.argtypes = [vp]
         L.remoe_last_cuda_error.restype = C.c_char_p
         L.remoe_stack_destroy.argtypes = [vp]
@@ -174,10 +175,16 @@ def remoe_set_profiling(h, on):
     return lib().remoe_set_profiling(h, int(bool(on)))
 
 
-def remoe_kernel_time(h):
+def remoe_kernel_time(h, phase):
     ms, n, b = C.c_double(), C.c_uint64(), C.c_uint64()
-    rc = lib().remoe_kernel_time(h, C.byref(ms), C.byref(n), C.byref(b))
+    rc = lib().remoe_kernel_time(h, int(phase), C.byref(ms), C.byref(n), C.byref(b))
     return rc, float(ms.value), int(n.value), int(b.value)
+
+
+def remoe_launch_count(h):
+    n = C.c_uint64()
+    rc = lib().remoe_launch_count(h, C.byref(n))
+    return rc, int(n.value)
 
 
 def remoe_last_cuda_error(h) -> str:
@@ -252,10 +259,15 @@ class Stack:
     def set_profiling(self, on):
         self._ck(remoe_set_profiling(self.h, on), "remoe_set_profiling")
 
-    def kernel_time(self):
-        rc, ms, n, b = remoe_kernel_time(self.h)
+    def kernel_time(self, phase):
+        rc, ms, n, b = remoe_kernel_time(self.h, phase)
         self._ck(rc, "remoe_kernel_time")
         return ms, n, b
+
+    def launch_count(self):
+        rc, n = remoe_launch_count(self.h)
+        self._ck(rc, "remoe_launch_count")
+        return n
 
     def close(self):
         if self.h is not None:

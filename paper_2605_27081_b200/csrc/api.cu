@@ -25,6 +25,7 @@ using namespace remoe;
 struct EvPair {
   cudaEvent_t a, b;
   uint64_t bytes;
+  int phase;
 };
 
 struct remoe_stack {
@@ -53,8 +54,9 @@ struct remoe_stack {
   // profiling
   bool profiling = false;
   std::vector<EvPair> ev_used, ev_free;
-  double prof_ms = 0.0;
-  uint64_t prof_launches = 0, prof_bytes = 0;
+  double prof_ms[2] = {0.0, 0.0};
+  uint64_t prof_launches[2] = {0, 0}, prof_bytes[2] = {0, 0};
+  uint64_t kernel_launches = 0;          // every kernel this stack has launched
   std::string cuda_err;
   int policy = REMOE_POLICY_LRU;
   float beta = 0.f;
@@ -127,7 +129,7 @@ bool everything_loaded(const remoe_stack* s) {
   return true;
 }
 
-int prof_begin(remoe_stack* s, cudaStream_t st, uint64_t bytes) {
+int prof_begin(remoe_stack* s, cudaStream_t st, uint64_t bytes, int phase) {
   if (!s->profiling) return REMOE_OK;
   EvPair p;
   if (!s->ev_free.empty()) {
@@ -138,6 +140,7 @@ int prof_begin(remoe_stack* s, cudaStream_t st, uint64_t bytes) {
     CK(cudaEventCreate(&p.b));
   }
   p.bytes = bytes;
+  p.phase = phase;
   CK(cudaEventRecord(p.a, st));
   s->ev_used.push_back(p);
   return REMOE_OK;
@@ -154,9 +157,9 @@ int prof_collect(remoe_stack* s) {
     float ms = 0.f;
     CK(cudaEventSynchronize(p.b));
     CK(cudaEventElapsedTime(&ms, p.a, p.b));
-    s->prof_ms += ms;
-    s->prof_launches += 1;
-    s->prof_bytes += p.bytes;
+    s->prof_ms[p.phase] += ms;
+    s->prof_launches[p.phase] += 1;
+    s->prof_bytes[p.phase] += p.bytes;
     s->ev_free.push_back(p);
   }
   s->ev_used.clear();
@@ -345,6 +348,7 @@ int remoe_decode_step(remoe_stack* s, const float* hin, float* hout, int32_t* id
   d.beta = s->beta;
 
   CK(launch_route(d, hin, ids, gates, s->contrib, s->stream));
+  s->kernel_launches += d.B > 1 ? 2 : 1;
   CK(cudaMemcpyAsync(s->host_block, s->dev_block, s->block_ints * sizeof(int), cudaMemcpyDeviceToHost, s->stream));
   CK(cudaEventRecord(s->ev_trace, s->stream));
 
@@ -358,9 +362,10 @@ int remoe_decode_step(remoe_stack* s, const float* hin, float* hout, int32_t* id
   a.phase = 0;
   a.layer = -1;
   // The resident phase needs no host decision: enqueue it before waiting for the trace.
-  int rc = prof_begin(s, s->stream, 0);
+  int rc = prof_begin(s, s->stream, 0, 0);
   if (rc != REMOE_OK) return rc;
   CK(launch_ffn_stream(a, s->grid, s->stream));
+  s->kernel_launches += 1;
   rc = prof_end(s, s->stream);
   if (rc != REMOE_OK) return rc;
   const size_t prof_slot = s->profiling ? s->ev_used.size() - 1 : 0;
@@ -400,15 +405,17 @@ int remoe_decode_step(remoe_stack* s, const float* hin, float* hout, int32_t* id
       CK(cudaStreamWaitEvent(s->stream, s->ev_layer[l], 0));
       a.phase = 1;
       a.layer = l;
-      rc = prof_begin(s, s->stream, (uint64_t)misses * d.slot_bytes);
+      rc = prof_begin(s, s->stream, (uint64_t)misses * d.slot_bytes, 1);
       if (rc != REMOE_OK) return rc;
       CK(launch_ffn_stream(a, s->grid, s->stream));
+  s->kernel_launches += 1;
       rc = prof_end(s, s->stream);
       if (rc != REMOE_OK) return rc;
     }
   }
   if (s->profiling) s->ev_used[prof_slot].bytes = resident_bytes;
   CK(launch_combine(a, hout, s->stream));
+  s->kernel_launches += 1;
   return REMOE_OK;
 }
 
@@ -513,19 +520,27 @@ int remoe_set_profiling(remoe_stack* s, int32_t on) {
   int rc = prof_collect(s);
   if (rc != REMOE_OK) return rc;
   s->profiling = on != 0;
-  s->prof_ms = 0.0;
-  s->prof_launches = 0;
-  s->prof_bytes = 0;
+  for (int p = 0; p < 2; ++p) {
+    s->prof_ms[p] = 0.0;
+    s->prof_launches[p] = 0;
+    s->prof_bytes[p] = 0;
+  }
   return REMOE_OK;
 }
 
-int remoe_kernel_time(remoe_stack* s, double* ms_sum, uint64_t* launches, uint64_t* bytes) {
-  if (!s) return REMOE_E_ARG;
+int remoe_kernel_time(remoe_stack* s, int32_t phase, double* ms_sum, uint64_t* launches, uint64_t* bytes) {
+  if (!s || phase < 0 || phase > 1) return REMOE_E_ARG;
   int rc = prof_collect(s);
   if (rc != REMOE_OK) return rc;
-  if (ms_sum) *ms_sum = s->prof_ms;
-  if (launches) *launches = s->prof_launches;
-  if (bytes) *bytes = s->prof_bytes;
+  if (ms_sum) *ms_sum = s->prof_ms[phase];
+  if (launches) *launches = s->prof_launches[phase];
+  if (bytes) *bytes = s->prof_bytes[phase];
+  return REMOE_OK;
+}
+
+int remoe_launch_count(remoe_stack* s, uint64_t* launches) {
+  if (!s || !launches) return REMOE_E_ARG;
+  *launches = s->kernel_launches;
   return REMOE_OK;
 }
 

@@ -27,7 +27,7 @@ namespace {
 
 constexpr int kConsumerWarps = 8;
 constexpr int kThreads = (kConsumerWarps + 1) * 32;
-constexpr int kMaxStages = 16;
+constexpr int kMaxStages = 16;                 // multiple of kConsumerWarps
 constexpr unsigned kSpinLimit = 1u << 20;
 constexpr unsigned kFull = 0xffffffffu;
 
@@ -93,6 +93,10 @@ struct Elems<2> {
 };
 
 // Shared-memory carve-up (dynamic): barriers | row prefix table | reduce buffer | stage ring.
+// The ring depth is a multiple of the consumer-warp count, so a stage is always consumed by
+// the same warp.  That warp has waited for fill k-1 of the stage before it waits for fill k,
+// hence the barrier can never be a whole phase behind the parity it is asked about (a parity
+// wait cannot tell "phase k done" from "phase k-2 done").
 struct Layout {
   size_t bars, prefix, red, stages, total;
   int n_stages;
@@ -101,13 +105,13 @@ __host__ __device__ inline Layout make_layout(int H, int wbytes) {
   Layout y;
   y.bars = 0;
   y.prefix = 2 * kMaxStages * sizeof(uint64_t);
-  y.red = y.prefix + (size_t)(kMaxPairs + 1) * sizeof(int) + 12;           // keep 16-byte alignment
+  y.red = y.prefix + (size_t)(kMaxPairs + 1) * sizeof(int);
   y.red = (y.red + 127) / 128 * 128;
-  y.stages = y.red + (size_t)kConsumerWarps * H * sizeof(float);
+  y.stages = y.red + (size_t)kConsumerWarps * 32 * (16 / wbytes) * sizeof(float);
   const size_t stage = (size_t)3 * H * wbytes;
-  const size_t budget = 227 * 1024;
+  const size_t budget = 227 * 1024 - 1024;              // leave room for static shared memory
   int n = (int)((budget - y.stages) / stage);
-  if (n > kMaxStages) n = kMaxStages;
+  n = n >= kMaxStages ? kMaxStages : (n / kConsumerWarps) * kConsumerWarps;
   y.n_stages = n;
   y.total = y.stages + (size_t)n * stage;
   return y;
@@ -308,23 +312,26 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(const __grid_co
       }
 
       // Layer flush: add the eight private copies in warp order, write this CTA's partial.
-      float* mine = red + (size_t)warp * H;
+      // One pass per 32*kVec columns keeps the exchange buffer at a few KB.
+      float* dst = a.partial + (((size_t)a.phase * d.L + l) * a.grid_cap + blockIdx.x) * H;
+      constexpr int kPassCols = 32 * kVec;
 #pragma unroll
-      for (int it = 0; it < kIter; ++it)
+      for (int it = 0; it < kIter; ++it) {
+        float* mine = red + (size_t)warp * kPassCols + lane * kVec;
 #pragma unroll
         for (int v4 = 0; v4 < kVec / 4; ++v4)
-          *reinterpret_cast<float4*>(mine + (it * 32 + lane) * kVec + v4 * 4) =
+          *reinterpret_cast<float4*>(mine + v4 * 4) =
               make_float4(acc[it * kVec + v4 * 4], acc[it * kVec + v4 * 4 + 1], acc[it * kVec + v4 * 4 + 2],
                           acc[it * kVec + v4 * 4 + 3]);
-      consumer_bar();
-      float* dst = a.partial + (((size_t)a.phase * d.L + l) * a.grid_cap + blockIdx.x) * H;
-      for (int c = tid; c < H; c += kConsumerWarps * 32) {
-        float t = 0.f;
+        consumer_bar();
+        if (tid < kPassCols) {
+          float t = 0.f;
 #pragma unroll
-        for (int w = 0; w < kConsumerWarps; ++w) t += red[(size_t)w * H + c];
-        dst[c] = t;
+          for (int w = 0; w < kConsumerWarps; ++w) t += red[(size_t)w * kPassCols + tid];
+          dst[it * kPassCols + tid] = t;
+        }
+        consumer_bar();
       }
-      consumer_bar();
     }
   }
 }

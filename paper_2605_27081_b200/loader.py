@@ -37,15 +37,21 @@ class LoadedWorkload:
         self.shared_gates = [synth.gen_shared_gate(seed, shape, l) for l in range(L)] if shape.shared_gate else None
         self.shared = [[synth.gen_shared_block(seed, shape, l, i) for i in range(shape.n_shared)] for l in range(L)]
 
-        self.stack = Stack(shape, cache_slots, stream)
+        self.stack = self.new_stack(cache_slots, stream)
+
+    def new_stack(self, cache_slots: int, stream: int | None = None) -> Stack:
+        """Another stack (e.g. with a different capacity) borrowing the same host tensors."""
+        shape, nd = self.shape, self.n_distinct
+        stack = Stack(shape, cache_slots, stream)
         base = self._store_t.data_ptr()
-        blk = elems * shape.elem_bytes
-        for l in range(L):
-            self.stack.load_router(l, self.routers[l], None if self.shared_gates is None else self.shared_gates[l])
+        blk = synth.expert_block_bytes(shape)
+        for l in range(shape.n_layers):
+            stack.load_router(l, self.routers[l], None if self.shared_gates is None else self.shared_gates[l])
             for i in range(shape.n_shared):
-                self.stack.load_shared(l, i, self.shared[l][i])
-            ptrs = [base + (l * nd + (e % nd)) * blk for e in range(N)]
-            self.stack.load_experts_host(l, 0, ptrs, keep=self._store_t)
+                stack.load_shared(l, i, self.shared[l][i])
+            ptrs = [base + (l * nd + (e % nd)) * blk for e in range(shape.n_routed)]
+            stack.load_experts_host(l, 0, ptrs, keep=self._store_t)
+        return stack
 
     def expert_block(self, layer: int, expert: int) -> np.ndarray:
         return self.store[layer, expert % self.n_distinct]

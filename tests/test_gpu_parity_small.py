@@ -61,6 +61,14 @@ def test_many_layers_span_ctas():
     _run(shape, 6, 0.7, steps=12, seed=2, dense_steps=1)
 
 
+def test_long_streams_per_cta():
+    """Hundreds of weight rows per CTA: the stage ring wraps many times, so every stage's
+    barriers go through many phases (a ring whose stages change hands between warps would
+    let a warp run a phase ahead of the data)."""
+    shape = synth.Shape(4, 2048, 12, 6, 1280, 2, 640, 0, 0, 1, 1)
+    _run(shape, 8, 0.8, steps=10, seed=6, dense_steps=0)
+
+
 @pytest.mark.parametrize("policy", [1, 2])
 def test_other_policies(policy):
     _run(synth.Shape(2, 256, 24, 3, 16, 0, 0, 0, 0, 0, 1), 5, 0.5, steps=60, seed=3, dense_steps=0, policy=policy)
