@@ -165,6 +165,48 @@ int remoe_kernel_time(remoe_stack*, int32_t phase, double* ms_sum, uint64_t* lau
 /* Number of kernels this stack has launched since creation (all kinds). */
 int remoe_launch_count(remoe_stack*, uint64_t* launches);
 
+/*
+ * Gate-weighted SwiGLU expert sum of ONE layer without any allocation (the paper has no
+ * counterpart: this exists for embedders, not for the method).
+ *
+ *     hidden_out[0:H] = sum_{e < n_experts} scales[e] * W_down^e (silu(W_gate^e h) * (W_up^e h))
+ *
+ * For callers that cannot call cudaMalloc where they use this library -- a serving loop whose
+ * device memory is handed out once at start-up by someone else, worker threads on which the
+ * host framework bans allocator calls, a device that is already full.  The stack-based entry
+ * points above allocate their scratch at remoe_stack_create; this one keeps its scratch (one
+ * partial output vector per CTA) in a fixed device array inside the library image, 1.25 MiB on
+ * every GPU that loads the library, held until the process exits.  A call makes no cudaMalloc,
+ * no cudaFree and no allocating library call; it launches two kernels on `cuda_stream`.
+ *
+ *   hidden, weight_dtype   as in remoe_shape; hidden <= REMOE_STATIC_MAX_HIDDEN
+ *   n_experts              1 .. REMOE_STATIC_MAX_EXPERTS (routed and shared alike)
+ *   expert_blocks_dev      HOST array of n_experts DEVICE pointers, each one expert block in
+ *                          the [I, 3, H] layout above, 16-byte aligned, owned by the caller
+ *   inter                  HOST array: I of each block, 1 .. REMOE_STATIC_MAX_INTER
+ *   scales                 HOST array: gate weight (or shared-expert scale) of each block
+ *   hidden_in_dev          DEVICE [H] float32;  hidden_out_dev  DEVICE [H] float32 (overwritten)
+ *
+ * The host arrays are read before the call returns.  The result is complete when `cuda_stream`
+ * reaches the end of the call's work.  Sizes beyond the limits above, or a hidden width the
+ * kernels are not built for, are refused with REMOE_E_UNSUPPORTED before anything is launched;
+ * bad pointers with REMOE_E_ARG.  The first call on each device also looks up the scratch
+ * array's device address and sets kernel attributes for that device (with that device
+ * current), so make that first call outside any stream capture.  All calls on a device share
+ * the one scratch array: calls whose kernels could run at the same time (different streams
+ * without ordering, or several host threads) race on it and must be serialised by the caller.
+ * Each call overwrites the part of the scratch it reads, so earlier contents never matter.  If
+ * an internal bounded wait ever runs out, the output is filled with NaN rather than a wrong
+ * value.
+ */
+#define REMOE_STATIC_MAX_EXPERTS 16
+#define REMOE_STATIC_MAX_HIDDEN 2048
+#define REMOE_STATIC_MAX_INTER 65536
+int remoe_expert_ffn_static(int32_t hidden, int32_t weight_dtype, int32_t n_experts,
+                            const void* const* expert_blocks_dev, const int32_t* inter,
+                            const float* scales, const float* hidden_in_dev, float* hidden_out_dev,
+                            void* cuda_stream);
+
 /* Text of the last CUDA runtime error seen by this stack ("" if none). */
 const char* remoe_last_cuda_error(const remoe_stack*);
 

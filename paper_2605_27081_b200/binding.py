@@ -25,7 +25,7 @@ EXPORTS = [
     "remoe_decode_step", "remoe_decode_step_host", "remoe_last_step_trace", "remoe_cache_stats",
     "remoe_reuse_stats", "remoe_cache_reset", "remoe_set_policy", "remoe_set_reroute_beta",
     "remoe_set_profiling", "remoe_kernel_time", "remoe_launch_count", "remoe_last_cuda_error", "remoe_stack_destroy",
-    "remoe_strerror",
+    "remoe_strerror", "remoe_expert_ffn_static",
 ]
 
 
@@ -74,6 +74,8 @@ def lib():
         L.remoe_set_profiling.argtypes = [vp, i32]
         L.remoe_kernel_time.argtypes = [vp, i32, C.POINTER(C.c_double), C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
         L.remoe_launch_count.argtypes = [vp, C.POINTER(C.c_uint64)]
+        L.remoe_expert_ffn_static.argtypes = [i32, i32, i32, C.POINTER(vp), C.POINTER(i32), C.POINTER(C.c_float),
+                                              vp, vp, vp]
         L.remoe_last_cuda_error.argtypes = [vp]
         L.remoe_last_cuda_error.restype = C.c_char_p
         L.remoe_stack_destroy.argtypes = [vp]
@@ -185,6 +187,17 @@ def remoe_launch_count(h):
     n = C.c_uint64()
     rc = lib().remoe_launch_count(h, C.byref(n))
     return rc, int(n.value)
+
+
+def remoe_expert_ffn_static(hidden, weight_dtype, expert_blocks_dev, inter, scales, hidden_in, hidden_out,
+                            cuda_stream=None):
+    """Allocation-free expert sum of one layer; `expert_blocks_dev` are device tensors/addresses."""
+    n = len(expert_blocks_dev)
+    ptrs = (C.c_void_p * n)(*[_ptr(p) for p in expert_blocks_dev])
+    inter_a = (C.c_int32 * n)(*[int(i) for i in inter])
+    scales_a = (C.c_float * n)(*[float(x) for x in scales])
+    return lib().remoe_expert_ffn_static(int(hidden), int(weight_dtype), n, ptrs, inter_a, scales_a,
+                                         _ptr(hidden_in), _ptr(hidden_out), cuda_stream)
 
 
 def remoe_last_cuda_error(h) -> str:

@@ -1,0 +1,362 @@
+// remoe_expert_ffn_static: the gate-weighted SwiGLU expert sum of one layer for callers that
+// must not allocate device memory.
+//
+// Some embedders of this library run where cudaMalloc is off limits: inside a latency-critical
+// serving loop whose memory is carved up once at start-up by another component, under a
+// framework that forbids allocator calls on its worker threads, or in a process whose device
+// memory is already fully committed.  The regular path allocates its scratch (per-CTA partial
+// sums) when a stack is created; this entry point instead keeps that scratch in a file-scope
+// device array of fixed size that is part of the loaded module, so a call performs no
+// cudaMalloc, no cudaFree and no allocating library routine -- it only launches two kernels
+// on the caller's stream.  The price is a fixed ceiling on the problem size and one shared
+// scratch area per device.
+//
+// It is a variant of the expert-streaming kernel of ffn_stream.cu (same channel-major expert
+// block, same bulk-copy stage ring, same warp-per-triple arithmetic), restricted to one layer
+// whose experts are given directly as device pointers.
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <mutex>
+
+#include "remoe.h"
+
+namespace {
+
+constexpr int kConsumerWarps = 8;
+constexpr int kThreads = (kConsumerWarps + 1) * 32;
+constexpr int kStages = 16;                                 // multiple of kConsumerWarps
+constexpr unsigned kSpinLimit = 1u << 20;
+constexpr unsigned kFull = 0xffffffffu;
+constexpr int kMaxCtas = 160;                               // scratch rows; grids are capped to this
+constexpr int kMaxDevices = 64;
+
+// Scratch of the no-allocation entry point: one partial output vector per CTA.  Lives in the
+// module image on every device that loads the library (1.25 MiB) until the process exits.
+// Every call overwrites the rows it uses before reading them, so nothing needs clearing; two
+// calls that overlap on the GPU would race on it.
+static __device__ __align__(256) float g_static_partial[kMaxCtas * REMOE_STATIC_MAX_HIDDEN];
+
+struct StaticArgs {
+  const char* base[REMOE_STATIC_MAX_EXPERTS];
+  float scale[REMOE_STATIC_MAX_EXPERTS];
+  int prefix[REMOE_STATIC_MAX_EXPERTS + 1];                 // exclusive prefix of rows per expert
+  int n_experts;
+  int rows_per_cta;
+  const float* hidden_in;
+  float* partial;                                           // device address of g_static_partial
+  int n_active;                                             // CTAs that own at least one row
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// Bounded wait: false if the phase did not complete within the spin limit.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+  for (unsigned it = 0; it < kSpinLimit; ++it) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    if (ok) return true;
+  }
+  return false;
+}
+__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+          smem_u32(dst)),
+      "l"(__cvta_generic_to_global(src)), "r"(bytes), "r"(smem_u32(bar))
+      : "memory");
+}
+__device__ __forceinline__ void consumer_bar() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+
+template <int WB>
+struct Elems;
+template <>
+struct Elems<4> {
+  static constexpr int kVec = 4;
+  __device__ static __forceinline__ void load(const char* p, float* f) {
+    const float4 v = *reinterpret_cast<const float4*>(p);
+    f[0] = v.x; f[1] = v.y; f[2] = v.z; f[3] = v.w;
+  }
+};
+template <>
+struct Elems<2> {
+  static constexpr int kVec = 8;
+  __device__ static __forceinline__ void load(const char* p, float* f) {
+    const uint4 v = *reinterpret_cast<const uint4*>(p);
+    f[0] = __uint_as_float(v.x << 16); f[1] = __uint_as_float(v.x & 0xffff0000u);
+    f[2] = __uint_as_float(v.y << 16); f[3] = __uint_as_float(v.y & 0xffff0000u);
+    f[4] = __uint_as_float(v.z << 16); f[5] = __uint_as_float(v.z & 0xffff0000u);
+    f[6] = __uint_as_float(v.w << 16); f[7] = __uint_as_float(v.w & 0xffff0000u);
+  }
+};
+
+template <int WB, int H>
+constexpr size_t smem_bytes() {
+  return 2 * kStages * sizeof(uint64_t) + (size_t)kConsumerWarps * 32 * (16 / WB) * sizeof(float) +
+         (size_t)kStages * 3 * H * WB;
+}
+
+template <int WB, int H>
+__global__ void __launch_bounds__(kThreads, 1) ffn_static_kernel(const __grid_constant__ StaticArgs a) {
+  using E = Elems<WB>;
+  constexpr int kVec = E::kVec;
+  constexpr int kIter = H / (32 * kVec);
+  constexpr int kCols = kIter * kVec;
+  constexpr int kPassCols = 32 * kVec;
+  constexpr uint32_t kStageBytes = 3u * H * WB;
+  constexpr uint32_t kRowBytes = (uint32_t)H * WB;
+
+  extern __shared__ __align__(128) unsigned char smem[];
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem);
+  uint64_t* empty = full + kStages;
+  float* red = reinterpret_cast<float*>(smem + 2 * kStages * sizeof(uint64_t));
+  unsigned char* stages = reinterpret_cast<unsigned char*>(red + kConsumerWarps * kPassCols);
+  __shared__ int s_abort;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  if (tid == 0) {
+    s_abort = 0;
+    for (int s = 0; s < kStages; ++s) { mbar_init(full + s, 1); mbar_init(empty + s, 1); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  const int M = a.prefix[a.n_experts];
+  const int r0 = min(M, (int)blockIdx.x * a.rows_per_cta), r1 = min(M, r0 + a.rows_per_cta);
+  if (r0 >= r1) return;
+
+  if (warp == kConsumerWarps) {
+    // producer: one thread streams this CTA's channel triples into the stage ring
+    if (lane == 0) {
+      int e = 0, issued = 0;
+      bool ok = true;
+      for (int r = r0; r < r1; ++r, ++issued) {
+        while (a.prefix[e + 1] <= r) ++e;
+        const int n = r - r0, s = n % kStages;
+        if (n >= kStages &&
+            (*(volatile int*)&s_abort || !mbar_wait(empty + s, ((n / kStages) - 1) & 1))) { ok = false; break; }
+        mbar_expect_tx(full + s, kStageBytes);
+        bulk_g2s(stages + (size_t)s * kStageBytes, a.base[e] + (size_t)(r - a.prefix[e]) * kStageBytes,
+                 kStageBytes, full + s);
+      }
+      if (!ok) {
+        // let the consumers leave, then wait (bounded) for copies that are still landing
+        atomicExch(&s_abort, 1);
+        for (int n = max(0, issued - kStages); n < issued; ++n) mbar_wait(full + (n % kStages), (n / kStages) & 1);
+      }
+    }
+    return;
+  }
+
+  float hreg[kCols], acc[kCols];
+#pragma unroll
+  for (int it = 0; it < kIter; ++it)
+#pragma unroll
+    for (int v4 = 0; v4 < kVec / 4; ++v4) {
+      const float4 x = __ldg(reinterpret_cast<const float4*>(a.hidden_in + (it * 32 + lane) * kVec) + v4);
+      hreg[it * kVec + v4 * 4 + 0] = x.x; hreg[it * kVec + v4 * 4 + 1] = x.y;
+      hreg[it * kVec + v4 * 4 + 2] = x.z; hreg[it * kVec + v4 * 4 + 3] = x.w;
+    }
+#pragma unroll
+  for (int c = 0; c < kCols; ++c) acc[c] = 0.f;
+
+  int e = 0;
+  for (int r = r0 + warp; r < r1; r += kConsumerWarps) {
+    while (a.prefix[e + 1] <= r) ++e;
+    const float scale = a.scale[e];
+    const int n = r - r0, s = n % kStages;
+    if (*(volatile int*)&s_abort || !mbar_wait(full + s, (n / kStages) & 1)) {
+      // A wait that ran out: there is no flag word to report through without allocating, so
+      // poison this CTA's partial; the caller sees NaN in the output instead of a wrong number.
+      atomicExch(&s_abort, 1);
+#pragma unroll
+      for (int c = 0; c < kCols; ++c) acc[c] = __int_as_float(0x7fc00000);
+      break;
+    }
+    const char* st = reinterpret_cast<const char*>(stages) + (size_t)s * kStageBytes;
+    float g = 0.f, u = 0.f;
+#pragma unroll
+    for (int it = 0; it < kIter; ++it) {
+      float w[kVec];
+      E::load(st + (it * 32 + lane) * 16, w);
+#pragma unroll
+      for (int j = 0; j < kVec; ++j) g = fmaf(w[j], hreg[it * kVec + j], g);
+    }
+#pragma unroll
+    for (int it = 0; it < kIter; ++it) {
+      float w[kVec];
+      E::load(st + kRowBytes + (it * 32 + lane) * 16, w);
+#pragma unroll
+      for (int j = 0; j < kVec; ++j) u = fmaf(w[j], hreg[it * kVec + j], u);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      g += __shfl_xor_sync(kFull, g, o);
+      u += __shfl_xor_sync(kFull, u, o);
+    }
+    const float av = g / (1.f + __expf(-g)) * u * scale;
+#pragma unroll
+    for (int it = 0; it < kIter; ++it) {
+      float w[kVec];
+      E::load(st + 2 * kRowBytes + (it * 32 + lane) * 16, w);
+#pragma unroll
+      for (int j = 0; j < kVec; ++j) acc[it * kVec + j] = fmaf(av, w[j], acc[it * kVec + j]);
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(empty + s);
+  }
+
+  // add the eight warps' private sums in warp order and write this CTA's row of the scratch
+  float* dst = a.partial + (size_t)blockIdx.x * H;
+#pragma unroll
+  for (int it = 0; it < kIter; ++it) {
+    float* mine = red + (size_t)warp * kPassCols + lane * kVec;
+#pragma unroll
+    for (int v4 = 0; v4 < kVec / 4; ++v4)
+      *reinterpret_cast<float4*>(mine + v4 * 4) = make_float4(
+          acc[it * kVec + v4 * 4], acc[it * kVec + v4 * 4 + 1], acc[it * kVec + v4 * 4 + 2], acc[it * kVec + v4 * 4 + 3]);
+    consumer_bar();
+    if (tid < kPassCols) {
+      float t = 0.f;
+#pragma unroll
+      for (int w = 0; w < kConsumerWarps; ++w) t += red[(size_t)w * kPassCols + tid];
+      dst[it * kPassCols + tid] = t;
+    }
+    consumer_bar();
+  }
+}
+
+__global__ void __launch_bounds__(256) combine_static_kernel(const float* __restrict__ partial, int n_active, int H,
+                                                             float* __restrict__ out) {
+  const int c = blockIdx.x * 256 + threadIdx.x;
+  if (c >= H) return;
+  float t = 0.f;
+  for (int b = 0; b < n_active; ++b) t += partial[(size_t)b * H + c];
+  out[c] = t;
+}
+
+// Per-device set-up, done by the first call on that device with that device current: resolve
+// the scratch array's device address (in host code the array's name is only a stand-in for the
+// symbol, not an address a kernel could use) and raise the kernels' dynamic shared-memory limit.
+struct DeviceState {
+  bool ready = false;
+  float* scratch = nullptr;
+  int sms = 0;
+};
+DeviceState g_dev[kMaxDevices];
+std::mutex g_mu;
+
+template <int WB, int H>
+cudaError_t launch(const StaticArgs& a, int grid, cudaStream_t st) {
+  ffn_static_kernel<WB, H><<<grid, kThreads, smem_bytes<WB, H>(), st>>>(a);
+  return cudaGetLastError();
+}
+
+template <int WB, int H>
+cudaError_t configure() {
+  return cudaFuncSetAttribute(ffn_static_kernel<WB, H>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              (int)smem_bytes<WB, H>());
+}
+
+cudaError_t setup_device(int dev) {
+  DeviceState& d = g_dev[dev];
+  if (d.ready) return cudaSuccess;
+  float* p = nullptr;
+  cudaError_t e = cudaGetSymbolAddress((void**)&p, g_static_partial);
+  if (e != cudaSuccess) return e;
+  if ((e = cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+  if ((e = configure<4, 128>()) != cudaSuccess) return e;
+  if ((e = configure<4, 256>()) != cudaSuccess) return e;
+  if ((e = configure<4, 512>()) != cudaSuccess) return e;
+  if ((e = configure<4, 1024>()) != cudaSuccess) return e;
+  if ((e = configure<2, 256>()) != cudaSuccess) return e;
+  if ((e = configure<2, 512>()) != cudaSuccess) return e;
+  if ((e = configure<2, 1024>()) != cudaSuccess) return e;
+  if ((e = configure<2, 2048>()) != cudaSuccess) return e;
+  d.scratch = p;
+  d.ready = true;
+  return cudaSuccess;
+}
+
+}  // namespace
+
+extern "C" int remoe_expert_ffn_static(int32_t hidden, int32_t weight_dtype, int32_t n_experts,
+                                       const void* const* expert_blocks_dev, const int32_t* inter,
+                                       const float* scales, const float* hidden_in_dev, float* hidden_out_dev,
+                                       void* cuda_stream) {
+  if (!expert_blocks_dev || !inter || !scales || !hidden_in_dev || !hidden_out_dev || n_experts < 1)
+    return REMOE_E_ARG;
+  if (weight_dtype != REMOE_F32 && weight_dtype != REMOE_BF16) return REMOE_E_ARG;
+  if (n_experts > REMOE_STATIC_MAX_EXPERTS || hidden > REMOE_STATIC_MAX_HIDDEN) return REMOE_E_UNSUPPORTED;
+  const int wb = weight_dtype == REMOE_BF16 ? 2 : 4;
+  const bool width_ok = wb == 4 ? (hidden == 128 || hidden == 256 || hidden == 512 || hidden == 1024)
+                                : (hidden == 256 || hidden == 512 || hidden == 1024 || hidden == 2048);
+  if (!width_ok) return REMOE_E_UNSUPPORTED;
+  if ((reinterpret_cast<uintptr_t>(hidden_in_dev) | reinterpret_cast<uintptr_t>(hidden_out_dev)) & 15u)
+    return REMOE_E_ARG;
+
+  StaticArgs a{};
+  a.n_experts = n_experts;
+  a.prefix[0] = 0;
+  for (int e = 0; e < n_experts; ++e) {
+    if (!expert_blocks_dev[e] || (reinterpret_cast<uintptr_t>(expert_blocks_dev[e]) & 15u) || inter[e] < 1)
+      return REMOE_E_ARG;
+    if (inter[e] > REMOE_STATIC_MAX_INTER) return REMOE_E_UNSUPPORTED;
+    a.base[e] = static_cast<const char*>(expert_blocks_dev[e]);
+    a.scale[e] = scales[e];
+    a.prefix[e + 1] = a.prefix[e] + inter[e];
+  }
+  a.hidden_in = hidden_in_dev;
+
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return REMOE_E_CUDA;
+  if (dev < 0 || dev >= kMaxDevices) return REMOE_E_UNSUPPORTED;
+  {
+    std::lock_guard<std::mutex> lock(g_mu);
+    if (setup_device(dev) != cudaSuccess) return REMOE_E_CUDA;
+  }
+  const DeviceState& ds = g_dev[dev];
+  const int grid = ds.sms < kMaxCtas ? ds.sms : kMaxCtas;
+  const int M = a.prefix[n_experts];
+  a.rows_per_cta = (M + grid - 1) / grid;
+  a.n_active = (M + a.rows_per_cta - 1) / a.rows_per_cta;
+  a.partial = ds.scratch;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+
+  cudaError_t e = cudaErrorInvalidValue;
+  if (wb == 4) {
+    switch (hidden) {
+      case 128: e = launch<4, 128>(a, grid, st); break;
+      case 256: e = launch<4, 256>(a, grid, st); break;
+      case 512: e = launch<4, 512>(a, grid, st); break;
+      case 1024: e = launch<4, 1024>(a, grid, st); break;
+    }
+  } else {
+    switch (hidden) {
+      case 256: e = launch<2, 256>(a, grid, st); break;
+      case 512: e = launch<2, 512>(a, grid, st); break;
+      case 1024: e = launch<2, 1024>(a, grid, st); break;
+      case 2048: e = launch<2, 2048>(a, grid, st); break;
+    }
+  }
+  if (e != cudaSuccess) return REMOE_E_CUDA;
+  combine_static_kernel<<<(hidden + 255) / 256, 256, 0, st>>>(ds.scratch, a.n_active, hidden, hidden_out_dev);
+  return cudaGetLastError() == cudaSuccess ? REMOE_OK : REMOE_E_CUDA;
+}
