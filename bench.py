@@ -255,6 +255,9 @@ def run_ours(args, rank, world, local_rank):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     cfg = synth.config(WORKLOAD)
     shape, C, seed = cfg["shape"], cfg["cache_slots"], cfg["seed"]
+    if args.layers:
+        # a shallower stack of the same layer shape: for profiler captures, not a bench line
+        shape = synth.Shape(**{**shape.asdict(), "n_layers": args.layers})
     S_e = synth.expert_block_bytes(shape)
     peak_hbm, peak_kind = measured_peaks()
 
@@ -402,6 +405,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=16)
     ap.add_argument("--rho", type=float, default=0.9)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--layers", type=int, default=0, help="use only this many layers (profiling captures)")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-resident", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
