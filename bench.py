@@ -223,25 +223,28 @@ def run_rho(torch, wl, stream, shape, seed, rho, steps, warmup, with_e2e, prewar
     return res
 
 
-def measure_h2d(torch, nbytes, reps=10):
-    """Pinned host -> device copy rate for expert-sized blocks (GB/s, best of `reps`)."""
+def measure_h2d(torch, nbytes, reps=8):
+    """Pinned host -> device copy rate (GB/s): the better of a train of expert-sized copies and
+    one large copy, best of `reps`, CUDA events on the copying stream."""
     n_copies = 32
     h = torch.empty(n_copies * nbytes, dtype=torch.uint8).pin_memory()
     h.fill_(1)
-    d = torch.empty(2 * nbytes, dtype=torch.uint8, device="cuda")
+    d = torch.empty(n_copies * nbytes, dtype=torch.uint8, device="cuda")
     st = torch.cuda.Stream()
-    best = float("inf")
+    best = 0.0
     with torch.cuda.stream(st):
-        for _ in range(reps):
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            torch.cuda.synchronize()
-            a.record(st)
-            for i in range(n_copies):
-                d[(i % 2) * nbytes:(i % 2 + 1) * nbytes].copy_(h[i * nbytes:(i + 1) * nbytes], non_blocking=True)
-            b.record(st)
-            torch.cuda.synchronize()
-            best = min(best, a.elapsed_time(b) / n_copies)
-    return nbytes / best / 1e6
+        for rep in range(reps):
+            for pieces in (n_copies, 1):
+                chunk = n_copies * nbytes // pieces
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                torch.cuda.synchronize()
+                a.record(st)
+                for i in range(pieces):
+                    d[i * chunk:(i + 1) * chunk].copy_(h[i * chunk:(i + 1) * chunk], non_blocking=True)
+                b.record(st)
+                torch.cuda.synchronize()
+                best = max(best, n_copies * nbytes / a.elapsed_time(b) / 1e6)
+    return best
 
 
 def run_ours(args, rank, world, local_rank):

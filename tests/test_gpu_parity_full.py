@@ -1,0 +1,65 @@
+"""GPU parity at the full shapes of the batch-1 workloads, in the launch configuration bench.py times.
+
+Integer results (ids, cache trace, slots, counters, reuse) are compared with the oracle at every
+step; floating-point outputs at sampled (step, layer) pairs, which the oracle computes one by one.
+The DeepSeek-V2-Lite-shaped stack uses its full host store; the two larger stacks keep their full
+shape (layers, experts, router, cache) but let expert ids share 16 distinct weight blocks per layer
+(both sides read the same aliased blocks), which bounds host memory and set-up time.
+"""
+import numpy as np
+import pytest
+
+import synth
+
+pytestmark = pytest.mark.gpu
+
+
+def _full(name, rho, steps, distinct=None, sample_layers=(0, -1)):
+    import torch
+    from paper_2605_27081_b200.loader import LoadedWorkload
+    from parity_util import StepChecker, oracle_for
+
+    cfg = synth.config(name)
+    shape = cfg["shape"]
+    stream = torch.cuda.Stream()
+    wl = LoadedWorkload(shape, cfg["cache_slots"], cfg["seed"], stream=stream.cuda_stream, distinct_experts=distinct)
+    try:
+        rhos = rho if isinstance(rho, (list, tuple)) else [rho]
+        out = {}
+        for r, n in zip(rhos, steps if isinstance(steps, (list, tuple)) else [steps] * len(rhos)):
+            wl.stack.cache_reset()
+            chk = StepChecker(wl, oracle_for(wl), torch)
+            hs = synth.HiddenStream(cfg["seed"], shape, r)
+            sampled = {0, 1, n // 2, n - 1}
+            layers = [l % shape.n_layers for l in sample_layers]
+            with torch.cuda.stream(stream):
+                for t in range(n):
+                    h = hs.step()
+                    if t in sampled:
+                        chk.step(h, ffn="selected", ffn_layers=layers, host_api=(t == 1))
+                    else:
+                        chk.step(h, ffn=None)
+            chk.check_counters()
+            st = wl.stack.cache_stats()
+            assert st["uniq_hits"] + st["uniq_misses"] == shape.n_layers * shape.top_k * n
+            assert abs(st["uniq_hits"] / (st["uniq_hits"] + st["uniq_misses"]) - chk.o.uhr()) == 0.0
+            out[r] = (chk.near_ties, chk.max_out_err, chk.o.uhr(), chk.o.eor())
+        return out
+    finally:
+        wl.close()
+
+
+def test_dsv2lite_full_store_all_rhos():
+    res = _full("dsv2lite", [0.9, 0.5, 0.0], [512, 160, 160])
+    print("dsv2lite (near ties, max out err, uHR, EOR):", res)
+    assert res[0.9][2] > res[0.5][2] > res[0.0][2]          # more temporal correlation, more hits
+
+
+def test_qwen15moe_full_shape():
+    res = _full("qwen15moe", 0.8, 256, distinct=16)
+    print("qwen15moe:", res)
+
+
+def test_qwen3_30b_full_shape():
+    res = _full("qwen3_30b", [0.5, 0.9], [192, 192], distinct=16)
+    print("qwen3_30b:", res)
