@@ -44,6 +44,14 @@ struct remoe_stack {
   int* contrib = nullptr;
   cudaEvent_t ev_trace = nullptr;
   std::vector<cudaEvent_t> ev_layer;
+  // batched path (B > 1)
+  float* part = nullptr;
+  int* flags = nullptr;
+  int* plan = nullptr;
+  int max_items = 0;
+  int step_serial = 0;                    // never reset: stamps partial rows
+  cudaEvent_t ev_resident = nullptr;
+  std::vector<cudaEvent_t> ev_pool;        // copy-done / compute-done events of the waves
   uint64_t steps = 0, steps_since_reset = 0;
   std::vector<uint64_t> h2d_bytes;         // per layer
   // staging for the host-buffer entry point
@@ -170,6 +178,126 @@ int check_device_flag(remoe_stack* s) {
   return s->host_block[0] != kErrNone ? REMOE_E_DEVICE_FLAG : REMOE_OK;
 }
 
+// One decode step for B > 1.  The step's distinct requests may outnumber the slots, so a slot
+// can be handed on within the step: its occupants are processed in "depth" order.  Depth-0
+// experts are the cache hits (computed at once together with the shared experts) and the misses
+// that displace experts nobody asked for in this step; a depth-d miss displaces a depth-(d-1)
+// expert of this step and may only be copied once that one has been computed.  Copies are queued
+// depth by depth, layer by layer, so the copy engine stays busy; each (depth, layer) group is
+// computed as soon as its copies have landed.
+int decode_step_batched(remoe_stack* s, const float* hin, float* hout, int32_t* ids, float* gates) {
+  DevStack& d = s->d;
+  d.has_prev = s->steps_since_reset > 0 ? 1 : 0;
+  d.policy = s->policy;
+  d.beta = s->beta;
+  const int BK = s->BK;
+
+  CK(launch_route(d, hin, ids, gates, s->contrib, s->stream));
+  s->kernel_launches += 2;
+  CK(cudaMemcpyAsync(s->host_block, s->dev_block, s->block_ints * sizeof(int), cudaMemcpyDeviceToHost, s->stream));
+  CK(cudaEventRecord(s->ev_trace, s->stream));
+
+  BatchArgs a{};
+  a.d = d;
+  a.hidden_in = hin;
+  a.gates = gates;
+  a.part = s->part;
+  a.flags = s->flags;
+  a.plan = s->plan;
+  a.max_items = s->max_items;
+  a.step_id = ++s->step_serial;
+  a.phase = 0;
+  a.layer = -1;
+  a.depth = 0;
+  int rc = prof_begin(s, s->stream, 0, 0);
+  if (rc != REMOE_OK) return rc;
+  CK(launch_ffn_batched(a, s->grid, s->stream));
+  s->kernel_launches += 2;
+  rc = prof_end(s, s->stream);
+  if (rc != REMOE_OK) return rc;
+  const size_t prof_slot = s->profiling ? s->ev_used.size() - 1 : 0;
+  CK(cudaEventRecord(s->ev_resident, s->stream));
+
+  CK(cudaEventSynchronize(s->ev_trace));
+  s->steps += 1;
+  s->steps_since_reset += 1;
+  if (check_device_flag(s) != REMOE_OK) return REMOE_E_DEVICE_FLAG;
+
+  int* tr = s->host_block + 1;
+  const int* t_nu = trace_n_unique(tr);
+  const int* t_req = trace_requests(tr, d.L, BK);
+  const int* t_hit = trace_hit(tr, d.L, BK);
+  const int* t_slot = trace_slot(tr, d.L, BK);
+  const int* t_depth = trace_depth(tr, d.L, BK);
+  int max_depth = -1;
+  uint64_t resident_bytes = 0;
+  for (int l = 0; l < d.L; ++l) {
+    if (t_nu[l] < 0 || t_nu[l] > BK) return REMOE_E_DEVICE_FLAG;
+    for (int i = 0; i < t_nu[l]; ++i) {
+      const int j = l * BK + i;
+      if (t_hit[j]) { resident_bytes += d.slot_bytes; continue; }
+      if (t_req[j] < 0 || t_req[j] >= d.N || t_slot[j] < 0 || t_slot[j] >= d.C || t_depth[j] < 0)
+        return REMOE_E_DEVICE_FLAG;
+      if (t_depth[j] > max_depth) max_depth = t_depth[j];
+    }
+    resident_bytes += (uint64_t)d.S * d.shared_bytes * ((d.B + kTokTile - 1) / kTokTile);
+  }
+  if (s->profiling) s->ev_used[prof_slot].bytes = resident_bytes;
+
+  // events: [depth][layer] copy-done and compute-done
+  const size_t need = (size_t)2 * (max_depth + 1) * d.L;
+  while (s->ev_pool.size() < need) {
+    cudaEvent_t e;
+    CK(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+    s->ev_pool.push_back(e);
+  }
+  auto ev_copy = [&](int dep, int l) { return s->ev_pool[((size_t)dep * d.L + l) * 2]; };
+  auto ev_comp = [&](int dep, int l) { return s->ev_pool[((size_t)dep * d.L + l) * 2 + 1]; };
+  std::vector<char> had(((size_t)max_depth + 2) * d.L, 0);
+
+  if (max_depth >= 0) CK(cudaStreamWaitEvent(s->copy_stream, s->ev_trace, 0));
+  for (int dep = 0; dep <= max_depth; ++dep) {
+    if (dep == 1) CK(cudaStreamWaitEvent(s->copy_stream, s->ev_resident, 0));   // displaced hits are done
+    for (int l = 0; l < d.L; ++l) {
+      int misses = 0;
+      for (int i = 0; i < t_nu[l]; ++i) {
+        const int j = l * BK + i;
+        if (t_hit[j] || t_depth[j] != dep) continue;
+        if (!misses && dep >= 1 && had[(size_t)(dep - 1) * d.L + l])
+          CK(cudaStreamWaitEvent(s->copy_stream, ev_comp(dep - 1, l), 0));        // displaced misses are done
+        CK(cudaMemcpyAsync(d.slots + ((size_t)l * d.C + t_slot[j]) * d.slot_bytes,
+                           s->host_ptrs[(size_t)l * d.N + t_req[j]], d.slot_bytes, cudaMemcpyHostToDevice,
+                           s->copy_stream));
+        ++misses;
+      }
+      if (!misses) continue;
+      had[(size_t)dep * d.L + l] = 1;
+      s->h2d_bytes[l] += (uint64_t)misses * d.slot_bytes;
+      CK(cudaEventRecord(ev_copy(dep, l), s->copy_stream));
+    }
+    for (int l = 0; l < d.L; ++l) {
+      if (!had[(size_t)dep * d.L + l]) continue;
+      CK(cudaStreamWaitEvent(s->stream, ev_copy(dep, l), 0));
+      a.phase = 1;
+      a.layer = l;
+      a.depth = dep;
+      uint64_t bytes = 0;
+      for (int i = 0; i < t_nu[l]; ++i)
+        if (!t_hit[l * BK + i] && t_depth[l * BK + i] == dep) bytes += d.slot_bytes;
+      rc = prof_begin(s, s->stream, bytes, 1);
+      if (rc != REMOE_OK) return rc;
+      CK(launch_ffn_batched(a, s->grid, s->stream));
+      s->kernel_launches += 2;
+      rc = prof_end(s, s->stream);
+      if (rc != REMOE_OK) return rc;
+      CK(cudaEventRecord(ev_comp(dep, l), s->stream));
+    }
+  }
+  CK(launch_combine_batched(a, hout, s->stream));
+  s->kernel_launches += 1;
+  return REMOE_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -202,6 +330,8 @@ void remoe_stack_destroy(remoe_stack* s) {
   for (EvPair& p : s->ev_used) { cudaEventDestroy(p.a); cudaEventDestroy(p.b); }
   for (EvPair& p : s->ev_free) { cudaEventDestroy(p.a); cudaEventDestroy(p.b); }
   if (s->ev_trace) cudaEventDestroy(s->ev_trace);
+  if (s->ev_resident) cudaEventDestroy(s->ev_resident);
+  for (cudaEvent_t e : s->ev_pool) cudaEventDestroy(e);
   for (cudaEvent_t e : s->ev_layer) cudaEventDestroy(e);
   for (void* p : s->dev_allocs) cudaFree(p);
   for (void* p : s->host_allocs) cudaFreeHost(p);
@@ -219,8 +349,9 @@ int remoe_stack_create(const remoe_shape* sh, int32_t cache_slots, void* cuda_st
   const int wbytes = sh->weight_dtype == REMOE_BF16 ? 2 : 4;
   const long pairs = (long)sh->n_layers * (sh->top_k + sh->n_shared);
   if (sh->n_routed > kMaxRouted || sh->top_k > 32 || cache_slots > kMaxSlots || cache_slots > sh->n_routed ||
-      (long)sh->batch * sh->top_k > kMaxRequests || pairs > kMaxPairs || !ffn_stream_supported(sh->hidden, wbytes))
+      (long)sh->batch * sh->top_k > kMaxRequests || !ffn_stream_supported(sh->hidden, wbytes))
     return REMOE_E_UNSUPPORTED;
+  if (sh->batch == 1 && pairs > kMaxPairs) return REMOE_E_UNSUPPORTED;
 
   remoe_stack* s = new (std::nothrow) remoe_stack();
   if (!s) return REMOE_E_NOMEM;
@@ -276,6 +407,19 @@ int remoe_stack_create(const remoe_shape* sh, int32_t cache_slots, void* cuda_st
   d.trace = s->dev_block + 1;
   TRY(dev_alloc(s, &s->partial, (size_t)2 * L * s->grid * d.H));
   TRY(dev_alloc(s, &s->contrib, (size_t)2 * L * 2));
+  if (d.B > 1) {
+    if (!ffn_batched_supported(d)) return bail(REMOE_E_UNSUPPORTED);
+    const size_t P = d.K + d.S;
+    TRY(dev_alloc(s, &d.grp_count, L * s->BK));
+    TRY(dev_alloc(s, &d.grp_tok, L * s->BK * d.B));
+    TRY(dev_alloc(s, &d.grp_k, L * s->BK * d.B));
+    TRY(dev_alloc(s, &s->part, L * d.B * P * kUnitsPerItem * d.H));
+    TRY(dev_alloc(s, &s->flags, L * d.B * P * kUnitsPerItem));
+    s->max_items = (int)(L * (s->BK + (size_t)d.S * ((d.B + kTokTile - 1) / kTokTile))) + 1;
+    TRY(dev_alloc(s, &s->plan, (size_t)8 + 4 * (size_t)s->max_items));
+    if (cudaMemset(s->flags, 0, L * d.B * P * kUnitsPerItem * sizeof(int)) != cudaSuccess) return bail(REMOE_E_CUDA);
+    if (cudaEventCreateWithFlags(&s->ev_resident, cudaEventDisableTiming) != cudaSuccess) return bail(REMOE_E_CUDA);
+  }
   const size_t io = L * d.B * d.H, kk = L * (size_t)s->BK;
   TRY(dev_alloc(s, &s->st_in_d, io));
   TRY(dev_alloc(s, &s->st_out_d, io));
@@ -341,7 +485,7 @@ int remoe_decode_step(remoe_stack* s, const float* hin, float* hout, int32_t* id
   if (!s || !hin || !hout || !ids || !gates) return REMOE_E_ARG;
   if ((reinterpret_cast<uintptr_t>(hin) | reinterpret_cast<uintptr_t>(hout)) & 15u) return REMOE_E_ARG;
   if (!everything_loaded(s)) return REMOE_E_NOT_LOADED;
-  if (s->d.B != 1) return REMOE_E_UNSUPPORTED;
+  if (s->d.B != 1) return decode_step_batched(s, hin, hout, ids, gates);
   DevStack& d = s->d;
   d.has_prev = s->steps_since_reset > 0 ? 1 : 0;
   d.policy = s->policy;

@@ -1,0 +1,521 @@
+// Batched expert step (B > 1): tensor-core grouped GEMM over per-expert token groups, sm_100a.
+//
+// Tokens are grouped per requested expert (App. E.2.3: the step's distinct requests U); a work
+// item is (layer, expert, tile of up to 8 of its tokens).  For an item the expert's channel-major
+// block is streamed once, eight channels (24 rows) per stage, by bulk async copies into a
+// two-stage shared-memory ring (rows padded by 16 bytes so that ldmatrix is conflict free).
+// Eight consumer warps share every stage; warp w owns columns [256w/8.., ) of H -- the same slice
+// for both contractions:
+//   1. [W_gate rows; W_up rows] (16 x H_slice, A operand by ldmatrix) times X (H_slice x 8 tokens,
+//      B operand held in registers as bf16) -> partial gate/up pre-activations, mma m16n8k16;
+//      the eight K-slices are added through shared memory (double buffered, one barrier/stage);
+//   2. a = silu(g) * u * gate weight, rounded to bf16, is the B operand (8 channels x 8 tokens)
+//      of W_down^T (H_slice x 8 channels, A operand by ldmatrix.trans) -> mma m16n8k8 into fp32
+//      accumulators out[H_slice x 8 tokens] kept in registers for the whole item.
+// Items are laid end to end in units (1/16 of an item's channels); each CTA takes an equal
+// contiguous range of units and writes one partial row per (token, expert) and piece, stamped
+// with the step number; a combine kernel adds a token's stamped rows in a fixed order.  No float
+// atomics; every wait is bounded.
+#include "remoe_internal.cuh"
+
+namespace remoe {
+
+namespace {
+
+constexpr int kConsumerWarps = 8;
+constexpr int kThreads = (kConsumerWarps + 1) * 32;
+constexpr int kStages = 2;
+constexpr int kBlockCh = 8;                           // channels per stage
+constexpr unsigned kSpinLimit = 1u << 20;
+constexpr unsigned kFull = 0xffffffffu;
+constexpr int kPlanHeader = 8;                        // ints: n_items, n_units, ...
+constexpr int kBarBytes = 128;                        // barrier area at the start of shared memory
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+  for (unsigned it = 0; it < kSpinLimit; ++it) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    if (ok) return true;
+  }
+  return false;
+}
+__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+          smem_u32(dst)),
+      "l"(__cvta_generic_to_global(src)), "r"(bytes), "r"(smem_u32(bar))
+      : "memory");
+}
+// Barrier over the 256 consumer threads that also ORs a flag: every thread learns whether any
+// of them failed, so that they leave a loop containing barriers together.
+__device__ __forceinline__ bool consumer_bar_any(bool flag) {
+  uint32_t out;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.u32 q, %1, 0;\n\t"
+      "bar.red.or.pred p, 1, 256, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(out)
+      : "r"((uint32_t)flag)
+      : "memory");
+  return out != 0;
+}
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2,
+                                                  uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(addr));
+}
+__device__ __forceinline__ void mma_k16(float* c, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                        uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void mma_k8(float* c, uint32_t a0, uint32_t a1, uint32_t b0) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k8.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(b0));
+}
+// two floats -> packed bf16 pair (lo in the low half), round to nearest even
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+
+// ---------------------------------------------------------------------------------- plan
+// Item list of one launch, in a fixed order: layer ascending; within a layer the distinct
+// requests in request order (those matching the launch's filter), each cut into token tiles;
+// then, in the resident phase, the shared experts, each cut into token tiles.
+// plan[0] = n_items, plan[1] = n_units; item j at plan[8 + 4j]: {layer, candidate, tile, unit0}
+// where candidate < B*K is a distinct-request index and candidate >= B*K a shared expert.
+__device__ __forceinline__ int cand_tiles(const BatchArgs& a, int l, int c) {
+  const DevStack& d = a.d;
+  const int BK = d.B * d.K;
+  if (a.phase != 0 && l != a.layer) return 0;
+  if (c >= BK) return a.phase == 0 ? (d.B + kTokTile - 1) / kTokTile : 0;
+  if (c >= trace_n_unique(d.trace)[l]) return 0;
+  const int hit = trace_hit(d.trace, d.L, BK)[l * BK + c];
+  if (a.phase == 0) {
+    if (!hit) return 0;
+  } else {
+    if (hit || trace_depth(d.trace, d.L, BK)[l * BK + c] != a.depth) return 0;
+  }
+  return (d.grp_count[l * BK + c] + kTokTile - 1) / kTokTile;
+}
+
+__device__ __forceinline__ int item_units(const DevStack& d, bool shared) {
+  const int blocks = (shared ? d.Is : d.I) / kBlockCh;
+  const int per_unit = (blocks + kUnitsPerItem - 1) / kUnitsPerItem;
+  return (blocks + per_unit - 1) / per_unit;
+}
+
+__global__ void __launch_bounds__(1024) plan_kernel(BatchArgs a) {
+  __shared__ int warp_tot[32];
+  __shared__ int s_carry;
+  const DevStack& d = a.d;
+  const int BK = d.B * d.K, P = BK + d.S;
+  const int n_cand = d.L * P;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) s_carry = 0;
+  __syncthreads();
+  for (int base = 0; base < n_cand; base += 1024) {
+    const int c = base + tid;
+    const int l = c / P, cc = c % P;
+    const int tiles = c < n_cand ? cand_tiles(a, l, cc) : 0;
+    int v = tiles;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int t = __shfl_up_sync(kFull, v, o);
+      if (lane >= o) v += t;
+    }
+    if (lane == 31) warp_tot[warp] = v;
+    __syncthreads();
+    if (warp == 0) {
+      int w = warp_tot[lane];
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(kFull, w, o);
+        if (lane >= o) w += t;
+      }
+      warp_tot[lane] = w;
+    }
+    __syncthreads();
+    const int first = s_carry + (warp ? warp_tot[warp - 1] : 0) + v - tiles;   // index of my first item
+    const int u_r = item_units(d, false), u_s = d.S ? item_units(d, true) : 0;
+    for (int t = 0; t < tiles; ++t) {
+      const int j = first + t;
+      if (j < a.max_items) {
+        int* it = a.plan + kPlanHeader + 4 * j;
+        it[0] = l; it[1] = cc; it[2] = t; it[3] = cc >= BK ? u_s : u_r;            // unit count for now
+      }
+    }
+    __syncthreads();
+    if (tid == 1023) s_carry = first + tiles;
+    __syncthreads();
+  }
+  // Second pass: exclusive prefix of unit counts (items are few thousand at most).
+  const int n_items = min(s_carry, a.max_items);
+  __syncthreads();
+  if (tid == 0) s_carry = 0;
+  __syncthreads();
+  for (int base = 0; base < n_items; base += 1024) {
+    const int j = base + tid;
+    const int units = j < n_items ? a.plan[kPlanHeader + 4 * j + 3] : 0;
+    int v = units;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int t = __shfl_up_sync(kFull, v, o);
+      if (lane >= o) v += t;
+    }
+    if (lane == 31) warp_tot[warp] = v;
+    __syncthreads();
+    if (warp == 0) {
+      int w = warp_tot[lane];
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(kFull, w, o);
+        if (lane >= o) w += t;
+      }
+      warp_tot[lane] = w;
+    }
+    __syncthreads();
+    const int excl = s_carry + (warp ? warp_tot[warp - 1] : 0) + v - units;
+    if (j < n_items) a.plan[kPlanHeader + 4 * j + 3] = excl;
+    __syncthreads();
+    if (tid == 1023) s_carry = excl + units;
+    __syncthreads();
+  }
+  if (tid == 0) {
+    a.plan[0] = n_items;
+    a.plan[1] = s_carry;
+    if (s_carry < 0 || n_items >= a.max_items) atomicCAS(d.err, kErrNone, kErrBadIndex);
+  }
+}
+
+// ------------------------------------------------------------------------------- kernel
+
+template <int H>
+struct Geo {
+  static constexpr int kRowStride = H * 2 + 16;                        // padded bf16 row
+  static constexpr int kStageBytes = 3 * kBlockCh * kRowStride;
+  static constexpr uint32_t kTxBytes = 3u * kBlockCh * H * 2;
+  static constexpr int kSlice = H / kConsumerWarps;                    // columns of H per warp
+  static constexpr int kKSteps = kSlice / 16;
+  static constexpr int kMTiles = kSlice / 16;
+  static constexpr size_t kRedBytes = 2 * kConsumerWarps * 16 * 8 * sizeof(float);
+  static constexpr size_t kSmem = kBarBytes + kRedBytes + (size_t)kStages * kStageBytes;
+};
+
+struct PieceInfo {
+  const char* base;       // expert block
+  int l, cand, tile, n_tok;
+  int blk0, blk1;         // channel-block range [blk0, blk1) of this piece
+  int first_unit;
+  bool shared;
+};
+
+// Decode the piece of item `j` that falls inside units [ua, ub).
+__device__ __forceinline__ bool make_piece(const BatchArgs& a, int j, int ua, int ub, PieceInfo& p) {
+  const DevStack& d = a.d;
+  const int BK = d.B * d.K;
+  const int* it = a.plan + kPlanHeader + 4 * j;
+  p.l = it[0]; p.cand = it[1]; p.tile = it[2];
+  const int unit0 = it[3];
+  p.shared = p.cand >= BK;
+  const int blocks = (p.shared ? d.Is : d.I) / kBlockCh;
+  const int per_unit = (blocks + kUnitsPerItem - 1) / kUnitsPerItem;
+  const int units = (blocks + per_unit - 1) / per_unit;
+  const int lo = max(ua, unit0) - unit0, hi = min(ub, unit0 + units) - unit0;
+  if (lo >= hi) return false;
+  p.first_unit = lo;
+  p.blk0 = lo * per_unit;
+  p.blk1 = min(blocks, hi * per_unit);
+  if (p.shared) {
+    p.base = d.shared_blocks + ((size_t)p.l * d.S + (p.cand - BK)) * d.shared_bytes;
+    p.n_tok = min(kTokTile, d.B - p.tile * kTokTile);
+  } else {
+    const int slot = trace_slot(d.trace, d.L, BK)[p.l * BK + p.cand];
+    if (slot < 0 || slot >= d.C) { atomicCAS(d.err, kErrNone, kErrBadIndex); return false; }
+    p.base = d.slots + ((size_t)p.l * d.C + slot) * d.slot_bytes;
+    p.n_tok = min(kTokTile, d.grp_count[p.l * BK + p.cand] - p.tile * kTokTile);
+  }
+  return true;
+}
+
+template <int H>
+__global__ void __launch_bounds__(kThreads, 1) ffn_batched_kernel(const __grid_constant__ BatchArgs a) {
+  using G = Geo<H>;
+  extern __shared__ __align__(128) unsigned char smem[];
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem);
+  uint64_t* empty = full + kStages;
+  float* red = reinterpret_cast<float*>(smem + kBarBytes);
+  unsigned char* stages = reinterpret_cast<unsigned char*>(red) + G::kRedBytes;
+  __shared__ int s_abort;
+
+  const DevStack& d = a.d;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int BK = d.B * d.K, P = d.K + d.S;
+  if (tid == 0) {
+    s_abort = 0;
+    for (int s = 0; s < kStages; ++s) { mbar_init(full + s, 1); mbar_init(empty + s, kConsumerWarps); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  const int n_items = a.plan[0], n_units = a.plan[1];
+  const int q = (n_units + gridDim.x - 1) / (int)gridDim.x;
+  const int ua = min(n_units, (int)blockIdx.x * q), ub = min(n_units, ua + q);
+  if (ua >= ub) return;
+  // first item whose unit range reaches past ua
+  int j0 = 0;
+  {
+    int lo = 0, hi = n_items - 1;
+    while (lo < hi) {
+      const int mid = (lo + hi + 1) >> 1;
+      if (a.plan[kPlanHeader + 4 * mid + 3] <= ua) lo = mid; else hi = mid - 1;
+    }
+    j0 = lo;
+  }
+
+  if (warp == kConsumerWarps) {
+    // ------------------------------------------------------------------ producer
+    if (lane == 0) {
+      int n = 0;
+      bool ok = true;
+      for (int j = j0; j < n_items && ok; ++j) {
+        if (a.plan[kPlanHeader + 4 * j + 3] >= ub) break;
+        PieceInfo p;
+        if (!make_piece(a, j, ua, ub, p)) continue;
+        for (int blk = p.blk0; blk < p.blk1; ++blk, ++n) {
+          const int s = n % kStages;
+          if (n >= kStages) {
+            if (*(volatile int*)&s_abort || !mbar_wait(empty + s, ((n / kStages) - 1) & 1)) {
+              if (!*(volatile int*)&s_abort) atomicCAS(d.err, kErrNone, kErrWaitEmpty);
+              ok = false;
+              break;
+            }
+          }
+          mbar_expect_tx(full + s, G::kTxBytes);
+          const char* src = p.base + (size_t)blk * (3 * kBlockCh * H * 2);
+          unsigned char* dst = stages + (size_t)s * G::kStageBytes;
+#pragma unroll 1
+          for (int r = 0; r < 3 * kBlockCh; ++r)
+            bulk_g2s(dst + r * G::kRowStride, src + (size_t)r * H * 2, H * 2, full + s);
+        }
+      }
+      if (!ok) {
+        atomicExch(&s_abort, 1);
+        for (int m = max(0, n - kStages); m < n; ++m)
+          if (!mbar_wait(full + (m % kStages), (m / kStages) & 1)) atomicCAS(d.err, kErrNone, kErrDrain);
+      }
+    }
+    return;
+  }
+
+  // ------------------------------------------------------------------- consumers
+  const int col0 = warp * G::kSlice;                 // this warp's slice of H
+  const int grp = lane >> 2, qd = lane & 3;          // MMA fragment coordinates
+  int n = 0, buf = 0;
+  bool aborted = false;
+  for (int j = j0; j < n_items; ++j) {
+    if (a.plan[kPlanHeader + 4 * j + 3] >= ub) break;
+    PieceInfo p;
+    if (!make_piece(a, j, ua, ub, p)) continue;
+
+    // token metadata: B-operand column `grp` is token grp of the tile; accumulator columns are
+    // tokens 2*qd and 2*qd+1.
+    const int gidx = (p.l * BK + p.cand) * d.B + p.tile * kTokTile;
+    auto tok_of = [&](int t) -> int {
+      if (t >= p.n_tok) return -1;
+      return p.shared ? p.tile * kTokTile + t : d.grp_tok[gidx + t];
+    };
+    auto kq_of = [&](int t) -> int { return p.shared ? d.K + (p.cand - BK) : d.grp_k[gidx + t]; };
+    const int my_tok = tok_of(grp);
+    float my_scale = 0.f;
+    if (my_tok >= 0)
+      my_scale = p.shared ? d.shared_scale[p.l * d.B + my_tok] : a.gates[((size_t)p.l * d.B + my_tok) * d.K + kq_of(grp)];
+
+    // X slice as B fragments: for k-step ks, b0 = X[col0+16ks+2qd .. +1][tok grp], b1 = same +8.
+    uint32_t xb[G::kKSteps][2];
+    {
+      const float* xr = my_tok >= 0 ? a.hidden_in + ((size_t)p.l * d.B + my_tok) * H + col0 : nullptr;
+#pragma unroll
+      for (int ks = 0; ks < G::kKSteps; ++ks) {
+        float2 lo = make_float2(0.f, 0.f), hi = make_float2(0.f, 0.f);
+        if (xr) {
+          lo = __ldg(reinterpret_cast<const float2*>(xr + 16 * ks + 2 * qd));
+          hi = __ldg(reinterpret_cast<const float2*>(xr + 16 * ks + 8 + 2 * qd));
+        }
+        xb[ks][0] = pack_bf16(lo.x, lo.y);
+        xb[ks][1] = pack_bf16(hi.x, hi.y);
+      }
+    }
+    float acc[G::kMTiles][4];
+#pragma unroll
+    for (int m = 0; m < G::kMTiles; ++m) { acc[m][0] = acc[m][1] = acc[m][2] = acc[m][3] = 0.f; }
+
+    for (int blk = p.blk0; blk < p.blk1 && !aborted; ++blk, ++n) {
+      const int s = n % kStages;
+      // warp-uniform, because the tensor-core instructions below need the whole warp
+      const bool fail = __any_sync(kFull, *(volatile int*)&s_abort || !mbar_wait(full + s, (n / kStages) & 1));
+      const uint32_t st = smem_u32(stages + (size_t)s * G::kStageBytes);
+      // contraction 1 over this warp's K slice: rows 0-7 = W_gate, rows 8-15 = W_up of the block
+      if (!fail) {
+        float c1[4] = {0.f, 0.f, 0.f, 0.f};
+        const int mat = lane >> 3, r = lane & 7;
+        const uint32_t row_addr = st + (3 * r + (mat & 1)) * G::kRowStride + (col0 + 8 * (mat >> 1)) * 2;
+#pragma unroll
+        for (int ks = 0; ks < G::kKSteps; ++ks) {
+          uint32_t a0, a1, a2, a3;
+          ldmatrix_x4(row_addr + ks * 32, a0, a1, a2, a3);
+          mma_k16(c1, a0, a1, a2, a3, xb[ks][0], xb[ks][1]);
+        }
+        float* rb = red + (size_t)buf * kConsumerWarps * 128 + warp * 128;
+        *reinterpret_cast<float2*>(rb + grp * 8 + 2 * qd) = make_float2(c1[0], c1[1]);
+        *reinterpret_cast<float2*>(rb + (grp + 8) * 8 + 2 * qd) = make_float2(c1[2], c1[3]);
+      }
+      if (consumer_bar_any(fail)) {
+        // some warp's wait ran out (or the producer gave up): everybody leaves together
+        if (tid == 0) { atomicCAS(d.err, kErrNone, kErrWaitFull); atomicExch(&s_abort, 1); }
+        aborted = true;
+        break;
+      }
+      // full pre-activations for channels 2qd, 2qd+1 and token grp, then the activation
+      uint32_t ab;
+      {
+        const float* r0 = red + (size_t)buf * kConsumerWarps * 128;
+        float g0 = 0.f, g1 = 0.f, u0 = 0.f, u1 = 0.f;
+#pragma unroll
+        for (int w = 0; w < kConsumerWarps; ++w) {
+          g0 += r0[w * 128 + (2 * qd) * 8 + grp];
+          g1 += r0[w * 128 + (2 * qd + 1) * 8 + grp];
+          u0 += r0[w * 128 + (8 + 2 * qd) * 8 + grp];
+          u1 += r0[w * 128 + (9 + 2 * qd) * 8 + grp];
+        }
+        const float v0 = g0 / (1.f + __expf(-g0)) * u0 * my_scale;
+        const float v1 = g1 / (1.f + __expf(-g1)) * u1 * my_scale;
+        ab = pack_bf16(v0, v1);
+      }
+      // contraction 2: out[H slice x 8 tokens] += W_down[:, block]^T (8 channels) x a
+      {
+        const int mat = lane >> 3, r = lane & 7;
+        const uint32_t row_addr = st + (3 * r + 2) * G::kRowStride + (col0 + 8 * mat) * 2;
+#pragma unroll
+        for (int mp = 0; mp < G::kMTiles / 2; ++mp) {
+          uint32_t a0, a1, a2, a3;
+          ldmatrix_x4_trans(row_addr + mp * 64, a0, a1, a2, a3);
+          mma_k8(acc[2 * mp], a0, a1, ab);
+          mma_k8(acc[2 * mp + 1], a2, a3, ab);
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(empty + s);
+      buf ^= 1;
+    }
+
+    // flush: one stamped partial row per (token, expert rank) for this piece
+    if (!aborted) {
+#pragma unroll
+      for (int tt = 0; tt < 2; ++tt) {
+        const int t = 2 * qd + tt;
+        const int tok = tok_of(t);
+        if (tok < 0) continue;
+        const size_t row = (((size_t)p.l * d.B + tok) * P + kq_of(t)) * kUnitsPerItem + p.first_unit;
+        float* dst = a.part + row * H + col0;
+#pragma unroll
+        for (int m = 0; m < G::kMTiles; ++m) {
+          dst[16 * m + grp] = acc[m][tt];
+          dst[16 * m + 8 + grp] = acc[m][2 + tt];
+        }
+        if (warp == 0 && grp == 0) a.flags[row] = a.step_id;
+      }
+    }
+  }
+}
+
+__global__ void __launch_bounds__(256) combine_batched_kernel(BatchArgs a, float* __restrict__ hidden_out) {
+  const DevStack& d = a.d;
+  const int lb = blockIdx.y;
+  const int c = blockIdx.x * 256 + threadIdx.x;
+  if (c >= d.H) return;
+  const int P = d.K + d.S;
+  float t = 0.f;
+  for (int k = 0; k < P; ++k)
+    for (int u = 0; u < kUnitsPerItem; ++u) {
+      const size_t row = ((size_t)lb * P + k) * kUnitsPerItem + u;
+      if (a.flags[row] == a.step_id) t += a.part[row * d.H + c];
+    }
+  hidden_out[(size_t)lb * d.H + c] = t;
+}
+
+template <int H>
+cudaError_t launch_one(const BatchArgs& a, int grid, cudaStream_t st) {
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(ffn_batched_kernel<H>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)Geo<H>::kSmem);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  plan_kernel<<<1, 1024, 0, st>>>(a);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  ffn_batched_kernel<H><<<grid, kThreads, Geo<H>::kSmem, st>>>(a);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+bool ffn_batched_supported(const DevStack& d) {
+  if (d.wbytes != 2) return false;
+  if (d.H != 256 && d.H != 512 && d.H != 1024 && d.H != 2048) return false;
+  if (d.I % kBlockCh || (d.S && d.Is % kBlockCh)) return false;
+  return true;
+}
+
+cudaError_t launch_ffn_batched(const BatchArgs& a, int grid, cudaStream_t st) {
+  switch (a.d.H) {
+    case 256: return launch_one<256>(a, grid, st);
+    case 512: return launch_one<512>(a, grid, st);
+    case 1024: return launch_one<1024>(a, grid, st);
+    case 2048: return launch_one<2048>(a, grid, st);
+  }
+  return cudaErrorInvalidValue;
+}
+
+cudaError_t launch_combine_batched(const BatchArgs& a, float* hidden_out, cudaStream_t st) {
+  dim3 grid((a.d.H + 255) / 256, a.d.L * a.d.B);
+  combine_batched_kernel<<<grid, 256, 0, st>>>(a, hidden_out);
+  return cudaGetLastError();
+}
+
+}  // namespace remoe

@@ -182,7 +182,8 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_static_kernel(const __grid_co
     while (a.prefix[e + 1] <= r) ++e;
     const float scale = a.scale[e];
     const int n = r - r0, s = n % kStages;
-    if (*(volatile int*)&s_abort || !mbar_wait(full + s, (n / kStages) & 1)) {
+    // decided for the whole warp: the shuffles below need every lane
+    if (__any_sync(kFull, *(volatile int*)&s_abort || !mbar_wait(full + s, (n / kStages) & 1))) {
       // A wait that ran out: there is no flag word to report through without allocating, so
       // poison this CTA's partial; the caller sees NaN in the output instead of a wrong number.
       atomicExch(&s_abort, 1);

@@ -273,7 +273,8 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(const __grid_co
           pair_of_scale = pair;
         }
         const int n = r - r0, s = n % NS;
-        if (*(volatile int*)&s_abort || !mbar_wait(full + s, (n / NS) & 1)) {
+        // decided for the whole warp: the shuffles below need every lane
+        if (__any_sync(kFull, *(volatile int*)&s_abort || !mbar_wait(full + s, (n / NS) & 1))) {
           if (!*(volatile int*)&s_abort) { atomicCAS(d.err, kErrNone, kErrWaitFull); atomicExch(&s_abort, 1); }
           aborted = true;
           break;

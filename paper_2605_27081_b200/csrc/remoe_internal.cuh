@@ -49,12 +49,19 @@ struct DevStack {
   float* shared_scale;                 // [L][B]
   int* last_overlap;                   // [L][B]   -1 when not counted
   // Step trace, one block so that a single copy brings it to the host:
-  // n_unique[L] | requests[L][B*K] | hit[L][B*K] | slot[L][B*K] | evicted[L][B*K]
+  // n_unique[L] | requests[L][B*K] | hit[L][B*K] | slot[L][B*K] | evicted[L][B*K] | depth[L][B*K]
+  // depth: how many of this step's experts occupied the request's slot before it within the
+  // step (0 unless the step asks for more distinct experts than there are slots).
   int* trace;
   int* err;
+  // Token groups per distinct request (batch > 1): which sequences selected it, at which rank.
+  int* grp_count;                      // [L][B*K]
+  int* grp_tok;                        // [L][B*K][B]
+  int* grp_k;                          // [L][B*K][B]
 };
 
-__host__ __device__ inline int trace_ints(int L, int BK) { return L + 4 * L * BK; }
+__host__ __device__ inline int trace_ints(int L, int BK) { return L + 5 * L * BK; }
+__host__ __device__ inline int* trace_depth(int* t, int L, int BK) { return t + L + 4 * L * BK; }
 __host__ __device__ inline int* trace_n_unique(int* t) { return t; }
 __host__ __device__ inline int* trace_requests(int* t, int L, int BK) { return t + L; }
 __host__ __device__ inline int* trace_hit(int* t, int L, int BK) { return t + L + L * BK; }
@@ -72,6 +79,25 @@ struct FfnArgs {
   int* contrib;                        // [2][L][2]  (first CTA, last CTA) contributing; first > last = none
   int grid_cap;                        // CTAs per phase the partial buffer is laid out for
 };
+
+// Batched (B > 1) expert kernels: tensor-core grouped GEMM over per-expert token groups.
+constexpr int kTokTile = 8;            // tokens per work item (the MMA's N)
+constexpr int kUnitsPerItem = 16;      // an item's channels are cut into this many units
+struct BatchArgs {
+  DevStack d;
+  const float* hidden_in;              // [L][B][H]
+  const float* gates;                  // [L][B][K]
+  int phase;                           // 0: cache hits + shared experts of all layers; 1: misses
+  int layer, depth;                    // phase 1: which layer, which depth
+  int step_id;                         // stamps the partial rows written in this step
+  float* part;                         // [L][B][K+S][kUnitsPerItem][H]
+  int* flags;                          // [L][B][K+S][kUnitsPerItem]
+  int* plan;                           // header (8 ints) + items (4 ints each)
+  int max_items;
+};
+bool ffn_batched_supported(const DevStack& d);
+cudaError_t launch_ffn_batched(const BatchArgs& a, int grid, cudaStream_t st);
+cudaError_t launch_combine_batched(const BatchArgs& a, float* hidden_out, cudaStream_t st);
 
 cudaError_t launch_route(const DevStack& d, const float* hidden_in, int* ids, float* gates,
                          int* contrib, cudaStream_t st);

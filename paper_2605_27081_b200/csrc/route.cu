@@ -72,6 +72,9 @@ struct DirSmem {
   int uniq[kMaxRequests];
   unsigned char hitf[kMaxRequests];
   unsigned seen[kMaskWords];
+  int uidx[kMaxRouted];                 // position of an expert in the unique list
+  int gcnt[kMaxRequests];               // tokens collected so far per unique request
+  unsigned char sgen[kMaxSlots];        // this step's occupants a slot has had so far
 };
 
 // Cache resolution for one layer by one warp.  `flat` holds the step's B*K requested ids in
@@ -80,6 +83,7 @@ __device__ void resolve_layer(const DevStack& d, int l, const int* flat, int n_f
                               int lane, int* contrib) {
   const int C = d.C, N = d.N, BK = d.B * d.K;
   for (int s = lane; s < C; s += 32) {
+    sm.sgen[s] = 0;
     sm.eos[s] = d.expert_of_slot[l * C + s];
     sm.stamp[s] = d.stamp[l * C + s];
     sm.freq[s] = d.freq[l * C + s];
@@ -114,6 +118,30 @@ __device__ void resolve_layer(const DevStack& d, int l, const int* flat, int n_f
   int* t_hit = trace_hit(d.trace, d.L, BK) + l * BK;
   int* t_slot = trace_slot(d.trace, d.L, BK) + l * BK;
   int* t_ev = trace_evicted(d.trace, d.L, BK) + l * BK;
+  int* t_depth = trace_depth(d.trace, d.L, BK) + l * BK;
+
+  if (d.B > 1) {
+    // Token groups: for every distinct request, the sequences that selected it (ascending)
+    // and the rank at which they did.
+    for (int i = lane; i < n_u; i += 32) { sm.uidx[sm.uniq[i]] = i; sm.gcnt[i] = 0; }
+    __syncwarp();
+    for (int base = 0; base < n_flat; base += 32) {
+      const int f = base + lane;
+      const bool valid = f < n_flat;
+      const int ui = valid ? sm.uidx[flat[f]] : -1 - lane;
+      const unsigned same = __match_any_sync(kFull, ui);
+      if (valid) {
+        const int pos = sm.gcnt[ui] + __popc(same & lt);
+        const size_t g = ((size_t)l * BK + ui) * d.B + pos;
+        d.grp_tok[g] = f / d.K;
+        d.grp_k[g] = f % d.K;
+      }
+      __syncwarp();
+      if (valid && (__ffs(same) - 1 == lane)) sm.gcnt[ui] += __popc(same);
+      __syncwarp();
+    }
+    for (int i = lane; i < BK; i += 32) d.grp_count[l * BK + i] = i < n_u ? sm.gcnt[i] : 0;
+  }
 
   // Classification against the pre-step state, then phase 1: touch hits in request order.
   unsigned long long clock = d.clock[l];
@@ -128,6 +156,7 @@ __device__ void resolve_layer(const DevStack& d, int l, const int* flat, int n_f
     if (hit) {
       if (d.policy != REMOE_POLICY_FIFO) sm.stamp[s] = clock + 1 + __popc(hm & lt);
       sm.freq[s] += 1u;
+      sm.sgen[s] = 1;
     }
     clock += __popc(hm);
     uniq_h += __popc(hm);
@@ -136,6 +165,7 @@ __device__ void resolve_layer(const DevStack& d, int l, const int* flat, int n_f
       t_hit[i] = valid ? (hit ? 1 : 0) : 0;
       t_slot[i] = s;
       t_ev[i] = -1;
+      t_depth[i] = 0;
       sm.hitf[i] = hit ? 1 : 0;
     }
     __syncwarp();
@@ -178,6 +208,8 @@ __device__ void resolve_layer(const DevStack& d, int l, const int* flat, int n_f
       sm.freq[best_s] = 1u;
       t_slot[i] = best_s;
       t_ev[i] = ev;
+      t_depth[i] = sm.sgen[best_s];
+      sm.sgen[best_s] += 1;
     }
     __syncwarp();
   }

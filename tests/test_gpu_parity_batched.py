@@ -1,0 +1,47 @@
+"""GPU parity of the batched step (B > 1): union of requests, shared cache, token groups,
+tensor-core grouped GEMM, against the CPU oracle on the same seeded inputs."""
+import pytest
+
+import synth
+
+pytestmark = pytest.mark.gpu
+
+
+def _run(shape, cache_slots, rho, steps, seed=0, dense_steps=1, policy=None):
+    import torch
+    from paper_2605_27081_b200.loader import LoadedWorkload
+    from parity_util import StepChecker, oracle_for
+
+    wl = LoadedWorkload(shape, cache_slots, seed)
+    try:
+        pol = "lru"
+        if policy is not None:
+            wl.stack.set_policy(policy)
+            pol = {0: "lru", 1: "fifo", 2: "lfu"}[policy]
+        chk = StepChecker(wl, oracle_for(wl, pol), torch)
+        hs = synth.HiddenStream(seed, shape, rho)
+        deepest = 0
+        for t in range(steps):
+            r, _ = chk.step(hs.step(), ffn="dense" if t < dense_steps else "selected", host_api=(t % 5 == 4))
+            deepest = max(deepest, max(len(q) for q in r["requests"]))
+        chk.check_counters()
+        return chk, deepest
+    finally:
+        wl.close()
+
+
+@pytest.mark.parametrize("shape,c,rho", [
+    (synth.Shape(2, 256, 16, 2, 64, 1, 32, 0, 0, 1, 4), 6, 0.5),         # union sometimes above capacity
+    (synth.Shape(3, 512, 24, 3, 80, 2, 40, 1, 0, 1, 12), 8, None),       # union far above capacity, sigmoid gate
+    (synth.Shape(2, 1024, 40, 4, 48, 0, 0, 0, 1, 1, 20), 40, 0.7),       # all resident, renormalised, B not a multiple of 8
+    (synth.Shape(2, 2048, 64, 6, 176, 2, 176, 0, 0, 1, 32), 32, None),   # the serving configuration's layer shape
+])
+def test_batched_shapes(shape, c, rho):
+    chk, deepest = _run(shape, c, rho, steps=12, seed=3)
+    assert chk.max_out_err <= 2e-2
+    if c < shape.n_routed and shape.batch * shape.top_k > 2 * c:
+        assert deepest > c                     # the case the capacity assumption excludes did occur
+
+
+def test_batched_other_policy():
+    _run(synth.Shape(2, 256, 16, 2, 64, 0, 0, 0, 0, 1, 6), 5, 0.4, steps=30, seed=4, dense_steps=0, policy=2)
