@@ -112,7 +112,7 @@ def oracle_sample(shape, cache_slots, seed, rho, layers, steps, warmup=0):
     for t in range(warmup + steps):
         r = st.step(hidden[t], ffn=None)
         for l in range(layers):
-            for e in r["ids"][l, 0]:
+            for e in r["ids"][l].reshape(-1):
                 ew(l, int(e))
     st.reset()
     for t in range(warmup):
@@ -134,20 +134,20 @@ def run_reference(args, rank, world):
     scaled to the full depth."""
     if rank != 0:
         return
-    cfg = synth.config(WORKLOAD)
+    cfg = synth.config(args.workload)
     shape = cfg["shape"]
     total = args.steps + args.warmup
     layers = int(max(1, min(4, 300 // max(1, total))))
     dt, cores = oracle_sample(shape, cfg["cache_slots"], cfg["seed"], args.rho, layers, args.steps, args.warmup)
     per_step = dt / args.steps * shape.n_layers / layers
-    value = 1.0 / per_step
+    value = shape.batch / per_step
     sample = (f"{args.steps} decode steps over the first {layers} of {shape.n_layers} layers, time scaled by "
               f"{shape.n_layers}/{layers}; selected-experts-only fp64 oracle")
     line = {
         "impl": "reference", "metric": "decode tokens/s (batch 1, MoE stack)", "value": value, "unit": "tokens/s",
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_step * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "rho": args.rho, "cache_slots": cfg["cache_slots"], "batch": 1},
+        "config": {"workload": args.workload, "rho": args.rho, "cache_slots": cfg["cache_slots"], "batch": shape.batch},
         "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
@@ -169,14 +169,14 @@ def timed_steps(torch, wl, stream, d_hidden, d_out, d_ids, d_g, first, count):
 
 def run_rho(torch, wl, stream, shape, seed, rho, steps, warmup, with_e2e, prewarm_iid=0):
     """Cold cache -> warm-up -> K timed steps (device inputs) [-> K timed steps through host buffers]."""
-    L, H, K = shape.n_layers, shape.hidden, shape.top_k
+    L, H, K, B = shape.n_layers, shape.hidden, shape.top_k, shape.batch
     n = warmup + steps * (2 if with_e2e else 1)
     hidden = synth.HiddenStream(seed, shape, rho).take(n)
     h_pinned = torch.from_numpy(hidden).pin_memory()
     d_hidden = h_pinned.to("cuda", non_blocking=False)
-    d_out = torch.empty((L, 1, H), dtype=torch.float32, device="cuda")
-    d_ids = torch.empty((L, 1, K), dtype=torch.int32, device="cuda")
-    d_g = torch.empty((L, 1, K), dtype=torch.float32, device="cuda")
+    d_out = torch.empty((L, B, H), dtype=torch.float32, device="cuda")
+    d_ids = torch.empty((L, B, K), dtype=torch.int32, device="cuda")
+    d_g = torch.empty((L, B, K), dtype=torch.float32, device="cuda")
     st = wl.stack
     st.cache_reset()
     st.set_profiling(False)
@@ -204,9 +204,9 @@ def run_rho(torch, wl, stream, shape, seed, rho, steps, warmup, with_e2e, prewar
         "kernel_resident": k_res, "kernel_miss": k_miss,
     }
     if with_e2e:
-        out_h = torch.empty((L, 1, H), dtype=torch.float32).pin_memory().numpy()
-        ids_h = torch.empty((L, 1, K), dtype=torch.int32).pin_memory().numpy()
-        g_h = torch.empty((L, 1, K), dtype=torch.float32).pin_memory().numpy()
+        out_h = torch.empty((L, B, H), dtype=torch.float32).pin_memory().numpy()
+        ids_h = torch.empty((L, B, K), dtype=torch.int32).pin_memory().numpy()
+        g_h = torch.empty((L, B, K), dtype=torch.float32).pin_memory().numpy()
         hp = h_pinned.numpy()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.synchronize()
@@ -256,8 +256,10 @@ def run_ours(args, rank, world, local_rank):
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
-    cfg = synth.config(WORKLOAD)
+    cfg = synth.config(args.workload)
     shape, C, seed = cfg["shape"], cfg["cache_slots"], cfg["seed"]
+    if args.rho is None:
+        args.rho = cfg["rhos"][0] if args.workload != "dsv2lite" else 0.9
     if args.layers:
         # a shallower stack of the same layer shape: for profiler captures, not a bench line
         shape = synth.Shape(**{**shape.asdict(), "n_layers": args.layers})
@@ -319,7 +321,7 @@ def run_ours(args, rank, world, local_rank):
         if dist is not None:
             dist.destroy_process_group()
         return
-    tokens = args.steps * world
+    tokens = args.steps * world * shape.batch
     value = tokens / (ms / 1e3)
     per_step_ms = ms / args.steps
 
@@ -339,7 +341,7 @@ def run_ours(args, rank, world, local_rank):
     km_ms, km_n, km_b = head["kernel_miss"]
     ach = kr_b / (kr_ms / 1e3) / 1e9 if kr_ms > 0 else 0.0
     roofline = {"bound": "hbm", "achieved": ach, "peak": peak_hbm, "unit": "GB/s", "frac": ach / peak_hbm,
-                "traffic": None, "peak_kind": f"of {peak_kind}", "kernel": "ffn_stream_kernel<bf16,2048> resident phase",
+                "traffic": None, "peak_kind": f"of {peak_kind}", "kernel": ("ffn_stream_kernel<bf16,2048>" if shape.batch == 1 else "ffn_batched_kernel<2048>") + " resident phase",
                 "launches": kr_n, "avg_launch_ms": kr_ms / max(1, kr_n), "bytes_per_launch": kr_b / max(1, kr_n),
                 "frac_of_nominal_8TBs": ach / NOMINAL_HBM_GBS}
     miss_phase = {"launches": km_n, "avg_launch_us": km_ms * 1e3 / max(1, km_n),
@@ -351,14 +353,14 @@ def run_ours(args, rank, world, local_rank):
         layers, steps_cpu = 2, 3
         dt, cores = oracle_sample(shape, C, seed, args.rho, layers, steps_cpu)
         per = dt / steps_cpu * shape.n_layers / layers
-        cpu = {"value": 1.0 / per, "unit": "tokens/s", "cores": cores, "kind": "oracle",
+        cpu = {"value": shape.batch / per, "unit": "tokens/s", "cores": cores, "kind": "oracle",
                "sample": f"first {steps_cpu} decode steps (cold cache) over the first {layers} of {shape.n_layers} "
                          f"layers, time scaled by {shape.n_layers}/{layers}; selected-experts-only fp64 oracle"}
 
     sweep = {}
     for rho, r in results.items():
         sweep[str(rho)] = {
-            "tokens_per_s": args.steps / (r["ms"] / 1e3),
+            "tokens_per_s": args.steps * shape.batch / (r["ms"] / 1e3),
             "hit_rate": r["uniq_hits"] / max(1, r["uniq_hits"] + r["uniq_misses"]),
             "eor": r["overlap"] / max(1, r["pairs"] * shape.top_k),
             "misses_per_step": r["uniq_misses"] / args.steps,
@@ -367,7 +369,8 @@ def run_ours(args, rank, world, local_rank):
         "metric": "decode tokens/s (batch 1, MoE stack)", "value": value, "unit": "tokens/s",
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_step_ms,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "rho": args.rho, "cache_slots": C, "batch": 1, "layers": shape.n_layers,
+        "config": {"workload": args.workload, "rho": args.rho, "cache_slots": C, "batch": shape.batch,
+                   "layers": shape.n_layers,
                    "l2": "inputs larger than L2 (>= 1.6 GB of expert weights streamed per step)",
                    "parallelism": "replicas only" if world > 1 else "single GPU",
                    "distinct_experts_per_layer": wl.n_distinct},
@@ -390,7 +393,7 @@ def run_ours(args, rank, world, local_rank):
         n = min(args.steps, 256)
         ms_r, n_r, b_r = resident["kernel_resident"]
         line["all_resident"] = {
-            "cache_slots": shape.n_routed, "tokens_per_s": n / (resident["ms"] / 1e3),
+            "cache_slots": shape.n_routed, "tokens_per_s": n * shape.batch / (resident["ms"] / 1e3),
             "ms_per_step": resident["ms"] / n, "misses": resident["uniq_misses"],
             "kernel_gbs": b_r / (ms_r / 1e3) / 1e9 if ms_r > 0 else 0.0,
             "kernel_frac_of_measured": (b_r / (ms_r / 1e3) / 1e9 / peak_hbm) if ms_r > 0 else 0.0,
@@ -406,7 +409,9 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=256)
     ap.add_argument("--warmup", type=int, default=16)
-    ap.add_argument("--rho", type=float, default=0.9)
+    ap.add_argument("--rho", type=float, default=None, help="AR(1) coefficient of the headline run (default 0.9)")
+    ap.add_argument("--workload", default=WORKLOAD, choices=sorted(synth.CONFIGS),
+                    help="default: the DeepSeek-V2-Lite-shaped batch-1 stack the metric is quoted on")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layers", type=int, default=0, help="use only this many layers (profiling captures)")
     ap.add_argument("--no-sweep", action="store_true")
@@ -419,6 +424,8 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if args.impl == "reference":
+        if args.rho is None:
+            args.rho = 0.9 if args.workload == "dsv2lite" else synth.config(args.workload)["rhos"][0]
         run_reference(args, rank, world)
     else:
         run_ours(args, rank, world, local_rank)

@@ -233,7 +233,7 @@ __device__ void resolve_layer(const DevStack& d, int l, const int* flat, int n_f
   }
 }
 
-__global__ void __launch_bounds__(256) route_kernel(DevStack d, const float* __restrict__ hidden_in,
+__global__ void __launch_bounds__(1024) route_kernel(DevStack d, const float* __restrict__ hidden_in,
                                                     int* __restrict__ ids, float* __restrict__ gates,
                                                     int* contrib) {
   __shared__ float z[kMaxRouted];
@@ -247,11 +247,12 @@ __global__ void __launch_bounds__(256) route_kernel(DevStack d, const float* __r
   const float* h = hidden_in + (size_t)lb * d.H;
   const size_t row_bytes = (size_t)d.H * d.wbytes;
 
-  for (int e = warp; e < d.N; e += 8) {
+  const int n_warps = blockDim.x >> 5;
+  for (int e = warp; e < d.N; e += n_warps) {
     const float acc = row_dot(d.router + ((size_t)l * d.N + e) * row_bytes, h, d.H, d.wbytes, lane);
     if (lane == 0) z[e] = acc;
   }
-  if (warp == 7) {
+  if (warp == n_warps - 1) {
     float sc = 1.f;
     if (d.shared_gate) {
       const float dot = row_dot(d.shared_gate_w + (size_t)l * row_bytes, h, d.H, d.wbytes, lane);
@@ -348,7 +349,8 @@ __global__ void __launch_bounds__(32) resolve_kernel(DevStack d, const int* __re
 
 cudaError_t launch_route(const DevStack& d, const float* hidden_in, int* ids, float* gates,
                          int* contrib, cudaStream_t st) {
-  route_kernel<<<d.L * d.B, 256, 0, st>>>(d, hidden_in, ids, gates, contrib);
+  // few CTAs at batch 1: give each as many warps as it can hold so the router rows load in parallel
+  route_kernel<<<d.L * d.B, d.B == 1 ? 1024 : 256, 0, st>>>(d, hidden_in, ids, gates, contrib);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   if (d.B > 1) {

@@ -63,3 +63,34 @@ def test_qwen15moe_full_shape():
 def test_qwen3_30b_full_shape():
     res = _full("qwen3_30b", [0.5, 0.9], [192, 192], distinct=16)
     print("qwen3_30b:", res)
+
+
+def test_dsv2lite_b32_full_shape():
+    """The batched serving configuration: 32 sequences share 32 slots per layer, so a step's distinct
+    requests (about 61) exceed the capacity and slots are handed on within the step."""
+    import torch
+    from paper_2605_27081_b200.loader import LoadedWorkload
+    from parity_util import StepChecker, oracle_for
+
+    cfg = synth.config("dsv2lite_b32")
+    shape = cfg["shape"]
+    stream = torch.cuda.Stream()
+    wl = LoadedWorkload(shape, cfg["cache_slots"], cfg["seed"], stream=stream.cuda_stream, distinct_experts=32)
+    try:
+        chk = StepChecker(wl, oracle_for(wl), torch)
+        hs = synth.HiddenStream(cfg["seed"], shape, None)
+        n, over = 20, 0
+        with torch.cuda.stream(stream):
+            for t in range(n):
+                h = hs.step()
+                if t in (0, n - 1):
+                    r, _ = chk.step(h, ffn="selected", ffn_layers=[t % shape.n_layers])
+                else:
+                    r, _ = chk.step(h, ffn=None)
+                over += sum(1 for q in r["requests"] if len(q) > cfg["cache_slots"])
+        chk.check_counters()
+        assert over > 0.9 * n * shape.n_layers
+        print("dsv2lite_b32: near ties", chk.near_ties, "max out err", chk.max_out_err, "uHR", chk.o.uhr(),
+              "tHR", chk.o.thr(), "EOR", chk.o.eor())
+    finally:
+        wl.close()
