@@ -247,6 +247,24 @@ def measure_h2d(torch, nbytes, reps=8):
     return best
 
 
+def reduce_over_ranks(dist, maxima: dict, sums: dict, device):
+    """Whole-job figures of N independent replicas: times are the maximum over ranks, counts the
+    sum.  `dist` is torch.distributed (initialised) or None for a single process."""
+    out = dict(maxima)
+    out.update(sums)
+    if dist is None:
+        return out
+    import torch
+    for keys, op in ((sorted(maxima), dist.ReduceOp.MAX), (sorted(sums), dist.ReduceOp.SUM)):
+        if not keys:
+            continue
+        t = torch.tensor([float(out[k]) for k in keys], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=op)
+        for k, v in zip(keys, t.tolist()):
+            out[k] = v
+    return out
+
+
 def run_ours(args, rank, world, local_rank):
     import torch
     from paper_2605_27081_b200.loader import LoadedWorkload
@@ -286,10 +304,10 @@ def run_ours(args, rank, world, local_rank):
     results = {}
     clocks = None
     for rho in rhos:
-        head = rho == args.rho
+        is_head = rho == args.rho
         barrier()
-        sampler = ClockSampler(local_rank) if (head and rank == 0) else None
-        results[rho] = run_rho(torch, wl, stream, shape, seed, rho, args.steps, args.warmup, with_e2e=head)
+        sampler = ClockSampler(local_rank) if (is_head and rank == 0) else None
+        results[rho] = run_rho(torch, wl, stream, shape, seed, rho, args.steps, args.warmup, with_e2e=is_head)
         barrier()
         if sampler is not None:
             clocks = sampler.stop()
@@ -305,17 +323,10 @@ def run_ours(args, rank, world, local_rank):
         resident = r
         wl_r.stack.close()
 
-    def agg(x, op="max"):
-        if dist is None:
-            return x
-        t = torch.tensor([float(x)], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX if op == "max" else dist.ReduceOp.SUM)
-        return float(t.item())
-
     head = results[args.rho]
-    ms = agg(head["ms"])
-    e2e_ms = agg(head["e2e_ms"])
-    launches = agg(head["launches"], "sum")
+    red = reduce_over_ranks(dist, {"ms": head["ms"], "e2e_ms": head["e2e_ms"]}, {"launches": head["launches"]},
+                            "cuda")
+    ms, e2e_ms, launches = red["ms"], red["e2e_ms"], red["launches"]
     if rank != 0:
         wl.close()
         if dist is not None:
