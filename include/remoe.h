@@ -141,6 +141,25 @@ int remoe_cache_stats(remoe_stack*, int32_t layer, remoe_cache_counters* out);
 int remoe_reuse_stats(remoe_stack*, int32_t layer, uint64_t* overlap_sum,
                       uint64_t* pairs_counted, float* last_ir);
 
+/* Reuse mass (Eq. 2): m_t = (1/K) * sum over k in E_{t-1} of P_t^(k), the probability the current
+ * router puts on the previous step's experts.  mass_sum = sum of m_t over the counted (step,
+ * sequence) pairs of the layer (layer = -1: all layers), pairs = their number, last_mass (host,
+ * [L, B] or [B], may be NULL) = m_t of the most recent step, -1 where t = 1. */
+int remoe_reuse_mass(remoe_stack*, int32_t layer, double* mass_sum, uint64_t* pairs, float* last_mass);
+
+/* Per-step aggregates over all layers since the last reset (App. E.2.5): for steps first ..
+ * first+count-1, umiss[i] = #uMiss^(all) of the step and tok_hits[i] = H_tok^(all) (either may be
+ * NULL); n_steps receives how many steps are recorded.  Host-side bookkeeping, no device work. */
+int remoe_step_history(remoe_stack*, int32_t first, int32_t count, uint32_t* umiss, uint32_t* tok_hits,
+                       int32_t* n_steps);
+
+/* I/O-time and TPOT proxy of App. E.2.5 / E.3: io_ms[i] = umiss[i] * expert_bytes / bandwidth * 1000
+ * with bandwidth_gbps in 10^9 bytes/s, TPOT_i = tpot_compute_ms + io_ms[i] / batch.  io_ms ([n], may
+ * be NULL) receives the per-step I/O time, tpot_p50_p95_p99 ([3], may be NULL) the percentiles of
+ * TPOT over the n steps (linear interpolation between order statistics).  Pure host arithmetic. */
+int remoe_tpot_proxy(const uint32_t* umiss, int32_t n, uint64_t expert_bytes, double bandwidth_gbps,
+                     int32_t batch, double tpot_compute_ms, double* io_ms, double* tpot_p50_p95_p99);
+
 /* Empty every layer's cache, forget E_{t-1} and zero all counters (Sec. 3: each request
  * starts from a cold expert cache). */
 int remoe_cache_reset(remoe_stack*);

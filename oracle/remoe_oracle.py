@@ -100,6 +100,31 @@ def unique_in_order(r):
     return out
 
 
+def reuse_mass(p_t, e_prev, k):
+    """m_t = (1/K) sum_{j in E_{t-1}} P_t^(j), the reuse mass (Eq. 2)."""
+    p_t = np.asarray(p_t, dtype=F64)
+    return float(sum(p_t[int(j)] for j in e_prev) / k)
+
+
+def io_ms_step(umiss, expert_bytes, bandwidth_gbps):
+    """IO_ms_step = #uMiss * expert_bytes / bandwidth * 1000, bandwidth in 1e9 bytes/s (App. E.2.5)."""
+    return np.asarray(umiss, dtype=F64) * float(expert_bytes) / (float(bandwidth_gbps) * 1e9) * 1000.0
+
+
+def tpot_proxy(umiss, expert_bytes, bandwidth_gbps, batch=1, tpot_compute_ms=0.0):
+    """TPOT ~ TPOT_compute + IO_step / B per step (App. E.3), and its P50/P95/P99 over the steps
+    (linear interpolation between order statistics; the paper does not say which rule it uses)."""
+    tpot = tpot_compute_ms + io_ms_step(umiss, expert_bytes, bandwidth_gbps) / batch
+    srt = sorted(float(x) for x in tpot)
+    out = []
+    for q in (0.50, 0.95, 0.99):
+        pos = q * (len(srt) - 1)
+        lo = int(pos)
+        hi = min(lo + 1, len(srt) - 1)
+        out.append(srt[lo] + (pos - lo) * (srt[hi] - srt[lo]))
+    return tpot, out
+
+
 def reuse_overlap(e_t, e_prev):
     """|E_t n E_{t-1}|, the numerator of IR_t (Eq. 1)."""
     return len(set(int(x) for x in e_t) & set(int(x) for x in e_prev))
@@ -284,6 +309,9 @@ class OracleStack:
         self.uniq_misses = [0] * L
         self.overlap_sum = [0] * L
         self.pairs_counted = [0] * L
+        self.mass_sum = [0.0] * L
+        self.hist_umiss = []          # per step, summed over layers (App. E.2.5)
+        self.hist_tok_hits = []
         self.steps = 0
 
     def route(self, l, h_lb, override=None):
@@ -319,14 +347,15 @@ class OracleStack:
         res = dict(
             ids=np.zeros((L, B, K), np.int64), gates=np.zeros((L, B, K), F64),
             margin=np.zeros((L, B), F64), overlap=np.full((L, B), -1, np.int64),
-            requests=[], hit=[], slot=[], evicted=[],
+            mass=np.full((L, B), -1.0, F64),
+            requests=[], hit=[], slot=[], evicted=[], tok_hits=[],
             out=None if ffn is None else np.zeros((L, B, s.hidden), F64),
             shared_scale=np.ones((L, B), F64))
         for l in range(L):
             flat = []
             for b in range(B):
                 ov = None if id_override is None else id_override.get((l, b))
-                ids, g, margin, _, _ = self.route(l, h[l, b], ov)
+                ids, g, margin, _, p = self.route(l, h[l, b], ov)
                 res["ids"][l, b], res["gates"][l, b], res["margin"][l, b] = ids, g, margin
                 flat.extend(int(e) for e in ids)
                 if self.prev[l][b] is not None:                       # Eq. (1), t >= 2
@@ -334,6 +363,8 @@ class OracleStack:
                     res["overlap"][l, b] = ov_n
                     self.overlap_sum[l] += ov_n
                     self.pairs_counted[l] += 1
+                    res["mass"][l, b] = reuse_mass(p, self.prev[l][b], K)          # Eq. (2)
+                    self.mass_sum[l] += res["mass"][l, b]
                 self.prev[l][b] = [int(e) for e in ids]
                 if s.shared_gate:
                     res["shared_scale"][l, b] = sigmoid(
@@ -342,6 +373,7 @@ class OracleStack:
             before = cache.resident()                                  # C_t
             th = sum(1 for e in flat if e in before)                   # token level, App. E.2.3
             self.tok_hits[l] += th
+            res["tok_hits"].append(th)
             self.tok_misses[l] += len(flat) - th
             req = unique_in_order(flat)                                # U
             hit, slot, evicted = cache.serve(req)
@@ -358,6 +390,8 @@ class OracleStack:
                         h[l, b], res["ids"][l, b], res["gates"][l, b], s.n_routed,
                         lambda e, l=l: self.expert_weights(l, e), shared,
                         res["shared_scale"][l, b], mode=ffn)
+        self.hist_umiss.append(sum(len(hh) - sum(hh) for hh in res["hit"]))
+        self.hist_tok_hits.append(sum(res["tok_hits"]))
         self.steps += 1
         return res
 

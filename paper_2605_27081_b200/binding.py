@@ -25,7 +25,7 @@ EXPORTS = [
     "remoe_decode_step", "remoe_decode_step_host", "remoe_last_step_trace", "remoe_cache_stats",
     "remoe_reuse_stats", "remoe_cache_reset", "remoe_set_policy", "remoe_set_reroute_beta",
     "remoe_set_profiling", "remoe_kernel_time", "remoe_launch_count", "remoe_last_cuda_error", "remoe_stack_destroy",
-    "remoe_strerror", "remoe_expert_ffn_static",
+    "remoe_strerror", "remoe_expert_ffn_static", "remoe_reuse_mass", "remoe_step_history", "remoe_tpot_proxy",
 ]
 
 
@@ -76,6 +76,9 @@ def lib():
         L.remoe_launch_count.argtypes = [vp, C.POINTER(C.c_uint64)]
         L.remoe_expert_ffn_static.argtypes = [i32, i32, i32, C.POINTER(vp), C.POINTER(i32), C.POINTER(C.c_float),
                                               vp, vp, vp]
+        L.remoe_reuse_mass.argtypes = [vp, i32, C.POINTER(C.c_double), C.POINTER(C.c_uint64), vp]
+        L.remoe_step_history.argtypes = [vp, i32, i32, vp, vp, C.POINTER(i32)]
+        L.remoe_tpot_proxy.argtypes = [vp, i32, C.c_uint64, C.c_double, i32, C.c_double, vp, vp]
         L.remoe_last_cuda_error.argtypes = [vp]
         L.remoe_last_cuda_error.restype = C.c_char_p
         L.remoe_stack_destroy.argtypes = [vp]
@@ -200,6 +203,31 @@ def remoe_expert_ffn_static(hidden, weight_dtype, expert_blocks_dev, inter, scal
                                          _ptr(hidden_in), _ptr(hidden_out), cuda_stream)
 
 
+def remoe_reuse_mass(h, layer=-1, last_mass=None):
+    m, p = C.c_double(), C.c_uint64()
+    rc = lib().remoe_reuse_mass(h, int(layer), C.byref(m), C.byref(p), _ptr(last_mass))
+    return rc, float(m.value), int(p.value)
+
+
+def remoe_step_history(h, first=0, count=None):
+    n = C.c_int32()
+    rc = lib().remoe_step_history(h, 0, 0, None, None, C.byref(n))
+    if rc != REMOE_OK:
+        return rc, None, None
+    count = max(0, n.value - first) if count is None else count
+    um, th = np.zeros(count, np.uint32), np.zeros(count, np.uint32)
+    rc = lib().remoe_step_history(h, int(first), int(count), _ptr(um), _ptr(th), C.byref(n))
+    return rc, um, th
+
+
+def remoe_tpot_proxy(umiss, expert_bytes, bandwidth_gbps, batch=1, tpot_compute_ms=0.0):
+    um = np.ascontiguousarray(umiss, dtype=np.uint32)
+    io, pct = np.zeros(um.size, np.float64), np.zeros(3, np.float64)
+    rc = lib().remoe_tpot_proxy(_ptr(um), um.size, int(expert_bytes), float(bandwidth_gbps), int(batch),
+                                float(tpot_compute_ms), _ptr(io), _ptr(pct))
+    return rc, io, pct
+
+
 def remoe_last_cuda_error(h) -> str:
     return lib().remoe_last_cuda_error(h).decode()
 
@@ -259,6 +287,18 @@ class Stack:
         rc, o, p = remoe_reuse_stats(self.h, layer, ir)
         self._ck(rc, "remoe_reuse_stats")
         return (o, p, ir) if want_last_ir else (o, p)
+
+    def reuse_mass(self, layer=-1, want_last=False):
+        n = self.shape.batch * (self.shape.n_layers if layer < 0 else 1)
+        last = np.empty(n, np.float32) if want_last else None
+        rc, m, p = remoe_reuse_mass(self.h, layer, last)
+        self._ck(rc, "remoe_reuse_mass")
+        return (m, p, last) if want_last else (m, p)
+
+    def step_history(self, first=0, count=None):
+        rc, um, th = remoe_step_history(self.h, first, count)
+        self._ck(rc, "remoe_step_history")
+        return um, th
 
     def cache_reset(self):
         self._ck(remoe_cache_reset(self.h), "remoe_cache_reset")

@@ -14,7 +14,9 @@
 // break the fetch bound of Prop. 3.1).
 #include "remoe_internal.cuh"
 
+#include <algorithm>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <string>
@@ -54,6 +56,7 @@ struct remoe_stack {
   std::vector<cudaEvent_t> ev_pool;        // copy-done / compute-done events of the waves
   uint64_t steps = 0, steps_since_reset = 0;
   std::vector<uint64_t> h2d_bytes;         // per layer
+  std::vector<uint32_t> hist_umiss, hist_tok_hits;   // per step since the last reset, summed over layers
   // staging for the host-buffer entry point
   float *st_in_d = nullptr, *st_out_d = nullptr, *st_g_d = nullptr;
   int* st_ids_d = nullptr;
@@ -122,11 +125,15 @@ int reset_state(remoe_stack* s) {
   CK(cudaMemsetAsync(d.prev_mask, 0, L * d.B * kMaskWords * sizeof(unsigned), s->stream));
   CK(cudaMemsetAsync(d.counters, 0, L * kCounters * sizeof(unsigned long long), s->stream));
   CK(cudaMemsetAsync(d.last_overlap, 0xff, L * d.B * sizeof(int), s->stream));
+  CK(cudaMemsetAsync(d.last_mass, 0, L * d.B * sizeof(float), s->stream));
+  CK(cudaMemsetAsync(d.mass_sum, 0, L * d.B * sizeof(double), s->stream));
   CK(cudaMemsetAsync(s->dev_block, 0, s->block_ints * sizeof(int), s->stream));
   CK(cudaStreamSynchronize(s->stream));
   s->steps = 0;
   s->steps_since_reset = 0;
   std::fill(s->h2d_bytes.begin(), s->h2d_bytes.end(), 0);
+  s->hist_umiss.clear();
+  s->hist_tok_hits.clear();
   return REMOE_OK;
 }
 
@@ -223,6 +230,20 @@ int decode_step_batched(remoe_stack* s, const float* hin, float* hout, int32_t* 
   s->steps_since_reset += 1;
   if (check_device_flag(s) != REMOE_OK) return REMOE_E_DEVICE_FLAG;
 
+  {
+    // per-step all-layer aggregates (App. E.2.5)
+    const int* th = trace_tok_hits(s->host_block + 1, d.L, s->BK);
+    const int* nu = trace_n_unique(s->host_block + 1);
+    const int* hh = trace_hit(s->host_block + 1, d.L, s->BK);
+    uint32_t um = 0, tk = 0;
+    for (int l = 0; l < d.L; ++l) {
+      tk += (uint32_t)th[l];
+      for (int i = 0; i < nu[l] && i < s->BK; ++i) um += hh[l * s->BK + i] ? 0u : 1u;
+    }
+    s->hist_umiss.push_back(um);
+    s->hist_tok_hits.push_back(tk);
+  }
+
   int* tr = s->host_block + 1;
   const int* t_nu = trace_n_unique(tr);
   const int* t_req = trace_requests(tr, d.L, BK);
@@ -240,7 +261,7 @@ int decode_step_batched(remoe_stack* s, const float* hin, float* hout, int32_t* 
         return REMOE_E_DEVICE_FLAG;
       if (t_depth[j] > max_depth) max_depth = t_depth[j];
     }
-    resident_bytes += (uint64_t)d.S * d.shared_bytes * ((d.B + kTokTile - 1) / kTokTile);
+    resident_bytes += (uint64_t)d.S * d.shared_bytes;   // algorithmic: once, although every token tile streams it
   }
   if (s->profiling) s->ev_used[prof_slot].bytes = resident_bytes;
 
@@ -399,6 +420,8 @@ int remoe_stack_create(const remoe_shape* sh, int32_t cache_slots, void* cuda_st
   TRY(dev_alloc(s, &d.counters, L * kCounters));
   TRY(dev_alloc(s, &d.shared_scale, L * d.B));
   TRY(dev_alloc(s, &d.last_overlap, L * d.B));
+  TRY(dev_alloc(s, &d.last_mass, L * d.B));
+  TRY(dev_alloc(s, &d.mass_sum, L * d.B));
   s->block_ints = 1 + (size_t)trace_ints(d.L, s->BK);
   TRY(dev_alloc(s, &s->dev_block, s->block_ints));
   TRY(host_alloc(s, &s->host_block, s->block_ints));
@@ -519,6 +542,20 @@ int remoe_decode_step(remoe_stack* s, const float* hin, float* hout, int32_t* id
   s->steps_since_reset += 1;
   if (check_device_flag(s) != REMOE_OK) return REMOE_E_DEVICE_FLAG;
 
+  {
+    // per-step all-layer aggregates (App. E.2.5)
+    const int* th = trace_tok_hits(s->host_block + 1, d.L, s->BK);
+    const int* nu = trace_n_unique(s->host_block + 1);
+    const int* hh = trace_hit(s->host_block + 1, d.L, s->BK);
+    uint32_t um = 0, tk = 0;
+    for (int l = 0; l < d.L; ++l) {
+      tk += (uint32_t)th[l];
+      for (int i = 0; i < nu[l] && i < s->BK; ++i) um += hh[l * s->BK + i] ? 0u : 1u;
+    }
+    s->hist_umiss.push_back(um);
+    s->hist_tok_hits.push_back(tk);
+  }
+
   int* tr = s->host_block + 1;
   const int* t_req = trace_requests(tr, d.L, s->BK);
   const int* t_hit = trace_hit(tr, d.L, s->BK);
@@ -636,6 +673,66 @@ int remoe_reuse_stats(remoe_stack* s, int32_t layer, uint64_t* overlap_sum, uint
         const int v = ov[(size_t)l * s->d.B + b];
         last_ir[j++] = v < 0 ? -1.f : (float)v / (float)s->d.K;
       }
+  }
+  return REMOE_OK;
+}
+
+int remoe_reuse_mass(remoe_stack* s, int32_t layer, double* mass_sum, uint64_t* pairs, float* last_mass) {
+  if (!s || layer < -1 || layer >= s->d.L) return REMOE_E_ARG;
+  CK(cudaStreamSynchronize(s->stream));
+  const size_t n = (size_t)s->d.L * s->d.B;
+  std::vector<double> ms(n);
+  std::vector<float> lm(n);
+  std::vector<unsigned long long> c((size_t)s->d.L * kCounters);
+  CK(cudaMemcpy(ms.data(), s->d.mass_sum, n * sizeof(double), cudaMemcpyDeviceToHost));
+  CK(cudaMemcpy(lm.data(), s->d.last_mass, n * sizeof(float), cudaMemcpyDeviceToHost));
+  CK(cudaMemcpy(c.data(), s->d.counters, c.size() * sizeof(unsigned long long), cudaMemcpyDeviceToHost));
+  double tot = 0.0;
+  uint64_t p = 0;
+  size_t j = 0;
+  for (int l = 0; l < s->d.L; ++l) {
+    if (layer >= 0 && l != layer) continue;
+    p += c[(size_t)l * kCounters + 5];
+    for (int b = 0; b < s->d.B; ++b) {
+      tot += ms[(size_t)l * s->d.B + b];           // fixed order: layer, then sequence
+      if (last_mass) last_mass[j++] = lm[(size_t)l * s->d.B + b];
+    }
+  }
+  if (mass_sum) *mass_sum = tot;
+  if (pairs) *pairs = p;
+  return REMOE_OK;
+}
+
+int remoe_step_history(remoe_stack* s, int32_t first, int32_t count, uint32_t* umiss, uint32_t* tok_hits,
+                       int32_t* n_steps) {
+  if (!s || first < 0 || count < 0) return REMOE_E_ARG;
+  const int32_t have = (int32_t)s->hist_umiss.size();
+  if (n_steps) *n_steps = have;
+  for (int32_t i = 0; i < count && first + i < have; ++i) {
+    if (umiss) umiss[i] = s->hist_umiss[first + i];
+    if (tok_hits) tok_hits[i] = s->hist_tok_hits[first + i];
+  }
+  return REMOE_OK;
+}
+
+int remoe_tpot_proxy(const uint32_t* umiss, int32_t n, uint64_t expert_bytes, double bandwidth_gbps, int32_t batch,
+                     double tpot_compute_ms, double* io_ms, double* tpot_p50_p95_p99) {
+  if (!umiss || n < 1 || batch < 1 || !(bandwidth_gbps > 0.0)) return REMOE_E_ARG;
+  std::vector<double> tpot((size_t)n);
+  for (int32_t i = 0; i < n; ++i) {
+    const double io = (double)umiss[i] * (double)expert_bytes / (bandwidth_gbps * 1e9) * 1000.0;
+    if (io_ms) io_ms[i] = io;
+    tpot[i] = tpot_compute_ms + io / (double)batch;
+  }
+  if (tpot_p50_p95_p99) {
+    std::sort(tpot.begin(), tpot.end());
+    const double q[3] = {0.50, 0.95, 0.99};
+    for (int k = 0; k < 3; ++k) {
+      const double pos = q[k] * (double)(n - 1);          // linear interpolation between order statistics
+      const int32_t lo = (int32_t)pos;
+      const int32_t hi = lo + 1 < n ? lo + 1 : lo;
+      tpot_p50_p95_p99[k] = tpot[lo] + (pos - (double)lo) * (tpot[hi] - tpot[lo]);
+    }
   }
   return REMOE_OK;
 }

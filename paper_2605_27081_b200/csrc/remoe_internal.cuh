@@ -48,8 +48,11 @@ struct DevStack {
 
   float* shared_scale;                 // [L][B]
   int* last_overlap;                   // [L][B]   -1 when not counted
+  float* last_mass;                    // [L][B]   reuse mass m_t of the last step (Eq. 2), -1 at t = 1
+  double* mass_sum;                    // [L][B]   running sum of m_t over counted steps
   // Step trace, one block so that a single copy brings it to the host:
   // n_unique[L] | requests[L][B*K] | hit[L][B*K] | slot[L][B*K] | evicted[L][B*K] | depth[L][B*K]
+  // | tok_hits[L]  (token-level hits of this step, App. E.2.3)
   // depth: how many of this step's experts occupied the request's slot before it within the
   // step (0 unless the step asks for more distinct experts than there are slots).
   int* trace;
@@ -60,7 +63,8 @@ struct DevStack {
   int* grp_k;                          // [L][B*K][B]
 };
 
-__host__ __device__ inline int trace_ints(int L, int BK) { return L + 5 * L * BK; }
+__host__ __device__ inline int trace_ints(int L, int BK) { return 2 * L + 5 * L * BK; }
+__host__ __device__ inline int* trace_tok_hits(int* t, int L, int BK) { return t + L + 5 * L * BK; }
 __host__ __device__ inline int* trace_depth(int* t, int L, int BK) { return t + L + 4 * L * BK; }
 __host__ __device__ inline int* trace_n_unique(int* t) { return t; }
 __host__ __device__ inline int* trace_requests(int* t, int L, int BK) { return t + L; }

@@ -228,6 +228,7 @@ __device__ void resolve_layer(const DevStack& d, int l, const int* flat, int n_f
     c[2] += (unsigned long long)uniq_h;
     c[3] += (unsigned long long)(n_u - uniq_h);
     trace_n_unique(d.trace)[l] = n_u;
+    trace_tok_hits(d.trace, d.L, BK)[l] = tok_h;
     contrib[(d.L + l) * 2 + 0] = 1;      // no miss-phase contribution yet for this layer
     contrib[(d.L + l) * 2 + 1] = 0;
   }
@@ -314,20 +315,28 @@ __global__ void __launch_bounds__(1024) route_kernel(DevStack d, const float* __
     gates[(size_t)lb * d.K + lane] = s_g[lane];
   }
 
-  // Reuse: |E_t n E_{t-1}| from selection bit masks (Eq. 1); counted from the second step on.
+  // Reuse: |E_t n E_{t-1}| from selection bit masks (Eq. 1) and the reuse mass
+  // m_t = (1/K) sum_{k in E_{t-1}} P_t^(k) (Eq. 2); both counted from the second step on.
   int ov = 0;
+  float mass = 0.f;
 #pragma unroll
   for (int j = 0; j < kMaskWords; ++j) {
     const unsigned word = __ballot_sync(kFull, (taken >> j) & 1u);
+    unsigned* pm = d.prev_mask + (size_t)lb * kMaskWords + j;
+    const unsigned prev = d.has_prev ? *pm : 0u;
+    __syncwarp();
+    if ((prev >> lane) & 1u) mass += expf(v[j] - m) / sum;
     if (lane == 0) {
-      unsigned* pm = d.prev_mask + (size_t)lb * kMaskWords + j;
-      if (d.has_prev) ov += __popc(word & *pm);
+      ov += __popc(word & prev);
       *pm = word;
     }
   }
+  mass = warp_sum(mass) / (float)d.K;
   if (lane == 0) {
     d.last_overlap[lb] = d.has_prev ? ov : -1;
+    d.last_mass[lb] = d.has_prev ? mass : -1.f;
     if (d.has_prev) {
+      d.mass_sum[lb] += (double)mass;
       atomicAdd(d.counters + (size_t)l * kCounters + 4, (unsigned long long)ov);
       atomicAdd(d.counters + (size_t)l * kCounters + 5, 1ull);
     }

@@ -96,6 +96,8 @@ class StepChecker:
                 assert [bool(x) for x in tr["hit"][l][:n]] == r["hit"][l]
                 assert list(tr["slot"][l][:n]) == r["slot"][l]
                 assert list(tr["evicted"][l][:n]) == r["evicted"][l]
+        _, _, last_mass = self.wl.stack.reuse_mass(-1, want_last=True)
+        assert np.allclose(last_mass, r["mass"].reshape(-1), atol=2e-6), "reuse mass differs"
         if ffn is not None:
             tol = TOL[self.wl.shape.weight_dtype]
             for l in (range(self.L) if ffn_layers is None else ffn_layers):
@@ -120,3 +122,15 @@ class StepChecker:
             assert (ov, pairs) == (o.overlap_sum[l], o.pairs_counted[l])
         ov, pairs = st.reuse_stats(-1)
         assert (ov, pairs) == (sum(o.overlap_sum), sum(o.pairs_counted))
+        # reporting: reuse mass (Eq. 2), per-step aggregates and the TPOT proxy (App. E.2.5)
+        from paper_2605_27081_b200 import binding as B
+        m, p = st.reuse_mass(-1)
+        assert p == sum(o.pairs_counted) and abs(m - sum(o.mass_sum)) <= 1e-5 * max(1.0, p)
+        um, th = st.step_history()
+        assert list(um) == o.hist_umiss and list(th) == o.hist_tok_hits
+        if len(um):
+            eb = synth.expert_block_bytes(self.wl.shape)
+            rc, io, pct = B.remoe_tpot_proxy(um, eb, 4.0, self.B, 12.5)
+            t_ref, pct_ref = orc.tpot_proxy(um, eb, 4.0, self.B, 12.5)
+            assert rc == 0 and np.allclose(io, orc.io_ms_step(um, eb, 4.0), rtol=1e-12)
+            assert np.allclose(pct, pct_ref, rtol=1e-12)
