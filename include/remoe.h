@@ -118,6 +118,22 @@ int remoe_load_experts_host(remoe_stack*, int32_t layer, int32_t first_expert, i
 int remoe_decode_step(remoe_stack*, const float* hidden_in_dev, float* hidden_out_dev,
                       int32_t* selected_ids_dev, float* gate_weights_dev);
 
+/*
+ * Chained variant of the step (batch 1): the layers feed each other through a residual
+ * connection, h_{l+1} = h_l + MoE_l(h_l), as in a decoder stack, instead of each reading its own
+ * stream (the paper treats layers independently, App. A.5; chaining is how they sit in a model).
+ *   hidden_in    dev [H]        h_0
+ *   hidden_out   dev [H]        h_L
+ *   layer_inputs dev [L, H]     h_0 .. h_{L-1} (may be NULL)
+ *   selected_ids dev [L, K], gate_weights dev [L, K]
+ * Routing of layer l+1 depends on layer l's output, so the host waits for one small trace per
+ * layer instead of one per step, and a layer's fetches cannot start before the layer above it
+ * has finished.  Cache, counters and reuse statistics behave exactly as in remoe_decode_step.
+ * Errors: ARG, NOT_LOADED, UNSUPPORTED (batch > 1), CUDA, DEVICE_FLAG.
+ */
+int remoe_decode_step_chained(remoe_stack*, const float* hidden_in_dev, float* hidden_out_dev,
+                              float* layer_inputs_dev, int32_t* selected_ids_dev, float* gate_weights_dev);
+
 /* Same step with HOST buffers (pageable or pinned): copies hidden_in to the device, runs
  * the step, copies the three outputs back and returns when they are complete. */
 int remoe_decode_step_host(remoe_stack*, const float* hidden_in_host, float* hidden_out_host,

@@ -333,8 +333,13 @@ class OracleStack:
         g = gate_weights(p, ids, s.renorm_topk)
         return ids, g, margin, z, p
 
-    def step(self, h, ffn="selected", id_override=None, ffn_layers=None):
+    def step(self, h, ffn="selected", id_override=None, ffn_layers=None, chained=False):
         """Advance every layer by one token.  h: [L, B, H].
+
+        chained=True: h is [B, H], the input of layer 0, and the layers feed each other through
+        a residual connection, h_{l+1} = h_l + MoE_l(h_l) (how MoE layers sit in a decoder; the
+        paper's analysis treats each layer on its own).  The result then also carries
+        "layer_inputs" [L, B, H] and "final" [B, H]; `ffn` must not be None.
 
         ffn: "dense", "selected" or None (integer parts only).  `ffn_layers` restricts the
         floating-point FFN to some layers.  `id_override[(l, b)]` forces the selected ids
@@ -351,11 +356,17 @@ class OracleStack:
             requests=[], hit=[], slot=[], evicted=[], tok_hits=[],
             out=None if ffn is None else np.zeros((L, B, s.hidden), F64),
             shared_scale=np.ones((L, B), F64))
+        if chained:
+            cur = np.asarray(h, dtype=F64).reshape(B, s.hidden).copy()
+            res["layer_inputs"] = np.zeros((L, B, s.hidden), F64)
         for l in range(L):
+            hl = cur if chained else h[l]
+            if chained:
+                res["layer_inputs"][l] = cur
             flat = []
             for b in range(B):
                 ov = None if id_override is None else id_override.get((l, b))
-                ids, g, margin, _, p = self.route(l, h[l, b], ov)
+                ids, g, margin, _, p = self.route(l, hl[b], ov)
                 res["ids"][l, b], res["gates"][l, b], res["margin"][l, b] = ids, g, margin
                 flat.extend(int(e) for e in ids)
                 if self.prev[l][b] is not None:                       # Eq. (1), t >= 2
@@ -368,7 +379,7 @@ class OracleStack:
                 self.prev[l][b] = [int(e) for e in ids]
                 if s.shared_gate:
                     res["shared_scale"][l, b] = sigmoid(
-                        np.asarray(self.shared_gates[l], dtype=F64) @ np.asarray(h[l, b], dtype=F64))
+                        np.asarray(self.shared_gates[l], dtype=F64) @ np.asarray(hl[b], dtype=F64))
             cache = self.caches[l]
             before = cache.resident()                                  # C_t
             th = sum(1 for e in flat if e in before)                   # token level, App. E.2.3
@@ -387,9 +398,13 @@ class OracleStack:
                 shared = [self.shared_weights(l, i) for i in range(s.n_shared)]
                 for b in range(B):
                     res["out"][l, b] = moe_output(
-                        h[l, b], res["ids"][l, b], res["gates"][l, b], s.n_routed,
+                        hl[b], res["ids"][l, b], res["gates"][l, b], s.n_routed,
                         lambda e, l=l: self.expert_weights(l, e), shared,
                         res["shared_scale"][l, b], mode=ffn)
+            if chained:
+                cur = cur + res["out"][l]
+        if chained:
+            res["final"] = cur
         self.hist_umiss.append(sum(len(hh) - sum(hh) for hh in res["hit"]))
         self.hist_tok_hits.append(sum(res["tok_hits"]))
         self.steps += 1

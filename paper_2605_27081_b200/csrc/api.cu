@@ -44,6 +44,8 @@ struct remoe_stack {
   size_t block_ints = 0;
   float* partial = nullptr;
   int* contrib = nullptr;
+  float* chain_in = nullptr;               // [L + 1][H] layer inputs of the chained mode
+  float* chain_out = nullptr;              // [L][H] per-layer MoE outputs of the chained mode
   cudaEvent_t ev_trace = nullptr;
   std::vector<cudaEvent_t> ev_layer;
   // batched path (B > 1)
@@ -199,7 +201,7 @@ int decode_step_batched(remoe_stack* s, const float* hin, float* hout, int32_t* 
   d.beta = s->beta;
   const int BK = s->BK;
 
-  CK(launch_route(d, hin, ids, gates, s->contrib, s->stream));
+  CK(launch_route(d, hin, ids, gates, s->contrib, 0, d.L, s->stream));
   s->kernel_launches += 2;
   CK(cudaMemcpyAsync(s->host_block, s->dev_block, s->block_ints * sizeof(int), cudaMemcpyDeviceToHost, s->stream));
   CK(cudaEventRecord(s->ev_trace, s->stream));
@@ -430,6 +432,8 @@ int remoe_stack_create(const remoe_shape* sh, int32_t cache_slots, void* cuda_st
   d.trace = s->dev_block + 1;
   TRY(dev_alloc(s, &s->partial, (size_t)2 * L * s->grid * d.H));
   TRY(dev_alloc(s, &s->contrib, (size_t)2 * L * 2));
+  TRY(dev_alloc(s, &s->chain_in, (L + 1) * d.B * d.H));
+  TRY(dev_alloc(s, &s->chain_out, L * d.B * d.H));
   if (d.B > 1) {
     if (!ffn_batched_supported(d)) return bail(REMOE_E_UNSUPPORTED);
     const size_t P = d.K + d.S;
@@ -514,7 +518,7 @@ int remoe_decode_step(remoe_stack* s, const float* hin, float* hout, int32_t* id
   d.policy = s->policy;
   d.beta = s->beta;
 
-  CK(launch_route(d, hin, ids, gates, s->contrib, s->stream));
+  CK(launch_route(d, hin, ids, gates, s->contrib, 0, d.L, s->stream));
   s->kernel_launches += d.B > 1 ? 2 : 1;
   CK(cudaMemcpyAsync(s->host_block, s->dev_block, s->block_ints * sizeof(int), cudaMemcpyDeviceToHost, s->stream));
   CK(cudaEventRecord(s->ev_trace, s->stream));
@@ -595,8 +599,78 @@ int remoe_decode_step(remoe_stack* s, const float* hin, float* hout, int32_t* id
     }
   }
   if (s->profiling) s->ev_used[prof_slot].bytes = resident_bytes;
-  CK(launch_combine(a, hout, s->stream));
+  CK(launch_combine(a, hout, 0, d.L, nullptr, s->stream));
   s->kernel_launches += 1;
+  return REMOE_OK;
+}
+
+int remoe_decode_step_chained(remoe_stack* s, const float* hin, float* hout, float* layer_inputs, int32_t* ids,
+                              float* gates) {
+  if (!s || !hin || !hout || !ids || !gates) return REMOE_E_ARG;
+  if (!everything_loaded(s)) return REMOE_E_NOT_LOADED;
+  if (s->d.B != 1) return REMOE_E_UNSUPPORTED;
+  DevStack& d = s->d;
+  d.has_prev = s->steps_since_reset > 0 ? 1 : 0;
+  d.policy = s->policy;
+  d.beta = s->beta;
+  const size_t row = (size_t)d.H * sizeof(float);
+  CK(cudaMemcpyAsync(s->chain_in, hin, row, cudaMemcpyDeviceToDevice, s->stream));
+
+  FfnArgs a{};
+  a.d = d;
+  a.hidden_in = s->chain_in;
+  a.gates = gates;
+  a.partial = s->partial;
+  a.contrib = s->contrib;
+  a.grid_cap = s->grid;
+  uint32_t um = 0, tk = 0;
+  for (int l = 0; l < d.L; ++l) {
+    // The layer's input exists only once the previous layer is done, so every layer has its own
+    // route -> trace -> fetch -> compute round trip.
+    CK(launch_route(d, s->chain_in, ids, gates, s->contrib, l, 1, s->stream));
+    CK(cudaMemcpyAsync(s->host_block, s->dev_block, s->block_ints * sizeof(int), cudaMemcpyDeviceToHost, s->stream));
+    CK(cudaEventRecord(s->ev_trace, s->stream));
+    a.phase = 0;
+    a.layer = l;
+    CK(launch_ffn_stream(a, s->grid, s->stream));
+    s->kernel_launches += 2;
+    CK(cudaEventSynchronize(s->ev_trace));
+    if (check_device_flag(s) != REMOE_OK) return REMOE_E_DEVICE_FLAG;
+    int* tr = s->host_block + 1;
+    const int* t_req = trace_requests(tr, d.L, s->BK);
+    const int* t_hit = trace_hit(tr, d.L, s->BK);
+    const int* t_slot = trace_slot(tr, d.L, s->BK);
+    tk += (uint32_t)trace_tok_hits(tr, d.L, s->BK)[l];
+    int misses = 0;
+    for (int k = 0; k < d.K; ++k) {
+      const int i = l * s->BK + k;
+      if (t_hit[i]) continue;
+      const int e = t_req[i], slot = t_slot[i];
+      if (e < 0 || e >= d.N || slot < 0 || slot >= d.C) return REMOE_E_DEVICE_FLAG;
+      if (!misses) CK(cudaStreamWaitEvent(s->copy_stream, s->ev_trace, 0));
+      CK(cudaMemcpyAsync(d.slots + ((size_t)l * d.C + slot) * d.slot_bytes, s->host_ptrs[(size_t)l * d.N + e],
+                         d.slot_bytes, cudaMemcpyHostToDevice, s->copy_stream));
+      ++misses;
+    }
+    um += (uint32_t)misses;
+    if (misses) {
+      s->h2d_bytes[l] += (uint64_t)misses * d.slot_bytes;
+      CK(cudaEventRecord(s->ev_layer[l], s->copy_stream));
+      CK(cudaStreamWaitEvent(s->stream, s->ev_layer[l], 0));
+      a.phase = 1;
+      CK(launch_ffn_stream(a, s->grid, s->stream));
+      s->kernel_launches += 1;
+    }
+    CK(launch_combine(a, s->chain_out, l, 1, s->chain_in, s->stream));
+    s->kernel_launches += 1;
+  }
+  s->steps += 1;
+  s->steps_since_reset += 1;
+  s->hist_umiss.push_back(um);
+  s->hist_tok_hits.push_back(tk);
+  CK(cudaMemcpyAsync(hout, s->chain_in + (size_t)d.L * d.H, row, cudaMemcpyDeviceToDevice, s->stream));
+  if (layer_inputs)
+    CK(cudaMemcpyAsync(layer_inputs, s->chain_in, row * d.L, cudaMemcpyDeviceToDevice, s->stream));
   return REMOE_OK;
 }
 

@@ -122,10 +122,11 @@ __device__ __forceinline__ int pair_rows(const FfnArgs& a, int pair) {
   const DevStack& d = a.d;
   const int P = d.K + d.S;
   const int l = pair / P, p = pair % P;
+  if (a.layer >= 0 && l != a.layer) return 0;
   if (p >= d.K) return a.phase == 0 ? d.Is : 0;
   const int hit = trace_hit(d.trace, d.L, d.K)[l * d.K + p];
   if (a.phase == 0) return hit ? d.I : 0;
-  return (l == a.layer && !hit) ? d.I : 0;
+  return hit ? 0 : d.I;
 }
 
 template <int WB, int H>
@@ -183,7 +184,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(const __grid_co
 
   if (blockIdx.x == 0) {
     for (int l = tid; l < d.L; l += kThreads) {
-      if (a.phase != 0 && l != a.layer) continue;
+      if (a.layer >= 0 && l != a.layer) continue;
       const int lo = prefix[l * P], hi = prefix[(l + 1) * P];
       int* c = a.contrib + ((size_t)a.phase * d.L + l) * 2;
       if (hi > lo) { c[0] = lo / q; c[1] = (hi - 1) / q; } else { c[0] = 1; c[1] = 0; }
@@ -337,9 +338,10 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(const __grid_co
   }
 }
 
-__global__ void __launch_bounds__(256) combine_kernel(FfnArgs a, float* __restrict__ hidden_out) {
+__global__ void __launch_bounds__(256) combine_kernel(FfnArgs a, float* __restrict__ hidden_out, int layer0,
+                                                      float* __restrict__ chain_in) {
   const DevStack& d = a.d;
-  const int l = blockIdx.y;
+  const int l = layer0 + blockIdx.y;
   const int c = blockIdx.x * 256 + threadIdx.x;
   if (c >= d.H) return;
   float t = 0.f;
@@ -350,6 +352,7 @@ __global__ void __launch_bounds__(256) combine_kernel(FfnArgs a, float* __restri
     for (int b = lo; b <= hi; ++b) t += p[(size_t)b * d.H];
   }
   hidden_out[(size_t)l * d.H + c] = t;
+  if (chain_in) chain_in[(size_t)(l + 1) * d.H + c] = chain_in[(size_t)l * d.H + c] + t;
 }
 
 template <int WB, int H>
@@ -400,9 +403,10 @@ cudaError_t launch_ffn_stream(const FfnArgs& a, int grid, cudaStream_t st) {
   return cudaErrorInvalidValue;
 }
 
-cudaError_t launch_combine(const FfnArgs& a, float* hidden_out, cudaStream_t st) {
-  dim3 grid((a.d.H + 255) / 256, a.d.L);
-  combine_kernel<<<grid, 256, 0, st>>>(a, hidden_out);
+cudaError_t launch_combine(const FfnArgs& a, float* hidden_out, int layer0, int n_layers, float* chain_in,
+                           cudaStream_t st) {
+  dim3 grid((a.d.H + 255) / 256, n_layers);
+  combine_kernel<<<grid, 256, 0, st>>>(a, hidden_out, layer0, chain_in);
   return cudaGetLastError();
 }
 

@@ -77,8 +77,8 @@ struct FfnArgs {
   DevStack d;
   const float* hidden_in;              // [L][1][H]
   const float* gates;                  // [L][1][K]
-  int phase;                           // 0: resident (hits + shared), all layers; 1: misses of `layer`
-  int layer;
+  int phase;                           // 0: resident (hits + shared); 1: misses of `layer`
+  int layer;                           // phase 1: the layer; phase 0: -1 = all layers, else only this one
   float* partial;                      // [2][L][grid][H]
   int* contrib;                        // [2][L][2]  (first CTA, last CTA) contributing; first > last = none
   int grid_cap;                        // CTAs per phase the partial buffer is laid out for
@@ -103,10 +103,14 @@ bool ffn_batched_supported(const DevStack& d);
 cudaError_t launch_ffn_batched(const BatchArgs& a, int grid, cudaStream_t st);
 cudaError_t launch_combine_batched(const BatchArgs& a, float* hidden_out, cudaStream_t st);
 
+// Routes layers [layer0, layer0 + n_layers); `hidden_in`, `ids`, `gates` are the full [L, B, .] arrays.
 cudaError_t launch_route(const DevStack& d, const float* hidden_in, int* ids, float* gates,
-                         int* contrib, cudaStream_t st);
+                         int* contrib, int layer0, int n_layers, cudaStream_t st);
 cudaError_t launch_ffn_stream(const FfnArgs& a, int grid, cudaStream_t st);
-cudaError_t launch_combine(const FfnArgs& a, float* hidden_out, cudaStream_t st);
+// Adds the partials of layers [layer0, layer0 + n_layers) into hidden_out[L, 1, H]; with `chain_in`
+// ([L + 1, 1, H]) also writes chain_in[l + 1] = chain_in[l] + out[l] (residual chaining).
+cudaError_t launch_combine(const FfnArgs& a, float* hidden_out, int layer0, int n_layers, float* chain_in,
+                           cudaStream_t st);
 size_t ffn_stream_smem_bytes(int H, int wbytes, int* stages_out);
 bool ffn_stream_supported(int H, int wbytes);
 

@@ -236,13 +236,13 @@ __device__ void resolve_layer(const DevStack& d, int l, const int* flat, int n_f
 
 __global__ void __launch_bounds__(1024) route_kernel(DevStack d, const float* __restrict__ hidden_in,
                                                     int* __restrict__ ids, float* __restrict__ gates,
-                                                    int* contrib) {
+                                                    int* contrib, int layer0) {
   __shared__ float z[kMaxRouted];
   __shared__ int s_ids[32];
   __shared__ float s_g[32];
   __shared__ DirSmem dir;
 
-  const int lb = blockIdx.x;
+  const int lb = layer0 * d.B + blockIdx.x;
   const int l = lb / d.B;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const float* h = hidden_in + (size_t)lb * d.H;
@@ -344,10 +344,11 @@ __global__ void __launch_bounds__(1024) route_kernel(DevStack d, const float* __
   if (d.B == 1) resolve_layer(d, l, s_ids, d.K, dir, lane, contrib);
 }
 
-__global__ void __launch_bounds__(32) resolve_kernel(DevStack d, const int* __restrict__ ids, int* contrib) {
+__global__ void __launch_bounds__(32) resolve_kernel(DevStack d, const int* __restrict__ ids, int* contrib,
+                                                     int layer0) {
   __shared__ DirSmem dir;
   __shared__ int flat[kMaxRequests];
-  const int l = blockIdx.x, lane = threadIdx.x;
+  const int l = layer0 + blockIdx.x, lane = threadIdx.x;
   const int BK = d.B * d.K;
   for (int i = lane; i < BK; i += 32) flat[i] = ids[(size_t)l * BK + i];
   __syncwarp();
@@ -357,13 +358,13 @@ __global__ void __launch_bounds__(32) resolve_kernel(DevStack d, const int* __re
 }  // namespace
 
 cudaError_t launch_route(const DevStack& d, const float* hidden_in, int* ids, float* gates,
-                         int* contrib, cudaStream_t st) {
+                         int* contrib, int layer0, int n_layers, cudaStream_t st) {
   // few CTAs at batch 1: give each as many warps as it can hold so the router rows load in parallel
-  route_kernel<<<d.L * d.B, d.B == 1 ? 1024 : 256, 0, st>>>(d, hidden_in, ids, gates, contrib);
+  route_kernel<<<n_layers * d.B, d.B == 1 ? 1024 : 256, 0, st>>>(d, hidden_in, ids, gates, contrib, layer0);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   if (d.B > 1) {
-    resolve_kernel<<<d.L, 32, 0, st>>>(d, ids, contrib);
+    resolve_kernel<<<n_layers, 32, 0, st>>>(d, ids, contrib, layer0);
     e = cudaGetLastError();
   }
   return e;

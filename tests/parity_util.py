@@ -106,6 +106,42 @@ class StepChecker:
                 assert e <= tol, f"layer {l}: output error {e} > {tol}"
         return r, (ids, g, out)
 
+    def step_chained(self, h0):
+        """One chained step (h_{l+1} = h_l + MoE_l(h_l)) on both sides.  A near-tie at one layer
+        changes the inputs of the layers below it, so the oracle is first run on a copy to find
+        such positions, then for real with the library's ids forced there."""
+        import copy
+        t = self.torch
+        L, H, K = self.L, self.H, self.K
+        d_h0 = t.from_numpy(np.ascontiguousarray(h0, dtype=np.float32).reshape(H)).to(self.d_in.device)
+        d_fin = t.empty(H, dtype=t.float32, device=d_h0.device)
+        d_lin = t.empty((L, H), dtype=t.float32, device=d_h0.device)
+        self.wl.stack.decode_step_chained(d_h0, d_fin, d_lin, self.d_ids, self.d_g)
+        t.cuda.synchronize()
+        ids = self.d_ids.cpu().numpy()
+        override = {}
+        for _ in range(L + 1):
+            trial = copy.deepcopy(self.o).step(np.asarray(h0).reshape(1, H), ffn="selected", chained=True,
+                                               id_override=override or None)
+            bad = [l for l in range(L) if list(trial["ids"][l, 0]) != list(ids[l, 0])]
+            if not bad:
+                break
+            l = bad[0]
+            assert trial["margin"][l, 0] < NEAR_TIE, f"chained ids differ at layer {l}, margin {trial['margin'][l, 0]}"
+            self.near_ties += 1
+            override[(l, 0)] = [int(e) for e in ids[l, 0]]
+        r = self.o.step(np.asarray(h0).reshape(1, H), ffn="selected", chained=True, id_override=override or None)
+        assert np.array_equal(r["ids"], ids)
+        tol = TOL[self.wl.shape.weight_dtype]
+        e_fin = rel_err(d_fin.cpu().numpy(), r["final"][0])
+        e_lin = rel_err(d_lin.cpu().numpy(), r["layer_inputs"][:, 0])
+        self.max_out_err = max(self.max_out_err, e_fin, e_lin)
+        assert e_fin <= tol and e_lin <= tol, (e_fin, e_lin)
+        tr = self.wl.stack.last_step_trace()
+        l = L - 1                                   # the trace block holds the last layer's round trip
+        assert list(tr["requests"][l][:K]) == r["requests"][l] and list(tr["slot"][l][:K]) == r["slot"][l]
+        return r
+
     def check_counters(self):
         st = self.wl.stack
         o = self.o

@@ -55,6 +55,16 @@ def test_small_shapes(shape, c, rho):
     _run(shape, c, rho, steps=24, seed=1, dense_steps=2, host_api_every=7)
 
 
+@pytest.mark.parametrize("shape,c,rho", [
+    (synth.Shape(2, 256, 256, 32, 8, 0, 0, 0, 1, 1, 1), 40, 0.5),       # largest N and K the kernels take
+    (synth.Shape(2, 256, 256, 32, 8, 0, 0, 0, 0, 0, 1), 256, 0.5),      # ... with every expert resident
+    (synth.Shape(1, 128, 4, 1, 1, 1, 1, 0, 0, 0, 1), 1, 0.2),           # one channel per expert, K = C = 1
+    (synth.Shape(40, 256, 8, 2, 8, 3, 8, 1, 0, 1, 1), 2, 0.9),          # more layers than CTAs get rows
+])
+def test_extreme_shapes(shape, c, rho):
+    _run(shape, c, rho, steps=10, seed=7, dense_steps=1)
+
+
 def test_many_layers_span_ctas():
     """Enough rows that CTAs cross expert and layer boundaries in the streaming kernel."""
     shape = synth.Shape(12, 512, 16, 4, 300, 1, 300, 0, 0, 1, 1)
@@ -114,6 +124,27 @@ def test_reset_and_errors():
         chk.o.reset()
         for t in range(10):
             chk.step(hs[t])
+        chk.check_counters()
+    finally:
+        wl.close()
+
+
+@pytest.mark.parametrize("shape,c", [
+    (synth.Shape(6, 512, 24, 3, 64, 1, 32, 1, 0, 1, 1), 6),
+    (synth.Shape(4, 256, 16, 2, 40, 0, 0, 0, 1, 0, 1), 4),
+])
+def test_chained_stack(shape, c):
+    """Layers feeding each other through the residual: routing of layer l+1 sees layer l's output."""
+    import torch
+    from paper_2605_27081_b200.loader import LoadedWorkload
+    from parity_util import StepChecker, oracle_for
+
+    wl = LoadedWorkload(shape, c, seed=8)
+    try:
+        chk = StepChecker(wl, oracle_for(wl), torch)
+        hs = synth.HiddenStream(8, synth.Shape(**{**shape.asdict(), "n_layers": 1}), 0.8)
+        for t in range(12):
+            chk.step_chained(hs.step()[0, 0])
         chk.check_counters()
     finally:
         wl.close()

@@ -224,3 +224,32 @@ def test_synth_is_reproducible_and_layout():
     long = synth.HiddenStream(6, synth.Shape(1, 4096, 4, 2, 6), 0.9).take(200)[:, 0, 0]
     c = np.mean(long[1:] * long[:-1]) / np.mean(long * long)
     assert abs(c - 0.9) < 0.02 and abs(long.std() - 1.0) < 0.05
+
+
+def test_chained_mode_identities():
+    """h_{l+1} = h_l + MoE_l(h_l): telescoping sum, agreement with one-layer stacks run by hand, and
+    the zero-weight case where every layer sees h_0."""
+    shape = synth.Shape(3, 64, 8, 2, 8, 1, 8)
+    st = _stack(shape, 3, seed=9, with_ffn=True)
+    h0 = np.random.default_rng(9).standard_normal((1, 64))
+    r = st.step(h0, ffn="dense", chained=True)
+    assert np.allclose(r["final"] - h0, r["out"].sum(axis=0), rtol=1e-13, atol=1e-13)
+    for l in range(2):
+        assert np.allclose(r["layer_inputs"][l + 1] - r["layer_inputs"][l], r["out"][l], rtol=1e-13, atol=1e-13)
+    assert np.array_equal(r["layer_inputs"][0], h0)
+    cur = h0.copy()
+    for l in range(3):
+        one = orc.OracleStack(synth.Shape(1, 64, 8, 2, 8, 1, 8), 3, [st.routers[l]],
+                              lambda _l, e, l=l: st.expert_weights(l, e), lambda _l, i, l=l: st.shared_weights(l, i))
+        r1 = one.step(cur[None], ffn="selected")
+        assert np.array_equal(r1["ids"][0], r["ids"][l])
+        assert np.allclose(r1["out"][0], r["out"][l], rtol=1e-13, atol=1e-13)
+        cur = cur + r1["out"][0]
+    assert np.allclose(cur, r["final"], rtol=1e-13, atol=1e-13)
+
+    zero = (np.zeros((8, 64)), np.zeros((8, 64)), np.zeros((64, 8)))
+    stz = orc.OracleStack(shape, 3, st.routers, lambda l, e: zero, lambda l, i: zero)
+    rz = stz.step(h0, ffn="selected", chained=True)
+    assert np.array_equal(rz["final"], h0) and all(np.array_equal(x, h0) for x in rz["layer_inputs"])
+    plain = orc.OracleStack(shape, 3, st.routers).step(np.repeat(h0[None], 3, axis=0), ffn=None)
+    assert np.array_equal(plain["ids"], rz["ids"])
