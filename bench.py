@@ -323,6 +323,33 @@ def run_ours(args, rank, world, local_rank):
         resident = r
         wl_r.stack.close()
 
+    # Chained variant (layers joined by a residual): same stack, one route/fetch round trip per layer.
+    chained = None
+    if shape.batch == 1 and not args.no_chained and rank == 0:
+        n = min(args.steps, 128)
+        hid = torch.from_numpy(synth.HiddenStream(seed, shape, args.rho).take(args.warmup + n)[:, 0, 0].copy()).to("cuda")
+        d_fin = torch.empty(shape.hidden, dtype=torch.float32, device="cuda")
+        d_ids = torch.empty((shape.n_layers, 1, shape.top_k), dtype=torch.int32, device="cuda")
+        d_g = torch.empty((shape.n_layers, 1, shape.top_k), dtype=torch.float32, device="cuda")
+        wl.stack.cache_reset()
+        torch.cuda.synchronize()
+        with torch.cuda.stream(stream):
+            for t in range(args.warmup):
+                wl.stack.decode_step_chained(hid[t], d_fin, None, d_ids, d_g)
+            c0 = wl.stack.cache_stats()
+            ea, eb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            ea.record(stream)
+            for t in range(args.warmup, args.warmup + n):
+                wl.stack.decode_step_chained(hid[t], d_fin, None, d_ids, d_g)
+            eb.record(stream)
+            torch.cuda.synchronize()
+        c1 = wl.stack.cache_stats()
+        ms_c = ea.elapsed_time(eb)
+        chained = {"tokens_per_s": n / (ms_c / 1e3), "ms_per_step": ms_c / n,
+                   "misses_per_step": (c1["uniq_misses"] - c0["uniq_misses"]) / n,
+                   "h2d_achieved_gbs": (c1["h2d_bytes"] - c0["h2d_bytes"]) / (ms_c / 1e3) / 1e9}
+
     head = results[args.rho]
     red = reduce_over_ranks(dist, {"ms": head["ms"], "e2e_ms": head["e2e_ms"]}, {"launches": head["launches"]},
                             "cuda")
@@ -409,6 +436,8 @@ def run_ours(args, rank, world, local_rank):
             "kernel_gbs": b_r / (ms_r / 1e3) / 1e9 if ms_r > 0 else 0.0,
             "kernel_frac_of_measured": (b_r / (ms_r / 1e3) / 1e9 / peak_hbm) if ms_r > 0 else 0.0,
             "step_frac_of_hbm_roofline": step_roofline(resident, n)["frac"]}
+    if chained is not None:
+        line["chained"] = chained
     print(json.dumps(line), flush=True)
     wl.close()
     if dist is not None:
@@ -427,6 +456,7 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="use only this many layers (profiling captures)")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-resident", action="store_true")
+    ap.add_argument("--no-chained", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.warmup < 3:
