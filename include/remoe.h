@@ -46,7 +46,7 @@ enum {
   REMOE_E_NOMEM = -8         /* host or device allocation failed                          */
 };
 
-enum { REMOE_F32 = 0, REMOE_BF16 = 1 };
+enum { REMOE_F32 = 0, REMOE_BF16 = 1, REMOE_FP8_E4M3 = 2 };
 enum { REMOE_POLICY_LRU = 0, REMOE_POLICY_FIFO = 1, REMOE_POLICY_LFU = 2 };
 
 /* Shape of the stack.  Sec. 3.1: N_r routed experts, Top-K; shared experts always active. */
@@ -60,7 +60,10 @@ typedef struct {
   int32_t inter_shared;  /* I of each shared expert                                        */
   int32_t shared_gate;   /* 1: shared output is scaled by sigmoid(w_sg . h)                */
   int32_t renorm_topk;   /* 1: top-K gate weights are renormalised to sum to 1             */
-  int32_t weight_dtype;  /* REMOE_F32 or REMOE_BF16 (router, shared gate, all experts)     */
+  int32_t weight_dtype;  /* REMOE_F32, REMOE_BF16 (router, shared gate, all experts) or    */
+                         /* REMOE_FP8_E4M3: expert blocks are OCP FP8 E4M3 bytes, value =  */
+                         /* byte * 2^-8; router and shared gate bf16; H multiple of 512;   */
+                         /* batch 1 only (halves the bytes a miss moves over the host link)*/
   int32_t batch;         /* B sequences per step                                           */
 } remoe_shape;
 
@@ -119,12 +122,13 @@ int remoe_decode_step(remoe_stack*, const float* hidden_in_dev, float* hidden_ou
                       int32_t* selected_ids_dev, float* gate_weights_dev);
 
 /*
- * Chained variant of the step (batch 1): the layers feed each other through a residual
- * connection, h_{l+1} = h_l + MoE_l(h_l), as in a decoder stack, instead of each reading its own
- * stream (the paper treats layers independently, App. A.5; chaining is how they sit in a model).
+ * Chained variant of the step (batch 1): the layers feed each other through a pre-norm residual
+ * connection as in a decoder stack, x_l = h_l / sqrt(mean(h_l^2) + 1e-6), h_{l+1} = h_l + MoE_l(x_l),
+ * instead of each reading its own stream (the paper treats layers independently, App. A.5;
+ * chaining is how they sit in a model; without the norm a randomly initialised stack diverges).
  *   hidden_in    dev [H]        h_0
  *   hidden_out   dev [H]        h_L
- *   layer_inputs dev [L, H]     h_0 .. h_{L-1} (may be NULL)
+ *   layer_inputs dev [L, H]     residual stream h_0 .. h_{L-1} (may be NULL)
  *   selected_ids dev [L, K], gate_weights dev [L, K]
  * Routing of layer l+1 depends on layer l's output, so the host waits for one small trace per
  * layer instead of one per step, and a layer's fetches cannot start before the layer above it
@@ -242,7 +246,8 @@ int remoe_expert_ffn_static(int32_t hidden, int32_t weight_dtype, int32_t n_expe
                             const float* scales, const float* hidden_in_dev, float* hidden_out_dev,
                             void* cuda_stream);
 
-/* Text of the last CUDA runtime error seen by this stack ("" if none). */
+/* Text of the last CUDA runtime error, or of the last device-flag / trace-validation failure,
+ * seen by this stack ("" if none). */
 const char* remoe_last_cuda_error(const remoe_stack*);
 
 void remoe_stack_destroy(remoe_stack*);

@@ -337,9 +337,10 @@ class OracleStack:
         """Advance every layer by one token.  h: [L, B, H].
 
         chained=True: h is [B, H], the input of layer 0, and the layers feed each other through
-        a residual connection, h_{l+1} = h_l + MoE_l(h_l) (how MoE layers sit in a decoder; the
-        paper's analysis treats each layer on its own).  The result then also carries
-        "layer_inputs" [L, B, H] and "final" [B, H]; `ffn` must not be None.
+        a pre-norm residual connection, x_l = h_l / sqrt(mean(h_l^2) + 1e-6) and
+        h_{l+1} = h_l + MoE_l(x_l) (how MoE layers sit in a decoder; the paper's analysis treats
+        each layer on its own).  The result then also carries "layer_inputs" [L, B, H] (the
+        residual stream h_l) and "final" [B, H]; `ffn` must not be None.
 
         ffn: "dense", "selected" or None (integer parts only).  `ffn_layers` restricts the
         floating-point FFN to some layers.  `id_override[(l, b)]` forces the selected ids
@@ -360,9 +361,11 @@ class OracleStack:
             cur = np.asarray(h, dtype=F64).reshape(B, s.hidden).copy()
             res["layer_inputs"] = np.zeros((L, B, s.hidden), F64)
         for l in range(L):
-            hl = cur if chained else h[l]
             if chained:
                 res["layer_inputs"][l] = cur
+                hl = cur / np.sqrt(np.mean(cur * cur, axis=1, keepdims=True) + 1e-6)
+            else:
+                hl = h[l]
             flat = []
             for b in range(B):
                 ov = None if id_override is None else id_override.get((l, b))

@@ -44,7 +44,8 @@ struct remoe_stack {
   size_t block_ints = 0;
   float* partial = nullptr;
   int* contrib = nullptr;
-  float* chain_in = nullptr;               // [L + 1][H] layer inputs of the chained mode
+  float* chain_in = nullptr;               // [L + 1][H] residual stream h_l of the chained mode
+  float* chain_x = nullptr;                // [L][H] normalised layer inputs x_l = rmsnorm(h_l)
   float* chain_out = nullptr;              // [L][H] per-layer MoE outputs of the chained mode
   cudaEvent_t ev_trace = nullptr;
   std::vector<cudaEvent_t> ev_layer;
@@ -184,7 +185,14 @@ int prof_collect(remoe_stack* s) {
 }
 
 int check_device_flag(remoe_stack* s) {
-  return s->host_block[0] != kErrNone ? REMOE_E_DEVICE_FLAG : REMOE_OK;
+  if (s->host_block[0] == kErrNone) return REMOE_OK;
+  static const char* names[] = {"none", "a consumer's bounded wait for a weight row ran out",
+                                "the producer's bounded wait for a free stage ran out",
+                                "an expert id or slot index was out of range",
+                                "copies were still in flight when a kernel bailed out"};
+  const int c = s->host_block[0];
+  s->cuda_err = std::string("device flag ") + std::to_string(c) + ": " + (c >= 1 && c <= 4 ? names[c] : "unknown");
+  return REMOE_E_DEVICE_FLAG;
 }
 
 // One decode step for B > 1.  The step's distinct requests may outnumber the slots, so a slot
@@ -366,10 +374,11 @@ int remoe_stack_create(const remoe_shape* sh, int32_t cache_slots, void* cuda_st
   *out = nullptr;
   if (sh->n_layers < 1 || sh->hidden < 1 || sh->n_routed < 1 || sh->top_k < 1 || sh->inter_routed < 1 ||
       sh->batch < 1 || sh->n_shared < 0 || cache_slots < 1 || sh->top_k > sh->n_routed ||
-      (sh->n_shared > 0 && sh->inter_shared < 1) || (sh->weight_dtype != REMOE_F32 && sh->weight_dtype != REMOE_BF16))
+      (sh->n_shared > 0 && sh->inter_shared < 1) || (sh->weight_dtype != REMOE_F32 && sh->weight_dtype != REMOE_BF16 && sh->weight_dtype != REMOE_FP8_E4M3))
     return REMOE_E_ARG;
   if (sh->batch == 1 && cache_slots < sh->top_k) return REMOE_E_CAPACITY;
-  const int wbytes = sh->weight_dtype == REMOE_BF16 ? 2 : 4;
+  const int wbytes = sh->weight_dtype == REMOE_BF16 ? 2 : (sh->weight_dtype == REMOE_FP8_E4M3 ? 1 : 4);
+  const int rbytes = sh->weight_dtype == REMOE_F32 ? 4 : 2;
   const long pairs = (long)sh->n_layers * (sh->top_k + sh->n_shared);
   if (sh->n_routed > kMaxRouted || sh->top_k > 32 || cache_slots > kMaxSlots || cache_slots > sh->n_routed ||
       (long)sh->batch * sh->top_k > kMaxRequests || !ffn_stream_supported(sh->hidden, wbytes))
@@ -401,15 +410,15 @@ int remoe_stack_create(const remoe_shape* sh, int32_t cache_slots, void* cuda_st
   DevStack& d = s->d;
   d.L = sh->n_layers; d.H = sh->hidden; d.N = sh->n_routed; d.K = sh->top_k; d.I = sh->inter_routed;
   d.S = sh->n_shared; d.Is = sh->n_shared ? sh->inter_shared : 0; d.B = sh->batch; d.C = cache_slots;
-  d.shared_gate = sh->shared_gate ? 1 : 0; d.renorm = sh->renorm_topk ? 1 : 0; d.wbytes = wbytes;
+  d.shared_gate = sh->shared_gate ? 1 : 0; d.renorm = sh->renorm_topk ? 1 : 0; d.wbytes = wbytes; d.rbytes = rbytes;
   d.policy = REMOE_POLICY_LRU; d.beta = 0.f; d.has_prev = 0;
   d.slot_bytes = (size_t)3 * d.I * d.H * wbytes;
   d.shared_bytes = (size_t)3 * d.Is * d.H * wbytes;
   const size_t L = d.L;
   char *router = nullptr, *sgw = nullptr, *shared = nullptr, *slots = nullptr;
 #define TRY(x) do { rc = (x); if (rc != REMOE_OK) return bail(rc); } while (0)
-  TRY(dev_alloc(s, &router, L * d.N * d.H * wbytes));
-  TRY(dev_alloc(s, &sgw, L * d.H * wbytes));
+  TRY(dev_alloc(s, &router, L * d.N * d.H * rbytes));
+  TRY(dev_alloc(s, &sgw, L * d.H * rbytes));
   TRY(dev_alloc(s, &shared, L * d.S * d.shared_bytes));
   TRY(dev_alloc(s, &slots, L * d.C * d.slot_bytes));
   d.router = router; d.shared_gate_w = sgw; d.shared_blocks = shared; d.slots = slots;
@@ -434,6 +443,7 @@ int remoe_stack_create(const remoe_shape* sh, int32_t cache_slots, void* cuda_st
   TRY(dev_alloc(s, &s->contrib, (size_t)2 * L * 2));
   TRY(dev_alloc(s, &s->chain_in, (L + 1) * d.B * d.H));
   TRY(dev_alloc(s, &s->chain_out, L * d.B * d.H));
+  TRY(dev_alloc(s, &s->chain_x, L * d.B * d.H));
   if (d.B > 1) {
     if (!ffn_batched_supported(d)) return bail(REMOE_E_UNSUPPORTED);
     const size_t P = d.K + d.S;
@@ -470,7 +480,7 @@ int remoe_stack_create(const remoe_shape* sh, int32_t cache_slots, void* cuda_st
 int remoe_load_router(remoe_stack* s, int32_t layer, const void* w, const void* wsg) {
   if (!s || !w || layer < 0 || layer >= s->d.L) return REMOE_E_ARG;
   if (s->d.shared_gate && !wsg) return REMOE_E_ARG;
-  const size_t row = (size_t)s->d.H * s->d.wbytes;
+  const size_t row = (size_t)s->d.H * s->d.rbytes;
   CK(cudaMemcpyAsync(const_cast<char*>(s->d.router) + (size_t)layer * s->d.N * row, w, s->d.N * row,
                      cudaMemcpyHostToDevice, s->stream));
   if (s->d.shared_gate)
@@ -572,7 +582,10 @@ int remoe_decode_step(remoe_stack* s, const float* hin, float* hout, int32_t* id
       const int i = l * s->BK + k;
       if (t_hit[i]) { resident_bytes += d.slot_bytes; continue; }
       const int e = t_req[i], slot = t_slot[i];
-      if (e < 0 || e >= d.N || slot < 0 || slot >= d.C) return REMOE_E_DEVICE_FLAG;
+      if (e < 0 || e >= d.N || slot < 0 || slot >= d.C) {
+        s->cuda_err = "trace holds an expert id or slot out of range (layer " + std::to_string(l) + ")";
+        return REMOE_E_DEVICE_FLAG;
+      }
       if (!copy_ordered) {
         // Victim slots may still be read by the previous step's kernels, all of which precede
         // this step's route kernel on the compute stream.
@@ -618,7 +631,7 @@ int remoe_decode_step_chained(remoe_stack* s, const float* hin, float* hout, flo
 
   FfnArgs a{};
   a.d = d;
-  a.hidden_in = s->chain_in;
+  a.hidden_in = s->chain_x;
   a.gates = gates;
   a.partial = s->partial;
   a.contrib = s->contrib;
@@ -626,8 +639,10 @@ int remoe_decode_step_chained(remoe_stack* s, const float* hin, float* hout, flo
   uint32_t um = 0, tk = 0;
   for (int l = 0; l < d.L; ++l) {
     // The layer's input exists only once the previous layer is done, so every layer has its own
-    // route -> trace -> fetch -> compute round trip.
-    CK(launch_route(d, s->chain_in, ids, gates, s->contrib, l, 1, s->stream));
+    // norm -> route -> trace -> fetch -> compute round trip.
+    CK(launch_rmsnorm(s->chain_in + (size_t)l * d.H, s->chain_x + (size_t)l * d.H, d.H, s->stream));
+    CK(launch_route(d, s->chain_x, ids, gates, s->contrib, l, 1, s->stream));
+    s->kernel_launches += 1;
     CK(cudaMemcpyAsync(s->host_block, s->dev_block, s->block_ints * sizeof(int), cudaMemcpyDeviceToHost, s->stream));
     CK(cudaEventRecord(s->ev_trace, s->stream));
     a.phase = 0;
@@ -646,7 +661,10 @@ int remoe_decode_step_chained(remoe_stack* s, const float* hin, float* hout, flo
       const int i = l * s->BK + k;
       if (t_hit[i]) continue;
       const int e = t_req[i], slot = t_slot[i];
-      if (e < 0 || e >= d.N || slot < 0 || slot >= d.C) return REMOE_E_DEVICE_FLAG;
+      if (e < 0 || e >= d.N || slot < 0 || slot >= d.C) {
+        s->cuda_err = "trace holds an expert id or slot out of range (layer " + std::to_string(l) + ")";
+        return REMOE_E_DEVICE_FLAG;
+      }
       if (!misses) CK(cudaStreamWaitEvent(s->copy_stream, s->ev_trace, 0));
       CK(cudaMemcpyAsync(d.slots + ((size_t)l * d.C + slot) * d.slot_bytes, s->host_ptrs[(size_t)l * d.N + e],
                          d.slot_bytes, cudaMemcpyHostToDevice, s->copy_stream));

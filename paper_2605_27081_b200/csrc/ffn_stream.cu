@@ -21,6 +21,8 @@
 // atomics are used.  HBM traffic is the weight bytes once plus O(grid * H) partials.
 #include "remoe_internal.cuh"
 
+#include <cuda_fp16.h>
+
 namespace remoe {
 
 namespace {
@@ -91,6 +93,31 @@ struct Elems<2> {
     f[6] = __uint_as_float(v.w << 16); f[7] = __uint_as_float(v.w & 0xffff0000u);
   }
 };
+
+// FP8 E4M3 expert blocks: sixteen values per 16 bytes; a stored byte q stands for q * 2^-8 (the
+// stack-wide power-of-two scale is applied to the dot products, not per element).
+template <>
+struct Elems<1> {
+  static constexpr int kVec = 16;
+  __device__ static __forceinline__ void pair(uint32_t two_bytes, float& lo, float& hi) {
+    uint32_t h2;
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"((unsigned short)two_bytes));
+    const __half2 v = *reinterpret_cast<const __half2*>(&h2);
+    lo = __low2float(v);
+    hi = __high2float(v);
+  }
+  __device__ static __forceinline__ void load(const char* p, float* f) {
+    const uint4 v = *reinterpret_cast<const uint4*>(p);
+    pair(v.x & 0xffffu, f[0], f[1]);   pair(v.x >> 16, f[2], f[3]);
+    pair(v.y & 0xffffu, f[4], f[5]);   pair(v.y >> 16, f[6], f[7]);
+    pair(v.z & 0xffffu, f[8], f[9]);   pair(v.z >> 16, f[10], f[11]);
+    pair(v.w & 0xffffu, f[12], f[13]); pair(v.w >> 16, f[14], f[15]);
+  }
+};
+template <int WB>
+struct WScale { static constexpr float value = 1.f; };
+template <>
+struct WScale<1> { static constexpr float value = 1.f / 256.f; };
 
 // Shared-memory carve-up (dynamic): barriers | row prefix table | reduce buffer | stage ring.
 // The ring depth is a multiple of the consumer-warp count, so a stage is always consumed by
@@ -301,7 +328,9 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(const __grid_co
           g += __shfl_xor_sync(kFull, g, o);
           u += __shfl_xor_sync(kFull, u, o);
         }
-        const float av = g / (1.f + __expf(-g)) * u * scale;
+        g *= WScale<WB>::value;
+        u *= WScale<WB>::value;
+        const float av = g / (1.f + __expf(-g)) * u * (scale * WScale<WB>::value);
 #pragma unroll
         for (int it = 0; it < kIter; ++it) {
           float w[kVec];
@@ -326,11 +355,11 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(const __grid_co
               make_float4(acc[it * kVec + v4 * 4], acc[it * kVec + v4 * 4 + 1], acc[it * kVec + v4 * 4 + 2],
                           acc[it * kVec + v4 * 4 + 3]);
         consumer_bar();
-        if (tid < kPassCols) {
+        for (int c = tid; c < kPassCols; c += kConsumerWarps * 32) {
           float t = 0.f;
 #pragma unroll
-          for (int w = 0; w < kConsumerWarps; ++w) t += red[(size_t)w * kPassCols + tid];
-          dst[it * kPassCols + tid] = t;
+          for (int w = 0; w < kConsumerWarps; ++w) t += red[(size_t)w * kPassCols + c];
+          dst[it * kPassCols + c] = t;
         }
         consumer_bar();
       }
@@ -355,6 +384,25 @@ __global__ void __launch_bounds__(256) combine_kernel(FfnArgs a, float* __restri
   if (chain_in) chain_in[(size_t)(l + 1) * d.H + c] = chain_in[(size_t)l * d.H + c] + t;
 }
 
+__global__ void __launch_bounds__(256) rmsnorm_kernel(const float* __restrict__ h, float* __restrict__ x, int H) {
+  __shared__ float warp_ss[8];
+  __shared__ float s_scale;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  float ss = 0.f;
+  for (int c = tid; c < H; c += 256) ss = fmaf(h[c], h[c], ss);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(kFull, ss, o);
+  if (lane == 0) warp_ss[warp] = ss;
+  __syncthreads();
+  if (tid == 0) {
+    float t = 0.f;
+    for (int w = 0; w < 8; ++w) t += warp_ss[w];
+    s_scale = rsqrtf(t / (float)H + 1e-6f);
+  }
+  __syncthreads();
+  for (int c = tid; c < H; c += 256) x[c] = h[c] * s_scale;
+}
+
 template <int WB, int H>
 cudaError_t launch_one(const FfnArgs& a, int grid, cudaStream_t st) {
   const Layout lay = make_layout(H, WB);
@@ -374,6 +422,7 @@ cudaError_t launch_one(const FfnArgs& a, int grid, cudaStream_t st) {
 bool ffn_stream_supported(int H, int wbytes) {
   if (wbytes == 4) return H == 128 || H == 256 || H == 512 || H == 1024;
   if (wbytes == 2) return H == 256 || H == 512 || H == 1024 || H == 2048;
+  if (wbytes == 1) return H == 512 || H == 1024 || H == 2048;
   return false;
 }
 
@@ -392,15 +441,26 @@ cudaError_t launch_ffn_stream(const FfnArgs& a, int grid, cudaStream_t st) {
       case 512: return launch_one<4, 512>(a, grid, st);
       case 1024: return launch_one<4, 1024>(a, grid, st);
     }
-  } else {
+  } else if (a.d.wbytes == 2) {
     switch (H) {
       case 256: return launch_one<2, 256>(a, grid, st);
       case 512: return launch_one<2, 512>(a, grid, st);
       case 1024: return launch_one<2, 1024>(a, grid, st);
       case 2048: return launch_one<2, 2048>(a, grid, st);
     }
+  } else {
+    switch (H) {
+      case 512: return launch_one<1, 512>(a, grid, st);
+      case 1024: return launch_one<1, 1024>(a, grid, st);
+      case 2048: return launch_one<1, 2048>(a, grid, st);
+    }
   }
   return cudaErrorInvalidValue;
+}
+
+cudaError_t launch_rmsnorm(const float* h, float* x, int H, cudaStream_t st) {
+  rmsnorm_kernel<<<1, 256, 0, st>>>(h, x, H);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_combine(const FfnArgs& a, float* hidden_out, int layer0, int n_layers, float* chain_in,

@@ -27,7 +27,8 @@ enum : int {
 // Everything the kernels need, passed by value.
 struct DevStack {
   int L, H, N, K, I, S, Is, B, C;
-  int shared_gate, renorm, wbytes;     // wbytes: 4 (float32) or 2 (bfloat16)
+  int shared_gate, renorm, wbytes;     // wbytes: bytes per expert-block element: 4 float32, 2 bfloat16, 1 fp8 e4m3
+  int rbytes;                          // bytes per router / shared-gate element: 4 or 2
   int policy;
   float beta;
   int has_prev;                        // 0 on the first step after a reset
@@ -111,6 +112,8 @@ cudaError_t launch_ffn_stream(const FfnArgs& a, int grid, cudaStream_t st);
 // ([L + 1, 1, H]) also writes chain_in[l + 1] = chain_in[l] + out[l] (residual chaining).
 cudaError_t launch_combine(const FfnArgs& a, float* hidden_out, int layer0, int n_layers, float* chain_in,
                            cudaStream_t st);
+// x = h / sqrt(mean(h^2) + 1e-6) for one [H] vector (pre-norm of the chained mode), fixed summation order.
+cudaError_t launch_rmsnorm(const float* h, float* x, int H, cudaStream_t st);
 size_t ffn_stream_smem_bytes(int H, int wbytes, int* stages_out);
 bool ffn_stream_supported(int H, int wbytes);
 

@@ -246,17 +246,17 @@ __global__ void __launch_bounds__(1024) route_kernel(DevStack d, const float* __
   const int l = lb / d.B;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const float* h = hidden_in + (size_t)lb * d.H;
-  const size_t row_bytes = (size_t)d.H * d.wbytes;
+  const size_t row_bytes = (size_t)d.H * d.rbytes;
 
   const int n_warps = blockDim.x >> 5;
   for (int e = warp; e < d.N; e += n_warps) {
-    const float acc = row_dot(d.router + ((size_t)l * d.N + e) * row_bytes, h, d.H, d.wbytes, lane);
+    const float acc = row_dot(d.router + ((size_t)l * d.N + e) * row_bytes, h, d.H, d.rbytes, lane);
     if (lane == 0) z[e] = acc;
   }
   if (warp == n_warps - 1) {
     float sc = 1.f;
     if (d.shared_gate) {
-      const float dot = row_dot(d.shared_gate_w + (size_t)l * row_bytes, h, d.H, d.wbytes, lane);
+      const float dot = row_dot(d.shared_gate_w + (size_t)l * row_bytes, h, d.H, d.rbytes, lane);
       sc = 1.f / (1.f + expf(-dot));
     }
     if (lane == 0) d.shared_scale[lb] = sc;

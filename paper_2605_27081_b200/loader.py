@@ -28,7 +28,7 @@ class LoadedWorkload:
         nd = N if distinct_experts is None else min(N, int(distinct_experts))
         self.n_distinct = nd
         elems = synth.expert_block_elems(shape.hidden, shape.inter_routed)
-        np_dt = np.uint16 if shape.weight_dtype == 1 else np.float32
+        np_dt = {0: np.float32, 1: np.uint16, 2: np.uint8}[shape.weight_dtype]
         gen_shape = synth.Shape(**{**shape.asdict(), "n_routed": nd})
         self._store_t = torch.empty(L * nd * elems * shape.elem_bytes, dtype=torch.uint8, pin_memory=True)
         self.store = self._store_t.numpy().view(np_dt).reshape(L, nd, elems)

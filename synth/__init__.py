@@ -14,6 +14,10 @@ from .workloads import (  # noqa: F401
     expert_block_bytes,
     bf16_round_to_bits,
     bf16_bits_to_f32,
+    fp8_e4m3_round_to_bits,
+    fp8_e4m3_bits_to_f32,
+    widen,
+    FP8_SHIFT,
     gen_router,
     gen_shared_gate,
     gen_expert_block,

@@ -15,7 +15,10 @@ Storage conventions produced here (they are data layouts, not arithmetic):
 * hidden states       ``[L, B, H]`` float32 per decode step.
 
 Element type is float32 (``weight_dtype == 0``) or bfloat16 stored as ``uint16`` bit
-patterns (``weight_dtype == 1``), rounded to nearest-even once, at generation.
+patterns (``weight_dtype == 1``), rounded to nearest-even once, at generation.  With
+``weight_dtype == 2`` the expert blocks are OCP FP8 E4M3 bytes whose value is
+``decode(byte) * 2**-FP8_SHIFT`` (a fixed power-of-two scale that puts N(0, 0.02^2) weights in
+the format's normal range) while the router and shared-gate weights stay bfloat16.
 """
 from __future__ import annotations
 
@@ -33,6 +36,7 @@ KIND_HIDDEN = 5
 KIND_RHO = 6
 
 EXPERT_STD = 0.02
+FP8_SHIFT = 8
 
 
 @dataclass(frozen=True)
@@ -54,7 +58,13 @@ class Shape:
 
     @property
     def elem_bytes(self) -> int:
-        return 2 if self.weight_dtype == 1 else 4
+        """Bytes per element of an expert block."""
+        return {0: 4, 1: 2, 2: 1}[self.weight_dtype]
+
+    @property
+    def router_dtype(self) -> int:
+        """Element type of router and shared-gate weights (fp8 stacks keep them in bf16)."""
+        return 0 if self.weight_dtype == 0 else 1
 
 
 # The five workloads; `rhos` lists the AR(1) coefficients swept for that workload
@@ -72,6 +82,9 @@ CONFIGS = {
     "qwen3_30b": dict(
         shape=Shape(48, 2048, 128, 8, 768, 0, 0, 0, 1, 1, 1),
         cache_slots=32, steps=1024, rhos=(0.5, 0.9), seed=0),
+    "dsv2lite_fp8": dict(
+        shape=Shape(26, 2048, 64, 6, 1408, 2, 1408, 0, 0, 2, 1),
+        cache_slots=16, steps=512, rhos=(0.9, 0.5, 0.0), seed=0),
     "dsv2lite_b32": dict(
         shape=Shape(26, 2048, 64, 6, 1408, 2, 1408, 0, 0, 1, 32),
         cache_slots=32, steps=1024, rhos=(None,), seed=0),
@@ -103,12 +116,65 @@ def bf16_bits_to_f32(bits: np.ndarray) -> np.ndarray:
     return (bits.astype(np.uint32) << np.uint32(16)).view(np.float32)
 
 
+def _fp8_table() -> np.ndarray:
+    """The 256 values of OCP FP8 E4M3: 1 sign, 4 exponent (bias 7), 3 mantissa bits; exponent 0 is
+    subnormal (m/8 * 2^-6); there are no infinities and S.1111.111 is NaN; largest finite 448."""
+    t = np.zeros(256, dtype=np.float32)
+    for b in range(256):
+        sgn = -1.0 if b & 0x80 else 1.0
+        e, m = (b >> 3) & 0xF, b & 7
+        if e == 0xF and m == 7:
+            t[b] = np.nan
+        elif e == 0:
+            t[b] = sgn * (m / 8.0) * 2.0 ** -6
+        else:
+            t[b] = sgn * (1.0 + m / 8.0) * 2.0 ** (e - 7)
+    return t
+
+
+_FP8 = _fp8_table()
+_FP8_POS = _FP8[:127].astype(np.float64)            # non-negative finite values, ascending (0 .. 448)
+_FP8_MID = (_FP8_POS[1:] + _FP8_POS[:-1]) / 2
+
+
+def fp8_e4m3_round_to_bits(x: np.ndarray) -> np.ndarray:
+    """float32 -> FP8 E4M3 bytes: nearest value, ties to the even code, magnitudes above 448 saturate."""
+    x = np.asarray(x, dtype=np.float32)
+    a = np.abs(x).astype(np.float64)
+    idx = np.searchsorted(_FP8_MID, a, side="left")                  # first midpoint >= |x|
+    tie = (idx < len(_FP8_MID)) & (a == _FP8_MID[np.minimum(idx, len(_FP8_MID) - 1)])
+    idx = np.where(tie & (idx % 2 == 1), idx + 1, idx)              # at a midpoint: the even neighbour
+    idx = np.minimum(idx, 126).astype(np.uint8)
+    return (idx | np.where(np.signbit(x), 0x80, 0).astype(np.uint8)).astype(np.uint8)
+
+
+def fp8_e4m3_bits_to_f32(bits: np.ndarray) -> np.ndarray:
+    """FP8 E4M3 bytes -> the float32 values they denote (exact), without the stack-wide scale."""
+    return _FP8[np.asarray(bits, dtype=np.uint8)]
+
+
+def widen(shape: "Shape", a: np.ndarray, router: bool = False) -> np.ndarray:
+    """Stored weights -> the float32 values they denote (router=True for router / gate tensors)."""
+    dt = shape.router_dtype if router else shape.weight_dtype
+    if dt == 1:
+        return bf16_bits_to_f32(a)
+    if dt == 2:
+        return fp8_e4m3_bits_to_f32(a) * np.float32(2.0 ** -FP8_SHIFT)
+    return a
+
+
 def _rng(seed: int, kind: int, a: int = 0, b: int = 0) -> np.random.Generator:
     key = np.array([(int(seed) << 32) | int(kind), (int(a) << 32) | int(b)], dtype=np.uint64)
     return np.random.Generator(np.random.Philox(key=key))
 
 
 def _store(x32: np.ndarray, weight_dtype: int, out: np.ndarray | None) -> np.ndarray:
+    if weight_dtype == 2:
+        bits = fp8_e4m3_round_to_bits(x32 * np.float32(2.0 ** FP8_SHIFT))
+        if out is None:
+            return bits
+        out[...] = bits.reshape(out.shape)
+        return out
     if weight_dtype == 1:
         bits = bf16_round_to_bits(x32)
         if out is None:
@@ -126,7 +192,7 @@ def gen_router(seed: int, shape: Shape, layer: int) -> np.ndarray:
     g = _rng(seed, KIND_ROUTER, layer)
     x = g.standard_normal((shape.n_routed, shape.hidden), dtype=np.float32)
     x *= np.float32(1.0 / np.sqrt(shape.hidden))
-    return _store(x, shape.weight_dtype, None)
+    return _store(x, shape.router_dtype, None)
 
 
 def gen_shared_gate(seed: int, shape: Shape, layer: int) -> np.ndarray:
@@ -134,7 +200,7 @@ def gen_shared_gate(seed: int, shape: Shape, layer: int) -> np.ndarray:
     g = _rng(seed, KIND_SHARED_GATE, layer)
     x = g.standard_normal((shape.hidden,), dtype=np.float32)
     x *= np.float32(1.0 / np.sqrt(shape.hidden))
-    return _store(x, shape.weight_dtype, None)
+    return _store(x, shape.router_dtype, None)
 
 
 def gen_expert_block(seed: int, shape: Shape, layer: int, expert: int,

@@ -65,6 +65,14 @@ def test_extreme_shapes(shape, c, rho):
     _run(shape, c, rho, steps=10, seed=7, dense_steps=1)
 
 
+@pytest.mark.parametrize("shape,c,rho", [
+    (synth.Shape(3, 512, 20, 3, 72, 2, 40, 1, 0, 2, 1), 5, 0.6),        # fp8 expert blocks, bf16 router and gate
+    (synth.Shape(2, 2048, 64, 6, 44, 2, 44, 0, 1, 2, 1), 16, 0.9),      # full hidden width
+])
+def test_fp8_expert_store(shape, c, rho):
+    _run(shape, c, rho, steps=16, seed=9, dense_steps=1, host_api_every=5)
+
+
 def test_many_layers_span_ctas():
     """Enough rows that CTAs cross expert and layer boundaries in the streaming kernel."""
     shape = synth.Shape(12, 512, 16, 4, 300, 1, 300, 0, 0, 1, 1)

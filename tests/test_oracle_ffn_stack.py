@@ -227,7 +227,7 @@ def test_synth_is_reproducible_and_layout():
 
 
 def test_chained_mode_identities():
-    """h_{l+1} = h_l + MoE_l(h_l): telescoping sum, agreement with one-layer stacks run by hand, and
+    """x_l = rmsnorm(h_l), h_{l+1} = h_l + MoE_l(x_l): telescoping sum, agreement with one-layer stacks run by hand, and
     the zero-weight case where every layer sees h_0."""
     shape = synth.Shape(3, 64, 8, 2, 8, 1, 8)
     st = _stack(shape, 3, seed=9, with_ffn=True)
@@ -241,7 +241,9 @@ def test_chained_mode_identities():
     for l in range(3):
         one = orc.OracleStack(synth.Shape(1, 64, 8, 2, 8, 1, 8), 3, [st.routers[l]],
                               lambda _l, e, l=l: st.expert_weights(l, e), lambda _l, i, l=l: st.shared_weights(l, i))
-        r1 = one.step(cur[None], ffn="selected")
+        x = cur / np.sqrt((cur ** 2).sum() / 64 + 1e-6)                # pre-norm, unit RMS
+        assert abs(np.sqrt((x ** 2).mean()) - 1.0) < 1e-5
+        r1 = one.step(x[None], ffn="selected")
         assert np.array_equal(r1["ids"][0], r["ids"][l])
         assert np.allclose(r1["out"][0], r["out"][l], rtol=1e-13, atol=1e-13)
         cur = cur + r1["out"][0]
@@ -251,5 +253,25 @@ def test_chained_mode_identities():
     stz = orc.OracleStack(shape, 3, st.routers, lambda l, e: zero, lambda l, i: zero)
     rz = stz.step(h0, ffn="selected", chained=True)
     assert np.array_equal(rz["final"], h0) and all(np.array_equal(x, h0) for x in rz["layer_inputs"])
-    plain = orc.OracleStack(shape, 3, st.routers).step(np.repeat(h0[None], 3, axis=0), ffn=None)
+    x0 = h0 / np.sqrt((h0 ** 2).mean() + 1e-6)
+    plain = orc.OracleStack(shape, 3, st.routers).step(np.repeat(x0[None], 3, axis=0), ffn=None)
     assert np.array_equal(plain["ids"], rz["ids"])
+
+
+def test_fp8_storage_matches_library_cast():
+    """FP8 E4M3 bytes of the generator against torch's float8_e4m3fn: decode of all 256 codes and
+    round-to-nearest-even encode of in-range values; larger magnitudes saturate at 448."""
+    codes = np.arange(256, dtype=np.uint8)
+    ours = synth.fp8_e4m3_bits_to_f32(codes)
+    ref = torch.from_numpy(codes).view(torch.float8_e4m3fn).to(torch.float32).numpy()
+    assert np.array_equal(np.isnan(ours), np.isnan(ref)) and np.array_equal(ours[~np.isnan(ours)], ref[~np.isnan(ref)])
+    x = np.random.default_rng(0).standard_normal(100000).astype(np.float32) * 5.12
+    x = np.concatenate([x, np.array([0.0, 448.0, 17.0, 18.0, 19.0, 2.0 ** -10, -2.0 ** -10, 0.0009], np.float32)])
+    ref_bits = torch.from_numpy(x).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    assert np.array_equal(synth.fp8_e4m3_round_to_bits(x), ref_bits)
+    assert list(synth.fp8_e4m3_round_to_bits(np.array([1000.0, -1000.0], np.float32))) == [126, 254]
+    shape = synth.Shape(1, 512, 4, 2, 8, 0, 0, 0, 0, 2, 1)
+    blk = synth.gen_expert_block(0, shape, 0, 1)
+    assert blk.dtype == np.uint8 and synth.gen_router(0, shape, 0).dtype == np.uint16
+    w = synth.widen(shape, blk)
+    assert 0.015 < w.std() < 0.025 and np.abs(w).max() < 448 / 256
