@@ -28,6 +28,7 @@ import synth  # noqa: E402
 
 WORKLOAD = "dsv2lite"
 NOMINAL_HBM_GBS = 8000.0
+DTYPE_NAME = {0: "f32", 1: "bf16", 2: "fp8_e4m3"}      # weight storage; accumulation is always f32
 CLOCK_QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
                "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
                "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
@@ -379,7 +380,8 @@ def run_ours(args, rank, world, local_rank):
     km_ms, km_n, km_b = head["kernel_miss"]
     ach = kr_b / (kr_ms / 1e3) / 1e9 if kr_ms > 0 else 0.0
     roofline = {"bound": "hbm", "achieved": ach, "peak": peak_hbm, "unit": "GB/s", "frac": ach / peak_hbm,
-                "traffic": None, "peak_kind": f"of {peak_kind}", "kernel": ("ffn_stream_kernel<bf16,2048>" if shape.batch == 1 else "ffn_batched_kernel<2048>") + " resident phase",
+                "traffic": None, "peak_kind": f"of {peak_kind}", "kernel": (f"ffn_stream_kernel<{DTYPE_NAME[shape.weight_dtype]},{shape.hidden}>" if shape.batch == 1
+                           else f"ffn_batched_kernel<{shape.hidden}>") + " resident phase",
                 "launches": kr_n, "avg_launch_ms": kr_ms / max(1, kr_n), "bytes_per_launch": kr_b / max(1, kr_n),
                 "frac_of_nominal_8TBs": ach / NOMINAL_HBM_GBS}
     miss_phase = {"launches": km_n, "avg_launch_us": km_ms * 1e3 / max(1, km_n),
@@ -406,7 +408,7 @@ def run_ours(args, rank, world, local_rank):
     line = {
         "metric": "decode tokens/s (batch 1, MoE stack)", "value": value, "unit": "tokens/s",
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_step_ms,
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": DTYPE_NAME[shape.weight_dtype], "data": "synthetic",
         "config": {"workload": args.workload, "rho": args.rho, "cache_slots": C, "batch": shape.batch,
                    "layers": shape.n_layers,
                    "l2": "inputs larger than L2 (>= 1.6 GB of expert weights streamed per step)",
