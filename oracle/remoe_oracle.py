@@ -37,14 +37,18 @@ documented property of the CUDA library, so the two can be compared):
   the oldest touch among all slots go (later misses displace this step's earlier entries).
 * Each layer has its own input stream: out[l] = MoE_l(h[l]); layers do not feed each other.
 
-Parity pins (tests/test_oracle_*.py): softmax against closed forms, top-K against a
-stable full sort and constructed ties, LRU against the set characterisation "the C most
-recently used distinct experts" recomputed from the whole history, the exact identity
-misses(t) = K - |E_t n E_{t-1}| when C = K (App. A.3 "Tightness"), both fetch bounds,
-counters against their totals, the FFN against a library matmul in the N = K = 1 case,
-dense-and-mask against selected-only, linearity in the gate weights.  The paper prints
-no worked numeric example for this path, so absolute output values are pinned only by
-those special cases.
+Parity pins (tests/test_oracle_*.py): softmax against closed forms and scipy, top-K against the
+counting definition and constructed ties, LRU/FIFO/LFU against hand-worked slot traces and LRU
+against the set characterisation "the C most recently used distinct experts" recomputed from
+the whole history, the exact identity misses(t) = K - |E_t n E_{t-1}| when C = K (App. A.3
+"Tightness"), both fetch bounds, Belady against exhaustive search, counters against their
+totals and against the uHR / #uMiss table the paper prints (App. E.3), the TPOT proxy against
+the slope of the paper's TPOT table, the FFN against a hand example and a library matmul in the
+N = K = 1 case, dense-and-mask against selected-only, linearity in the gate weights, the
+chained mode against its telescoping sum and hand-run one-layer stacks.  Every function has at
+least one such pin, so none is "parity unpinned"; but the paper prints no worked numeric
+example of a layer output, so absolute float outputs rest on those special cases and library
+routines alone.
 """
 from __future__ import annotations
 
