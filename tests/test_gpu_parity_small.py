@@ -156,3 +156,63 @@ def test_chained_stack(shape, c):
         chk.check_counters()
     finally:
         wl.close()
+
+
+def test_non_finite_input_is_reported_not_faulted():
+    """NaN hidden states make the top-K undefined; the kernels' own index checks turn that into the
+    device-flag status, the context stays usable and a reset clears the condition."""
+    import torch
+    from paper_2605_27081_b200 import binding as B
+    from paper_2605_27081_b200.loader import LoadedWorkload
+    from parity_util import StepChecker, oracle_for
+
+    shape = synth.Shape(2, 256, 64, 6, 16, 0, 0, 0, 0, 1, 1)
+    wl = LoadedWorkload(shape, 8, seed=12)
+    try:
+        x = torch.full((2, 1, 256), float("nan"), device="cuda")
+        out = torch.empty_like(x)
+        ids = torch.zeros((2, 1, 6), dtype=torch.int32, device="cuda")
+        g = torch.zeros((2, 1, 6), device="cuda")
+        rc = B.remoe_decode_step(wl.stack.h, x, out, ids, g)
+        torch.cuda.synchronize()
+        rc2 = B.remoe_decode_step(wl.stack.h, x, out, ids, g)
+        assert B.REMOE_E_DEVICE_FLAG in (rc, rc2)
+        assert "out of range" in B.remoe_last_cuda_error(wl.stack.h)
+        torch.cuda.synchronize()
+        wl.stack.cache_reset()
+        chk = StepChecker(wl, oracle_for(wl), torch)
+        hs = synth.HiddenStream(12, shape, 0.5)
+        for _ in range(5):
+            chk.step(hs.step())
+        chk.check_counters()
+    finally:
+        wl.close()
+
+
+def test_policy_switch_and_second_stack_share_a_store():
+    """Two stacks over the same pinned store (different capacity and policy) stay independent."""
+    import torch
+    from paper_2605_27081_b200.loader import LoadedWorkload
+    from parity_util import StepChecker, oracle_for
+    import copy
+
+    shape = synth.Shape(2, 256, 16, 2, 24, 1, 8, 0, 0, 1, 1)
+    wl = LoadedWorkload(shape, 4, seed=13)
+    wl2 = copy.copy(wl)
+    wl2.cache_slots = 7
+    wl2.stack = wl.new_stack(7)
+    try:
+        wl2.stack.set_policy(1)
+        a = StepChecker(wl, oracle_for(wl), torch)
+        b = StepChecker(wl2, oracle_for(wl2, "fifo"), torch)
+        hs = synth.HiddenStream(13, shape, 0.6)
+        for _ in range(25):
+            h = hs.step()
+            a.step(h)
+            b.step(h)
+        a.check_counters()
+        b.check_counters()
+        assert a.o.uniq_misses != b.o.uniq_misses
+    finally:
+        wl2.stack.close()
+        wl.close()
