@@ -10,7 +10,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libremoe.so")
-SOURCES = ["route.cu", "ffn_stream.cu", "ffn_batched.cu", "api.cu", "ffn_static.cu"]
+SOURCES = ["route.cu", "ffn_stream.cu", "ffn_batched.cu", "ffn_batched_tc.cu", "api.cu", "ffn_static.cu"]
 
 
 def _nvcc() -> str:

@@ -56,6 +56,8 @@ struct remoe_stack {
   int max_items = 0;
   int step_serial = 0;                    // never reset: stamps partial rows
   cudaEvent_t ev_resident = nullptr;
+  bool use_tc = false;                     // batched experts on tcgen05 / TMEM
+  alignas(64) unsigned char tc_maps[1024];
   std::vector<cudaEvent_t> ev_pool;        // copy-done / compute-done events of the waves
   uint64_t steps = 0, steps_since_reset = 0;
   std::vector<uint64_t> h2d_bytes;         // per layer
@@ -202,6 +204,11 @@ int check_device_flag(remoe_stack* s) {
 // expert of this step and may only be copied once that one has been computed.  Copies are queued
 // depth by depth, layer by layer, so the copy engine stays busy; each (depth, layer) group is
 // computed as soon as its copies have landed.
+cudaError_t launch_batched(remoe_stack* s, const BatchArgs& a) {
+  return s->use_tc ? launch_ffn_batched_tc(a, s->tc_maps, s->grid, s->stream)
+                   : launch_ffn_batched(a, s->grid, s->stream);
+}
+
 int decode_step_batched(remoe_stack* s, const float* hin, float* hout, int32_t* ids, float* gates) {
   DevStack& d = s->d;
   d.has_prev = s->steps_since_reset > 0 ? 1 : 0;
@@ -228,7 +235,7 @@ int decode_step_batched(remoe_stack* s, const float* hin, float* hout, int32_t* 
   a.depth = 0;
   int rc = prof_begin(s, s->stream, 0, 0);
   if (rc != REMOE_OK) return rc;
-  CK(launch_ffn_batched(a, s->grid, s->stream));
+  CK(launch_batched(s, a));
   s->kernel_launches += 2;
   rc = prof_end(s, s->stream);
   if (rc != REMOE_OK) return rc;
@@ -317,7 +324,7 @@ int decode_step_batched(remoe_stack* s, const float* hin, float* hout, int32_t* 
         if (!t_hit[l * BK + i] && t_depth[l * BK + i] == dep) bytes += d.slot_bytes;
       rc = prof_begin(s, s->stream, bytes, 1);
       if (rc != REMOE_OK) return rc;
-      CK(launch_ffn_batched(a, s->grid, s->stream));
+      CK(launch_batched(s, a));
       s->kernel_launches += 2;
       rc = prof_end(s, s->stream);
       if (rc != REMOE_OK) return rc;
@@ -452,10 +459,16 @@ int remoe_stack_create(const remoe_shape* sh, int32_t cache_slots, void* cuda_st
     TRY(dev_alloc(s, &d.grp_k, L * s->BK * d.B));
     TRY(dev_alloc(s, &s->part, L * d.B * P * kUnitsPerItem * d.H));
     TRY(dev_alloc(s, &s->flags, L * d.B * P * kUnitsPerItem));
-    s->max_items = (int)(L * (s->BK + (size_t)d.S * ((d.B + kTokTile - 1) / kTokTile))) + 1;
+    s->max_items = (int)(L * (s->BK + (size_t)d.S * ((d.B + kMinTokTile - 1) / kMinTokTile))) + 1;
     TRY(dev_alloc(s, &s->plan, (size_t)8 + 4 * (size_t)s->max_items));
     if (cudaMemset(s->flags, 0, L * d.B * P * kUnitsPerItem * sizeof(int)) != cudaSuccess) return bail(REMOE_E_CUDA);
     if (cudaEventCreateWithFlags(&s->ev_resident, cudaEventDisableTiming) != cudaSuccess) return bail(REMOE_E_CUDA);
+    const char* pick = std::getenv("REMOE_BATCHED_KERNEL");      // "mma" forces the mma.sync kernel
+    if (ffn_batched_tc_supported(d) && ffn_batched_tc_maps_bytes() <= sizeof(s->tc_maps) &&
+        !(pick && std::strcmp(pick, "mma") == 0)) {
+      if (ffn_batched_tc_init(d, s->tc_maps) != cudaSuccess) return bail(REMOE_E_CUDA);
+      s->use_tc = true;
+    }
   }
   const size_t io = L * d.B * d.H, kk = L * (size_t)s->BK;
   TRY(dev_alloc(s, &s->st_in_d, io));

@@ -1,0 +1,438 @@
+// Batched expert step on the fifth-generation tensor cores (tcgen05 / TMEM), sm_100a.
+//
+// Same work list as ffn_batched.cu, with a work item of (layer, expert, tile of up to 16 tokens)
+// and channel blocks of 64.  Per CTA (one per SM, 192 threads):
+//   warp 4   TMA producer: tiled tensor-map loads (cp.async.bulk.tensor, 128-byte swizzle, no
+//            multicast) of 16 KB operand tiles into a shared-memory ring:
+//              A1 tile  = [64 channels x {gate, up}] x 64 columns of H   (K-major, 128 rows)
+//              A2 tile  = 64 channels x 128 columns of W_down             (MN-major, two boxes)
+//   warp 5   one elected thread issues tcgen05.mma (M = 128, N = 16, K = 16, bf16 -> fp32):
+//              D1[128 x 16]        += A1(kc) . X^T(kc)        for the H/64 column chunks
+//              D2[ht][128 x 16]    += A2(ht)^T . a            for the H/128 output tiles
+//            and releases ring stages / signals the other warps with tcgen05.commit;
+//   warps 0-3  stage the token tile's hidden states as the bf16 B operand X^T (swizzled by hand),
+//            read D1 from TMEM (tcgen05.ld; gate and up rows of a channel sit in neighbouring
+//            lanes), form a = silu(g) * u * gate weight in bf16 as the second B operand, and at
+//            the end of a piece read D2 and write one stamped partial row per (token, rank).
+// Accumulators live in TMEM: D1 in 16 columns, D2 in 16 columns per 128 rows of H (256 columns
+// at H = 2048).  All waits are bounded mbarrier waits; a failed wait raises the error flag, every
+// role leaves its loops, the producer waits for copies in flight and TMEM is freed.
+#include <cuda.h>
+
+#include <cstring>
+
+#include "remoe_internal.cuh"
+#include "tma_ring.cuh"
+#include "batched_plan.cuh"
+
+namespace remoe {
+
+namespace {
+
+constexpr int kTcTokTile = 16;
+constexpr int kTcBlockCh = 64;
+constexpr int kTcThreads = 192;
+constexpr int kTileBytes = 16384;                      // one ring stage: 128 rows x 128 B
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kD2Col = 32;                        // D1 at column 0, D2 tiles from column 32
+
+using namespace ring;
+
+__device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, int c0, int c1, int c2, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];" ::"r"(
+          smem_u32(dst)),
+      "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+// Shared-memory matrix descriptor, 128-byte swizzle: start address, leading and stride byte
+// offsets in 16-byte units, descriptor version 1 in bits 46-47, layout type 2 in bits 61-63.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  return (uint64_t)((addr >> 4) & 0x3fffu) | ((uint64_t)((lbo_bytes >> 4) & 0x3fffu) << 16) |
+         ((uint64_t)((sbo_bytes >> 4) & 0x3fffu) << 32) | ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+// Instruction descriptor: fp32 accumulate (bits 4-5 = 1), bf16 A and B (bits 7-9, 10-12 = 1),
+// N >> 3 in bits 17-22, M >> 4 in bits 24-28; bit 15 set = A is MN-major.
+constexpr uint32_t kIdescK = (1u << 4) | (1u << 7) | (1u << 10) | ((kTcTokTile >> 3) << 17) | ((128u >> 4) << 24);
+constexpr uint32_t kIdescMN = kIdescK | (1u << 15);
+
+__device__ __forceinline__ void umma(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}" ::"r"(tmem_d),
+      "l"(da), "l"(db), "r"(idesc), "r"(accumulate), "r"(0u)
+      : "memory");
+}
+// Arrives on `bar` once every tcgen05.mma issued so far by this thread has completed.
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void proxy_fence() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+// 16 consecutive fp32 columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+
+struct TcMaps {
+  CUtensorMap slots_gu, slots_d, shared_gu, shared_d;
+};
+
+template <int H>
+struct TcGeo {
+  static constexpr int kChunks = H / 64;               // K chunks of the first contraction
+  static constexpr int kTiles = H / 128;               // output tiles of the second contraction
+  static constexpr int kB1Bytes = kChunks * 2048;      // X^T: 16 tokens x 128 B per chunk
+  static constexpr int kB2Bytes = 2048;                // a: 16 tokens x 64 channels
+  static constexpr int kFixed = kB1Bytes + kB2Bytes;
+  static constexpr int kStages = (227 * 1024 - 2048 - kFixed) / kTileBytes > 10 ? 10 : (227 * 1024 - 2048 - kFixed) / kTileBytes;
+  static constexpr size_t kSmem = 1024 + kFixed + (size_t)kStages * kTileBytes + 512;
+};
+
+template <int H>
+__global__ void __launch_bounds__(kTcThreads, 1)
+ffn_batched_tc_kernel(const __grid_constant__ BatchArgs a, const __grid_constant__ TcMaps maps) {
+  using G = TcGeo<H>;
+  constexpr int NS = G::kStages;
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  unsigned char* b1 = smem;
+  unsigned char* b2 = b1 + G::kB1Bytes;
+  unsigned char* ring = b2 + G::kB2Bytes;                              // 1024-byte aligned
+  uint64_t* bars = reinterpret_cast<uint64_t*>(ring + (size_t)NS * kTileBytes);
+  uint64_t *full = bars, *empty = bars + NS;
+  uint64_t* x_full = bars + 2 * NS;        // + 0 x_full, 1 x_empty, 2 d1_full, 3 d1_empty, 4 b2_full, 5 b2_empty,
+  uint64_t* x_empty = x_full + 1;          //   6 d2_full, 7 d2_empty, 8 drain
+  uint64_t* d1_full = x_full + 2;
+  uint64_t* d1_empty = x_full + 3;
+  uint64_t* b2_full = x_full + 4;
+  uint64_t* b2_empty = x_full + 5;
+  uint64_t* d2_full = x_full + 6;
+  uint64_t* d2_empty = x_full + 7;
+  uint64_t* drain = x_full + 8;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(x_full + 9);
+  __shared__ int s_abort;
+
+  const DevStack& d = a.d;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int BK = d.B * d.K, P = d.K + d.S;
+
+  if (tid == 0) {
+    s_abort = 0;
+    for (int s = 0; s < NS; ++s) { mbar_init(full + s, 1); mbar_init(empty + s, 1); }
+    mbar_init(x_full, 128); mbar_init(x_empty, 1);
+    mbar_init(d1_full, 1); mbar_init(d1_empty, 128);
+    mbar_init(b2_full, 128); mbar_init(b2_empty, 1);
+    mbar_init(d2_full, 1); mbar_init(d2_empty, 128);
+    mbar_init(drain, 1);
+    mbar_fence_init();
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"(kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  const int n_items = a.plan[0], n_units = a.plan[1];
+  const int q = (n_units + (int)gridDim.x - 1) / (int)gridDim.x;
+  const int ua = min(n_units, (int)blockIdx.x * q), ub = min(n_units, ua + q);
+  const bool have_work = ua < ub;
+  const int j0 = have_work ? first_item(a, n_items, ua) : 0;
+  auto aborted = [&]() { return *(volatile int*)&s_abort != 0; };
+  auto fail = [&](int code) { atomicCAS(d.err, kErrNone, code); atomicExch(&s_abort, 1); };
+
+  if (have_work && warp == 4) {
+    // ---------------------------------------------------------------- TMA producer
+    if (lane == 0) {
+      int n = 0;
+      bool ok = true;
+      for (int j = j0; j < n_items && ok; ++j) {
+        if (a.plan[kPlanHeader + 4 * j + 3] >= ub) break;
+        PieceInfo p;
+        if (!make_piece(a, j, ua, ub, p)) continue;
+        const CUtensorMap* m_gu = p.shared ? &maps.shared_gu : &maps.slots_gu;
+        const CUtensorMap* m_d = p.shared ? &maps.shared_d : &maps.slots_d;
+        const char* pool = p.shared ? d.shared_blocks : d.slots;
+        const int row0 = (int)((p.base - pool) / ((size_t)3 * H * 2));       // channel row of the expert's first channel
+        for (int blk = p.blk0; blk < p.blk1 && ok; ++blk) {
+          const int row = row0 + blk * kTcBlockCh;
+          for (int t = 0; t < G::kChunks + G::kTiles; ++t, ++n) {
+            const int s = n % NS;
+            if (n >= NS && (aborted() || !mbar_wait(empty + s, ((n / NS) - 1) & 1))) {
+              if (!aborted()) fail(kErrWaitEmpty);
+              ok = false;
+              break;
+            }
+            unsigned char* dst = ring + (size_t)s * kTileBytes;
+            mbar_expect_tx(full + s, kTileBytes);
+            if (t < G::kChunks) {
+              tma_load_3d(dst, m_gu, t * 64, 0, row, full + s);
+            } else {
+              const int ht = t - G::kChunks;
+              tma_load_3d(dst, m_d, ht * 128, 2, row, full + s);
+              tma_load_3d(dst + kTileBytes / 2, m_d, ht * 128 + 64, 2, row, full + s);
+            }
+          }
+        }
+      }
+      if (!ok) {
+        for (int m = max(0, n - NS); m < n; ++m)
+          if (!mbar_wait(full + (m % NS), (m / NS) & 1)) atomicCAS(d.err, kErrNone, kErrDrain);
+      }
+    }
+  } else if (have_work && warp == 5) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      int n = 0, np = 0, ng = 0;
+      bool ok = true;
+      for (int j = j0; j < n_items && ok; ++j) {
+        if (a.plan[kPlanHeader + 4 * j + 3] >= ub) break;
+        PieceInfo p;
+        if (!make_piece(a, j, ua, ub, p)) continue;
+        ok = !aborted() && mbar_wait(x_full, np & 1);
+        if (ok && np > 0) ok = mbar_wait(d2_empty, (np - 1) & 1);
+        for (int blk = p.blk0; blk < p.blk1 && ok; ++blk, ++ng) {
+          if (ng > 0) ok = !aborted() && mbar_wait(d1_empty, (ng - 1) & 1);
+          for (int kc = 0; kc < G::kChunks && ok; ++kc, ++n) {
+            const int s = n % NS;
+            ok = !aborted() && mbar_wait(full + s, (n / NS) & 1);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t a_addr = smem_u32(ring + (size_t)s * kTileBytes), b_addr = smem_u32(b1 + kc * 2048);
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+              umma(tmem, smem_desc(a_addr + k * 32, 16, 1024), smem_desc(b_addr + k * 32, 16, 1024), kIdescK,
+                   (kc | k) ? 1u : 0u);
+            umma_commit(empty + s);
+          }
+          if (!ok) break;
+          umma_commit(d1_full);
+          if (blk + 1 == p.blk1) umma_commit(x_empty);             // X^T of this piece is no longer needed
+          ok = !aborted() && mbar_wait(b2_full, ng & 1);
+          tc_fence_after();
+          for (int ht = 0; ht < G::kTiles && ok; ++ht, ++n) {
+            const int s = n % NS;
+            ok = !aborted() && mbar_wait(full + s, (n / NS) & 1);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t a_addr = smem_u32(ring + (size_t)s * kTileBytes), b_addr = smem_u32(b2);
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+              umma(tmem + kD2Col + ht * 16, smem_desc(a_addr + k * 2048, 8192, 1024), smem_desc(b_addr + k * 32, 16, 1024),
+                   kIdescMN, (blk > p.blk0 || k) ? 1u : 0u);
+            umma_commit(empty + s);
+          }
+          if (!ok) break;
+          umma_commit(b2_empty);
+        }
+        if (ok) { umma_commit(d2_full); ++np; }
+      }
+      if (!ok) {
+        if (!aborted()) fail(kErrWaitFull);
+        umma_commit(drain);                                       // let the tensor cores finish before TMEM is freed
+        mbar_wait(drain, 0);
+      }
+    }
+  } else if (have_work) {
+    // ------------------------------------------------------------- epilogue warps 0-3
+    int np = 0, ng = 0;
+    bool ok = true;
+    const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+    for (int j = j0; j < n_items && ok; ++j) {
+      if (a.plan[kPlanHeader + 4 * j + 3] >= ub) break;
+      PieceInfo p;
+      if (!make_piece(a, j, ua, ub, p)) continue;
+      const int gidx = (p.l * BK + p.cand) * d.B + p.tile * kTcTokTile;
+      auto tok_of = [&](int t) -> int {
+        if (t >= p.n_tok) return -1;
+        return p.shared ? p.tile * kTcTokTile + t : d.grp_tok[gidx + t];
+      };
+      auto kq_of = [&](int t) -> int { return p.shared ? d.K + (p.cand - BK) : d.grp_k[gidx + t]; };
+
+      // X^T tile: 16 tokens x H as bf16, 128-byte rows per 64-column chunk, 16-byte pieces XORed with the row
+      if (np > 0) ok = !aborted() && mbar_wait(x_empty, (np - 1) & 1);
+      if (!ok) break;
+      for (int e = tid; e < kTcTokTile * (H / 8); e += 128) {
+        const int t = e / (H / 8), c8 = e % (H / 8);              // token, 8-column group
+        const int tok = tok_of(t);
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (tok >= 0) {
+          const float4* src = reinterpret_cast<const float4*>(a.hidden_in + ((size_t)p.l * d.B + tok) * H + c8 * 8);
+          const float4 x0 = __ldg(src), x1 = __ldg(src + 1);
+          v = make_uint4(pack_bf16(x0.x, x0.y), pack_bf16(x0.z, x0.w), pack_bf16(x1.x, x1.y), pack_bf16(x1.z, x1.w));
+        }
+        const int kc = c8 >> 3, c = c8 & 7;
+        *reinterpret_cast<uint4*>(b1 + kc * 2048 + t * 128 + ((c ^ (t & 7)) << 4)) = v;
+      }
+      proxy_fence();
+      mbar_arrive(x_full);
+      // per-token scale of this piece (column j of the accumulators is token j of the tile)
+      float sc[kTcTokTile];
+#pragma unroll
+      for (int t = 0; t < kTcTokTile; ++t) {
+        const int tok = tok_of(t);
+        sc[t] = tok < 0 ? 0.f
+                        : (p.shared ? d.shared_scale[p.l * d.B + tok]
+                                    : a.gates[((size_t)p.l * d.B + tok) * d.K + kq_of(t)]);
+      }
+
+      for (int blk = p.blk0; blk < p.blk1 && ok; ++blk, ++ng) {
+        ok = !aborted() && mbar_wait(d1_full, ng & 1);
+        if (!ok) break;
+        tc_fence_after();
+        float v[16];
+        tmem_ld16(tmem + lane_base, v);
+        tc_fence_before();
+        mbar_arrive(d1_empty);
+        if (ng > 0) ok = !aborted() && mbar_wait(b2_empty, (ng - 1) & 1);
+        if (!ok) break;
+        // lane 2c holds the gate row of channel c, lane 2c+1 its up row
+        const int ch = (warp * 32 + lane) >> 1;
+#pragma unroll
+        for (int t = 0; t < kTcTokTile; ++t) {
+          const float u = __shfl_down_sync(kFull, v[t], 1);
+          if ((lane & 1) == 0) {
+            const float av = v[t] / (1.f + __expf(-v[t])) * u * sc[t];
+            const uint32_t bits = pack_bf16(av, 0.f) & 0xffffu;
+            *reinterpret_cast<unsigned short*>(b2 + t * 128 + (((ch >> 3) ^ (t & 7)) << 4) + ((ch & 7) << 1)) =
+                (unsigned short)bits;
+          }
+        }
+        proxy_fence();
+        mbar_arrive(b2_full);
+      }
+      if (!ok) break;
+      // piece done: read the output tiles and write one stamped partial row per (token, rank)
+      ok = !aborted() && mbar_wait(d2_full, np & 1);
+      if (!ok) break;
+      tc_fence_after();
+      size_t rows[kTcTokTile];
+#pragma unroll
+      for (int t = 0; t < kTcTokTile; ++t) {
+        const int tok = tok_of(t);
+        rows[t] = tok < 0 ? (size_t)-1 : (((size_t)p.l * d.B + tok) * P + kq_of(t)) * kUnitsPerItem + p.first_unit;
+      }
+      for (int ht = 0; ht < G::kTiles; ++ht) {
+        float v[16];
+        tmem_ld16(tmem + lane_base + kD2Col + ht * 16, v);
+        const int h = ht * 128 + warp * 32 + lane;
+#pragma unroll
+        for (int t = 0; t < kTcTokTile; ++t)
+          if (rows[t] != (size_t)-1) a.part[rows[t] * H + h] = v[t];
+      }
+      tc_fence_before();
+      mbar_arrive(d2_empty);
+#pragma unroll
+      for (int t = 0; t < kTcTokTile; ++t)
+        if (tid == t && rows[t] != (size_t)-1) a.flags[rows[t]] = a.step_id;
+      ++np;
+    }
+    if (!ok && !aborted()) fail(kErrWaitFull);
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (warp == 0)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// A pool of expert blocks as a 3-D bf16 tensor (H columns, 3 row kinds, channel rows of all blocks).
+bool encode_pool(EncodeTiledFn encode, CUtensorMap* gu, CUtensorMap* dn, const void* base, int H, size_t rows) {
+  if (rows == 0) {
+    std::memset(gu, 0, sizeof(*gu));
+    std::memset(dn, 0, sizeof(*dn));
+    return true;
+  }
+  cuuint64_t dims[3] = {(cuuint64_t)H, 3, (cuuint64_t)rows};
+  cuuint64_t strides[2] = {(cuuint64_t)H * 2, (cuuint64_t)3 * H * 2};
+  cuuint32_t box_gu[3] = {64, 2, 64}, box_d[3] = {64, 1, 64}, estr[3] = {1, 1, 1};
+  void* p = const_cast<void*>(base);
+  return encode(gu, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, p, dims, strides, box_gu, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS &&
+         encode(dn, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, p, dims, strides, box_d, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int H>
+cudaError_t launch_tc(const BatchArgs& a, const TcMaps& maps, int grid, cudaStream_t st) {
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(ffn_batched_tc_kernel<H>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)TcGeo<H>::kSmem);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  BatchArgs b = a;
+  b.tok_tile = kTcTokTile;
+  b.blk_ch = kTcBlockCh;
+  plan_kernel<<<1, 1024, 0, st>>>(b);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  ffn_batched_tc_kernel<H><<<grid, kTcThreads, TcGeo<H>::kSmem, st>>>(b, maps);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+bool ffn_batched_tc_supported(const DevStack& d) {
+  if (d.wbytes != 2) return false;
+  if (d.H != 256 && d.H != 512 && d.H != 1024 && d.H != 2048) return false;
+  if (d.I % kTcBlockCh || (d.S && d.Is % kTcBlockCh)) return false;
+  return true;
+}
+
+size_t ffn_batched_tc_maps_bytes() { return sizeof(TcMaps); }
+
+cudaError_t ffn_batched_tc_init(const DevStack& d, void* maps_out) {
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+  if (e != cudaSuccess) return e;
+  if (!fn) return cudaErrorNotSupported;
+  TcMaps* m = static_cast<TcMaps*>(maps_out);
+  EncodeTiledFn encode = reinterpret_cast<EncodeTiledFn>(fn);
+  if (!encode_pool(encode, &m->slots_gu, &m->slots_d, d.slots, d.H, (size_t)d.L * d.C * d.I)) return cudaErrorInvalidValue;
+  if (!encode_pool(encode, &m->shared_gu, &m->shared_d, d.shared_blocks, d.H, (size_t)d.L * d.S * d.Is))
+    return cudaErrorInvalidValue;
+  return cudaSuccess;
+}
+
+cudaError_t launch_ffn_batched_tc(const BatchArgs& a, const void* maps, int grid, cudaStream_t st) {
+  const TcMaps& m = *static_cast<const TcMaps*>(maps);
+  switch (a.d.H) {
+    case 256: return launch_tc<256>(a, m, grid, st);
+    case 512: return launch_tc<512>(a, m, grid, st);
+    case 1024: return launch_tc<1024>(a, m, grid, st);
+    case 2048: return launch_tc<2048>(a, m, grid, st);
+  }
+  return cudaErrorInvalidValue;
+}
+
+}  // namespace remoe

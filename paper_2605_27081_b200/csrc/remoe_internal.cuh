@@ -86,7 +86,7 @@ struct FfnArgs {
 };
 
 // Batched (B > 1) expert kernels: tensor-core grouped GEMM over per-expert token groups.
-constexpr int kTokTile = 8;            // tokens per work item (the MMA's N)
+constexpr int kMinTokTile = 8;         // smallest token tile of a batched kernel (bounds the item count)
 constexpr int kUnitsPerItem = 16;      // an item's channels are cut into this many units
 struct BatchArgs {
   DevStack d;
@@ -99,10 +99,17 @@ struct BatchArgs {
   int* flags;                          // [L][B][K+S][kUnitsPerItem]
   int* plan;                           // header (8 ints) + items (4 ints each)
   int max_items;
+  int tok_tile, blk_ch;                // tokens per item, channels per block (set by the launcher)
 };
 bool ffn_batched_supported(const DevStack& d);
 cudaError_t launch_ffn_batched(const BatchArgs& a, int grid, cudaStream_t st);
 cudaError_t launch_combine_batched(const BatchArgs& a, float* hidden_out, cudaStream_t st);
+// tcgen05 / TMEM variant (needs I and I_shared multiples of 64); `maps` is an opaque, 64-byte aligned
+// block of ffn_batched_tc_maps_bytes() bytes filled once per stack by ffn_batched_tc_init.
+bool ffn_batched_tc_supported(const DevStack& d);
+size_t ffn_batched_tc_maps_bytes();
+cudaError_t ffn_batched_tc_init(const DevStack& d, void* maps_out);
+cudaError_t launch_ffn_batched_tc(const BatchArgs& a, const void* maps, int grid, cudaStream_t st);
 
 // Routes layers [layer0, layer0 + n_layers); `hidden_in`, `ids`, `gates` are the full [L, B, .] arrays.
 cudaError_t launch_route(const DevStack& d, const float* hidden_in, int* ids, float* gates,

@@ -43,5 +43,18 @@ def test_batched_shapes(shape, c, rho):
         assert deepest > c                     # the case the capacity assumption excludes did occur
 
 
+@pytest.mark.parametrize("shape,c,rho", [
+    (synth.Shape(2, 256, 16, 2, 64, 1, 64, 0, 0, 1, 4), 6, 0.5),         # one 64-channel block per expert
+    (synth.Shape(3, 512, 24, 3, 128, 2, 64, 1, 0, 1, 12), 8, None),      # union far above capacity, sigmoid gate
+    (synth.Shape(2, 1024, 40, 4, 64, 0, 0, 0, 1, 1, 20), 40, 0.7),       # all resident, B not a multiple of 16
+    (synth.Shape(2, 2048, 64, 6, 192, 2, 192, 0, 0, 1, 32), 32, None),   # the serving configuration's layer shape
+    (synth.Shape(2, 512, 16, 4, 1408, 1, 128, 0, 0, 1, 40), 16, 0.6),    # 22 blocks per expert (11 units), groups above 16 tokens
+])
+def test_batched_tensor_core_path(shape, c, rho):
+    """Intermediate sizes that are multiples of 64 run on the tcgen05 / TMEM kernel."""
+    chk, _ = _run(shape, c, rho, steps=10, seed=5)
+    assert chk.max_out_err <= 2e-2
+
+
 def test_batched_other_policy():
     _run(synth.Shape(2, 256, 16, 2, 64, 0, 0, 0, 0, 1, 6), 5, 0.4, steps=30, seed=4, dense_steps=0, policy=2)
