@@ -14,7 +14,9 @@
 //            read D1 from TMEM (tcgen05.ld; gate and up rows of a channel sit in neighbouring
 //            lanes), form a = silu(g) * u * gate weight in bf16 as the second B operand, and at
 //            the end of a piece read D2 and write one stamped partial row per (token, rank).
-// Accumulators live in TMEM: D1 in 16 columns, D2 in 16 columns per 128 rows of H (256 columns
+// The first contraction of group g+1 is issued before the second contraction of group g (D1 is
+// double buffered), so the tensor pipe and the weight stream never wait for the activation step.
+// Accumulators live in TMEM: D1 in 2 x 16 columns, D2 in 16 columns per 128 rows of H (256 columns
 // at H = 2048).  All waits are bounded mbarrier waits; a failed wait raises the error flag, every
 // role leaves its loops, the producer waits for copies in flight and TMEM is freed.
 #include <cuda.h>
@@ -34,7 +36,7 @@ constexpr int kTcBlockCh = 64;
 constexpr int kTcThreads = 192;
 constexpr int kTileBytes = 16384;                      // one ring stage: 128 rows x 128 B
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kD2Col = 32;                        // D1 at column 0, D2 tiles from column 32
+constexpr uint32_t kD2Col = 32;                        // D1 buffers at columns 0 and 16, D2 tiles from column 32
 
 using namespace ring;
 
@@ -93,6 +95,36 @@ struct TcMaps {
   CUtensorMap slots_gu, slots_d, shared_gu, shared_d;
 };
 
+// Walks the 64-channel groups of a CTA's unit range in order, piece by piece.
+struct GroupRec {
+  PieceInfo p;
+  int blk;          // channel block within the expert
+  int np;           // running piece number within this CTA
+  int idx;          // running group number within this CTA
+  bool first, last; // first / last group of its piece
+};
+struct GroupWalk {
+  const BatchArgs& a;
+  int n_items, ua, ub, j, np, idx, blk;
+  PieceInfo p;
+  bool in_piece;
+  __device__ GroupWalk(const BatchArgs& a_, int n_items_, int ua_, int ub_, int j0)
+      : a(a_), n_items(n_items_), ua(ua_), ub(ub_), j(j0), np(-1), idx(0), blk(0), in_piece(false) {}
+  __device__ bool next(GroupRec& g) {
+    while (!in_piece) {
+      if (j >= n_items || a.plan[kPlanHeader + 4 * j + 3] >= ub) return false;
+      const bool got = make_piece(a, j, ua, ub, p);
+      ++j;
+      if (got && p.blk0 < p.blk1) { in_piece = true; blk = p.blk0; ++np; }
+    }
+    g.p = p; g.blk = blk; g.np = np; g.idx = idx++;
+    g.first = blk == p.blk0;
+    g.last = blk + 1 == p.blk1;
+    if (++blk == p.blk1) in_piece = false;
+    return true;
+  }
+};
+
 template <int H>
 struct TcGeo {
   static constexpr int kChunks = H / 64;               // K chunks of the first contraction
@@ -116,16 +148,16 @@ ffn_batched_tc_kernel(const __grid_constant__ BatchArgs a, const __grid_constant
   unsigned char* ring = b2 + G::kB2Bytes;                              // 1024-byte aligned
   uint64_t* bars = reinterpret_cast<uint64_t*>(ring + (size_t)NS * kTileBytes);
   uint64_t *full = bars, *empty = bars + NS;
-  uint64_t* x_full = bars + 2 * NS;        // + 0 x_full, 1 x_empty, 2 d1_full, 3 d1_empty, 4 b2_full, 5 b2_empty,
-  uint64_t* x_empty = x_full + 1;          //   6 d2_full, 7 d2_empty, 8 drain
-  uint64_t* d1_full = x_full + 2;
-  uint64_t* d1_empty = x_full + 3;
-  uint64_t* b2_full = x_full + 4;
-  uint64_t* b2_empty = x_full + 5;
-  uint64_t* d2_full = x_full + 6;
-  uint64_t* d2_empty = x_full + 7;
-  uint64_t* drain = x_full + 8;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(x_full + 9);
+  uint64_t* x_full = bars + 2 * NS;        // X^T of a piece staged            (128 epilogue threads)
+  uint64_t* x_empty = x_full + 1;          // X^T no longer read                 (commit)
+  uint64_t* d1_full = x_full + 2;          // [2] first contraction of a group done (commit)
+  uint64_t* d1_empty = x_full + 4;         // [2] D1 buffer read out             (128 threads)
+  uint64_t* b2_full = x_full + 6;          // activations of a group staged      (128 threads)
+  uint64_t* b2_empty = x_full + 7;         // second contraction of a group done (commit)
+  uint64_t* d2_full = x_full + 8;          // a piece's output complete          (commit)
+  uint64_t* d2_empty = x_full + 9;         // a piece's output read out          (128 threads)
+  uint64_t* drain = x_full + 10;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(x_full + 11);
   __shared__ int s_abort;
 
   const DevStack& d = a.d;
@@ -136,7 +168,8 @@ ffn_batched_tc_kernel(const __grid_constant__ BatchArgs a, const __grid_constant
     s_abort = 0;
     for (int s = 0; s < NS; ++s) { mbar_init(full + s, 1); mbar_init(empty + s, 1); }
     mbar_init(x_full, 128); mbar_init(x_empty, 1);
-    mbar_init(d1_full, 1); mbar_init(d1_empty, 128);
+    mbar_init(d1_full, 1); mbar_init(d1_full + 1, 1);
+    mbar_init(d1_empty, 128); mbar_init(d1_empty + 1, 128);
     mbar_init(b2_full, 128); mbar_init(b2_empty, 1);
     mbar_init(d2_full, 1); mbar_init(d2_empty, 128);
     mbar_init(drain, 1);
@@ -163,38 +196,45 @@ ffn_batched_tc_kernel(const __grid_constant__ BatchArgs a, const __grid_constant
 
   if (have_work && warp == 4) {
     // ---------------------------------------------------------------- TMA producer
+    // Tile order: A1(g0); A1(g1), A2(g0); A1(g2), A2(g1); ... ; A2(last) -- the order the MMA
+    // thread consumes them in.
     if (lane == 0) {
       int n = 0;
       bool ok = true;
-      for (int j = j0; j < n_items && ok; ++j) {
-        if (a.plan[kPlanHeader + 4 * j + 3] >= ub) break;
-        PieceInfo p;
-        if (!make_piece(a, j, ua, ub, p)) continue;
-        const CUtensorMap* m_gu = p.shared ? &maps.shared_gu : &maps.slots_gu;
-        const CUtensorMap* m_d = p.shared ? &maps.shared_d : &maps.slots_d;
-        const char* pool = p.shared ? d.shared_blocks : d.slots;
-        const int row0 = (int)((p.base - pool) / ((size_t)3 * H * 2));       // channel row of the expert's first channel
-        for (int blk = p.blk0; blk < p.blk1 && ok; ++blk) {
-          const int row = row0 + blk * kTcBlockCh;
-          for (int t = 0; t < G::kChunks + G::kTiles; ++t, ++n) {
-            const int s = n % NS;
-            if (n >= NS && (aborted() || !mbar_wait(empty + s, ((n / NS) - 1) & 1))) {
-              if (!aborted()) fail(kErrWaitEmpty);
-              ok = false;
-              break;
-            }
-            unsigned char* dst = ring + (size_t)s * kTileBytes;
-            mbar_expect_tx(full + s, kTileBytes);
-            if (t < G::kChunks) {
-              tma_load_3d(dst, m_gu, t * 64, 0, row, full + s);
-            } else {
-              const int ht = t - G::kChunks;
-              tma_load_3d(dst, m_d, ht * 128, 2, row, full + s);
-              tma_load_3d(dst + kTileBytes / 2, m_d, ht * 128 + 64, 2, row, full + s);
-            }
+      auto emit = [&](const GroupRec& g, bool second) {
+        const CUtensorMap* map = g.p.shared ? (second ? &maps.shared_d : &maps.shared_gu)
+                                            : (second ? &maps.slots_d : &maps.slots_gu);
+        const char* pool = g.p.shared ? d.shared_blocks : d.slots;
+        // channel row of this group's first channel within the pool's tensor
+        const int row = (int)((g.p.base - pool) / ((size_t)3 * H * 2)) + g.blk * kTcBlockCh;
+        const int tiles = second ? G::kTiles : G::kChunks;
+        for (int t = 0; t < tiles && ok; ++t, ++n) {
+          const int s = n % NS;
+          if (n >= NS && (aborted() || !mbar_wait(empty + s, ((n / NS) - 1) & 1))) {
+            if (!aborted()) fail(kErrWaitEmpty);
+            ok = false;
+            break;
+          }
+          unsigned char* dst = ring + (size_t)s * kTileBytes;
+          mbar_expect_tx(full + s, kTileBytes);
+          if (!second) {
+            tma_load_3d(dst, map, t * 64, 0, row, full + s);
+          } else {
+            tma_load_3d(dst, map, t * 128, 2, row, full + s);
+            tma_load_3d(dst + kTileBytes / 2, map, t * 128 + 64, 2, row, full + s);
           }
         }
+      };
+      GroupWalk walk(a, n_items, ua, ub, j0);
+      GroupRec g, prev;
+      bool have_prev = false;
+      while (ok && walk.next(g)) {
+        emit(g, false);
+        if (have_prev && ok) emit(prev, true);
+        prev = g;
+        have_prev = true;
       }
+      if (have_prev && ok) emit(prev, true);
       if (!ok) {
         for (int m = max(0, n - NS); m < n; ++m)
           if (!mbar_wait(full + (m % NS), (m / NS) & 1)) atomicCAS(d.err, kErrNone, kErrDrain);
@@ -203,50 +243,60 @@ ffn_batched_tc_kernel(const __grid_constant__ BatchArgs a, const __grid_constant
   } else if (have_work && warp == 5) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      int n = 0, np = 0, ng = 0;
+      int n = 0;
       bool ok = true;
-      for (int j = j0; j < n_items && ok; ++j) {
-        if (a.plan[kPlanHeader + 4 * j + 3] >= ub) break;
-        PieceInfo p;
-        if (!make_piece(a, j, ua, ub, p)) continue;
-        ok = !aborted() && mbar_wait(x_full, np & 1);
-        if (ok && np > 0) ok = mbar_wait(d2_empty, (np - 1) & 1);
-        for (int blk = p.blk0; blk < p.blk1 && ok; ++blk, ++ng) {
-          if (ng > 0) ok = !aborted() && mbar_wait(d1_empty, (ng - 1) & 1);
-          for (int kc = 0; kc < G::kChunks && ok; ++kc, ++n) {
-            const int s = n % NS;
-            ok = !aborted() && mbar_wait(full + s, (n / NS) & 1);
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t a_addr = smem_u32(ring + (size_t)s * kTileBytes), b_addr = smem_u32(b1 + kc * 2048);
-#pragma unroll
-            for (int k = 0; k < 4; ++k)
-              umma(tmem, smem_desc(a_addr + k * 32, 16, 1024), smem_desc(b_addr + k * 32, 16, 1024), kIdescK,
-                   (kc | k) ? 1u : 0u);
-            umma_commit(empty + s);
-          }
+      // first contraction of a group into D1 buffer (idx & 1)
+      auto gemm1 = [&](const GroupRec& g) {
+        if (g.first) ok = !aborted() && mbar_wait(x_full, g.np & 1);
+        if (ok && g.idx >= 2) ok = !aborted() && mbar_wait(d1_empty + (g.idx & 1), ((g.idx >> 1) - 1) & 1);
+        const uint32_t dcol = tmem + (uint32_t)(g.idx & 1) * 16;
+        for (int kc = 0; kc < G::kChunks && ok; ++kc, ++n) {
+          const int s = n % NS;
+          ok = !aborted() && mbar_wait(full + s, (n / NS) & 1);
           if (!ok) break;
-          umma_commit(d1_full);
-          if (blk + 1 == p.blk1) umma_commit(x_empty);             // X^T of this piece is no longer needed
-          ok = !aborted() && mbar_wait(b2_full, ng & 1);
           tc_fence_after();
-          for (int ht = 0; ht < G::kTiles && ok; ++ht, ++n) {
-            const int s = n % NS;
-            ok = !aborted() && mbar_wait(full + s, (n / NS) & 1);
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t a_addr = smem_u32(ring + (size_t)s * kTileBytes), b_addr = smem_u32(b2);
+          const uint32_t a_addr = smem_u32(ring + (size_t)s * kTileBytes), b_addr = smem_u32(b1 + kc * 2048);
 #pragma unroll
-            for (int k = 0; k < 4; ++k)
-              umma(tmem + kD2Col + ht * 16, smem_desc(a_addr + k * 2048, 8192, 1024), smem_desc(b_addr + k * 32, 16, 1024),
-                   kIdescMN, (blk > p.blk0 || k) ? 1u : 0u);
-            umma_commit(empty + s);
-          }
-          if (!ok) break;
-          umma_commit(b2_empty);
+          for (int k = 0; k < 4; ++k)
+            umma(dcol, smem_desc(a_addr + k * 32, 16, 1024), smem_desc(b_addr + k * 32, 16, 1024), kIdescK,
+                 (kc | k) ? 1u : 0u);
+          umma_commit(empty + s);
         }
-        if (ok) { umma_commit(d2_full); ++np; }
+        if (!ok) return;
+        umma_commit(d1_full + (g.idx & 1));
+        if (g.last) umma_commit(x_empty);                          // X^T of this piece is no longer needed
+      };
+      // second contraction of a group into the piece's output tiles
+      auto gemm2 = [&](const GroupRec& g) {
+        ok = !aborted() && mbar_wait(b2_full, g.idx & 1);
+        if (ok && g.first && g.np > 0) ok = !aborted() && mbar_wait(d2_empty, (g.np - 1) & 1);
+        tc_fence_after();
+        for (int ht = 0; ht < G::kTiles && ok; ++ht, ++n) {
+          const int s = n % NS;
+          ok = !aborted() && mbar_wait(full + s, (n / NS) & 1);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t a_addr = smem_u32(ring + (size_t)s * kTileBytes), b_addr = smem_u32(b2);
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            umma(tmem + kD2Col + ht * 16, smem_desc(a_addr + k * 2048, 8192, 1024), smem_desc(b_addr + k * 32, 16, 1024),
+                 kIdescMN, (!g.first || k) ? 1u : 0u);
+          umma_commit(empty + s);
+        }
+        if (!ok) return;
+        umma_commit(b2_empty);
+        if (g.last) umma_commit(d2_full);
+      };
+      GroupWalk walk(a, n_items, ua, ub, j0);
+      GroupRec g, prev;
+      bool have_prev = false;
+      while (ok && walk.next(g)) {
+        gemm1(g);
+        if (have_prev && ok) gemm2(prev);
+        prev = g;
+        have_prev = true;
       }
+      if (have_prev && ok) gemm2(prev);
       if (!ok) {
         if (!aborted()) fail(kErrWaitFull);
         umma_commit(drain);                                       // let the tensor cores finish before TMEM is freed
@@ -255,26 +305,21 @@ ffn_batched_tc_kernel(const __grid_constant__ BatchArgs a, const __grid_constant
     }
   } else if (have_work) {
     // ------------------------------------------------------------- epilogue warps 0-3
-    int np = 0, ng = 0;
     bool ok = true;
     const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
-    for (int j = j0; j < n_items && ok; ++j) {
-      if (a.plan[kPlanHeader + 4 * j + 3] >= ub) break;
-      PieceInfo p;
-      if (!make_piece(a, j, ua, ub, p)) continue;
-      const int gidx = (p.l * BK + p.cand) * d.B + p.tile * kTcTokTile;
-      auto tok_of = [&](int t) -> int {
-        if (t >= p.n_tok) return -1;
-        return p.shared ? p.tile * kTcTokTile + t : d.grp_tok[gidx + t];
-      };
-      auto kq_of = [&](int t) -> int { return p.shared ? d.K + (p.cand - BK) : d.grp_k[gidx + t]; };
-
-      // X^T tile: 16 tokens x H as bf16, 128-byte rows per 64-column chunk, 16-byte pieces XORed with the row
-      if (np > 0) ok = !aborted() && mbar_wait(x_empty, (np - 1) & 1);
-      if (!ok) break;
+    auto tok_of = [&](const PieceInfo& p, int t) -> int {
+      if (t >= p.n_tok) return -1;
+      return p.shared ? p.tile * kTcTokTile + t : d.grp_tok[(p.l * BK + p.cand) * d.B + p.tile * kTcTokTile + t];
+    };
+    auto kq_of = [&](const PieceInfo& p, int t) -> int {
+      return p.shared ? d.K + (p.cand - BK) : d.grp_k[(p.l * BK + p.cand) * d.B + p.tile * kTcTokTile + t];
+    };
+    // X^T tile of a piece: 16 tokens x H as bf16, 128-byte rows per 64-column chunk, 16-byte pieces
+    // XORed with the row number (the 128-byte swizzle the MMA descriptors expect).
+    auto stage_x = [&](const PieceInfo& p) {
       for (int e = tid; e < kTcTokTile * (H / 8); e += 128) {
-        const int t = e / (H / 8), c8 = e % (H / 8);              // token, 8-column group
-        const int tok = tok_of(t);
+        const int t = e / (H / 8), c8 = e % (H / 8);
+        const int tok = tok_of(p, t);
         uint4 v = make_uint4(0u, 0u, 0u, 0u);
         if (tok >= 0) {
           const float4* src = reinterpret_cast<const float4*>(a.hidden_in + ((size_t)p.l * d.B + tok) * H + c8 * 8);
@@ -286,51 +331,28 @@ ffn_batched_tc_kernel(const __grid_constant__ BatchArgs a, const __grid_constant
       }
       proxy_fence();
       mbar_arrive(x_full);
-      // per-token scale of this piece (column j of the accumulators is token j of the tile)
-      float sc[kTcTokTile];
+    };
+    float sc[kTcTokTile];
+    auto load_scales = [&](const PieceInfo& p) {
 #pragma unroll
       for (int t = 0; t < kTcTokTile; ++t) {
-        const int tok = tok_of(t);
+        const int tok = tok_of(p, t);
         sc[t] = tok < 0 ? 0.f
                         : (p.shared ? d.shared_scale[p.l * d.B + tok]
-                                    : a.gates[((size_t)p.l * d.B + tok) * d.K + kq_of(t)]);
+                                    : a.gates[((size_t)p.l * d.B + tok) * d.K + kq_of(p, t)]);
       }
-
-      for (int blk = p.blk0; blk < p.blk1 && ok; ++blk, ++ng) {
-        ok = !aborted() && mbar_wait(d1_full, ng & 1);
-        if (!ok) break;
-        tc_fence_after();
-        float v[16];
-        tmem_ld16(tmem + lane_base, v);
-        tc_fence_before();
-        mbar_arrive(d1_empty);
-        if (ng > 0) ok = !aborted() && mbar_wait(b2_empty, (ng - 1) & 1);
-        if (!ok) break;
-        // lane 2c holds the gate row of channel c, lane 2c+1 its up row
-        const int ch = (warp * 32 + lane) >> 1;
-#pragma unroll
-        for (int t = 0; t < kTcTokTile; ++t) {
-          const float u = __shfl_down_sync(kFull, v[t], 1);
-          if ((lane & 1) == 0) {
-            const float av = v[t] / (1.f + __expf(-v[t])) * u * sc[t];
-            const uint32_t bits = pack_bf16(av, 0.f) & 0xffffu;
-            *reinterpret_cast<unsigned short*>(b2 + t * 128 + (((ch >> 3) ^ (t & 7)) << 4) + ((ch & 7) << 1)) =
-                (unsigned short)bits;
-          }
-        }
-        proxy_fence();
-        mbar_arrive(b2_full);
-      }
-      if (!ok) break;
-      // piece done: read the output tiles and write one stamped partial row per (token, rank)
-      ok = !aborted() && mbar_wait(d2_full, np & 1);
-      if (!ok) break;
+    };
+    // piece done: read the output tiles and write one stamped partial row per (token, rank)
+    auto read_out = [&](const GroupRec& g) {
+      ok = !aborted() && mbar_wait(d2_full, g.np & 1);
+      if (!ok) return;
       tc_fence_after();
       size_t rows[kTcTokTile];
 #pragma unroll
       for (int t = 0; t < kTcTokTile; ++t) {
-        const int tok = tok_of(t);
-        rows[t] = tok < 0 ? (size_t)-1 : (((size_t)p.l * d.B + tok) * P + kq_of(t)) * kUnitsPerItem + p.first_unit;
+        const int tok = tok_of(g.p, t);
+        rows[t] = tok < 0 ? (size_t)-1
+                          : (((size_t)g.p.l * d.B + tok) * P + kq_of(g.p, t)) * kUnitsPerItem + g.p.first_unit;
       }
       for (int ht = 0; ht < G::kTiles; ++ht) {
         float v[16];
@@ -345,7 +367,49 @@ ffn_batched_tc_kernel(const __grid_constant__ BatchArgs a, const __grid_constant
 #pragma unroll
       for (int t = 0; t < kTcTokTile; ++t)
         if (tid == t && rows[t] != (size_t)-1) a.flags[rows[t]] = a.step_id;
-      ++np;
+    };
+
+    GroupWalk walk(a, n_items, ua, ub, j0);
+    GroupRec g, gn;
+    bool have = walk.next(g);
+    if (have) stage_x(g.p);
+    while (have && ok) {
+      if (g.first) load_scales(g.p);
+      // activation step of group g: D1 buffer (idx & 1) -> a -> second B operand
+      ok = !aborted() && mbar_wait(d1_full + (g.idx & 1), (g.idx >> 1) & 1);
+      if (!ok) break;
+      tc_fence_after();
+      float v[16];
+      tmem_ld16(tmem + lane_base + (uint32_t)(g.idx & 1) * 16, v);
+      tc_fence_before();
+      mbar_arrive(d1_empty + (g.idx & 1));
+      if (g.idx > 0) ok = !aborted() && mbar_wait(b2_empty, (g.idx - 1) & 1);
+      if (!ok) break;
+      const int ch = (warp * 32 + lane) >> 1;       // lane 2c holds the gate row of channel c, lane 2c+1 its up row
+#pragma unroll
+      for (int t = 0; t < kTcTokTile; ++t) {
+        const float u = __shfl_down_sync(kFull, v[t], 1);
+        if ((lane & 1) == 0) {
+          const float av = v[t] / (1.f + __expf(-v[t])) * u * sc[t];
+          *reinterpret_cast<unsigned short*>(b2 + t * 128 + (((ch >> 3) ^ (t & 7)) << 4) + ((ch & 7) << 1)) =
+              (unsigned short)(pack_bf16(av, 0.f) & 0xffffu);
+        }
+      }
+      proxy_fence();
+      mbar_arrive(b2_full);
+
+      const bool have_next = walk.next(gn);
+      if (g.last) {
+        if (have_next) {
+          // the next piece's X^T may replace this one's as soon as its last first-contraction is done
+          ok = !aborted() && mbar_wait(x_empty, g.np & 1);
+          if (!ok) break;
+          stage_x(gn.p);
+        }
+        read_out(g);
+      }
+      have = have_next;
+      g = gn;
     }
     if (!ok && !aborted()) fail(kErrWaitFull);
   }
