@@ -85,6 +85,16 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
 #pragma unroll
   for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
+// The same load without the wait: the caller issues several, then one tcgen05.wait::ld, and only
+// then reads the values.
+__device__ __forceinline__ void tmem_ld16_nowait(uint32_t taddr, float* v) {
+  uint32_t* r = reinterpret_cast<uint32_t*>(v);
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   uint32_t r;
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
@@ -317,17 +327,29 @@ ffn_batched_tc_kernel(const __grid_constant__ BatchArgs a, const __grid_constant
     // X^T tile of a piece: 16 tokens x H as bf16, 128-byte rows per 64-column chunk, 16-byte pieces
     // XORed with the row number (the 128-byte swizzle the MMA descriptors expect).
     auto stage_x = [&](const PieceInfo& p) {
-      for (int e = tid; e < kTcTokTile * (H / 8); e += 128) {
-        const int t = e / (H / 8), c8 = e % (H / 8);
+      constexpr int kPer = (H / 8 + 127) / 128;         // 16-byte pieces per thread and token
+#pragma unroll 2
+      for (int t = 0; t < kTcTokTile; ++t) {
         const int tok = tok_of(p, t);
-        uint4 v = make_uint4(0u, 0u, 0u, 0u);
-        if (tok >= 0) {
-          const float4* src = reinterpret_cast<const float4*>(a.hidden_in + ((size_t)p.l * d.B + tok) * H + c8 * 8);
-          const float4 x0 = __ldg(src), x1 = __ldg(src + 1);
-          v = make_uint4(pack_bf16(x0.x, x0.y), pack_bf16(x0.z, x0.w), pack_bf16(x1.x, x1.y), pack_bf16(x1.z, x1.w));
+        float4 x[kPer][2];
+#pragma unroll
+        for (int i = 0; i < kPer; ++i) {
+          x[i][0] = x[i][1] = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (tok >= 0 && tid + 128 * i < H / 8) {
+            const float4* src =
+                reinterpret_cast<const float4*>(a.hidden_in + ((size_t)p.l * d.B + tok) * H + (tid + 128 * i) * 8);
+            x[i][0] = __ldg(src);
+            x[i][1] = __ldg(src + 1);
+          }
         }
-        const int kc = c8 >> 3, c = c8 & 7;
-        *reinterpret_cast<uint4*>(b1 + kc * 2048 + t * 128 + ((c ^ (t & 7)) << 4)) = v;
+#pragma unroll
+        for (int i = 0; i < kPer; ++i) {
+          const int c8 = tid + 128 * i, kc = c8 >> 3, c = c8 & 7;
+          if (c8 < H / 8)
+            *reinterpret_cast<uint4*>(b1 + kc * 2048 + t * 128 + ((c ^ (t & 7)) << 4)) =
+              make_uint4(pack_bf16(x[i][0].x, x[i][0].y), pack_bf16(x[i][0].z, x[i][0].w),
+                         pack_bf16(x[i][1].x, x[i][1].y), pack_bf16(x[i][1].z, x[i][1].w));
+        }
       }
       proxy_fence();
       mbar_arrive(x_full);
@@ -354,13 +376,19 @@ ffn_batched_tc_kernel(const __grid_constant__ BatchArgs a, const __grid_constant
         rows[t] = tok < 0 ? (size_t)-1
                           : (((size_t)g.p.l * d.B + tok) * P + kq_of(g.p, t)) * kUnitsPerItem + g.p.first_unit;
       }
-      for (int ht = 0; ht < G::kTiles; ++ht) {
-        float v[16];
-        tmem_ld16(tmem + lane_base + kD2Col + ht * 16, v);
-        const int h = ht * 128 + warp * 32 + lane;
+      constexpr int kBatch = G::kTiles >= 4 ? 4 : G::kTiles;
+      for (int ht0 = 0; ht0 < G::kTiles; ht0 += kBatch) {
+        float v[kBatch][16];
 #pragma unroll
-        for (int t = 0; t < kTcTokTile; ++t)
-          if (rows[t] != (size_t)-1) a.part[rows[t] * H + h] = v[t];
+        for (int i = 0; i < kBatch; ++i) tmem_ld16_nowait(tmem + lane_base + kD2Col + (ht0 + i) * 16, v[i]);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+        for (int i = 0; i < kBatch; ++i) {
+          const int h = (ht0 + i) * 128 + warp * 32 + lane;
+#pragma unroll
+          for (int t = 0; t < kTcTokTile; ++t)
+            if (rows[t] != (size_t)-1) a.part[rows[t] * H + h] = v[i][t];
+        }
       }
       tc_fence_before();
       mbar_arrive(d2_empty);
