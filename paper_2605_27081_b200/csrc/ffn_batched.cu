@@ -276,12 +276,15 @@ __global__ void __launch_bounds__(256) combine_batched_kernel(BatchArgs a, float
 
 template <int H>
 cudaError_t launch_one(const BatchArgs& a, int grid, cudaStream_t st) {
-  static bool configured = false;
-  if (!configured) {
+  // the dynamic shared-memory limit is a per-device attribute of the kernel
+  static bool configured[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  if (!configured[dev]) {
     cudaError_t e = cudaFuncSetAttribute(ffn_batched_kernel<H>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)Geo<H>::kSmem);
     if (e != cudaSuccess) return e;
-    configured = true;
+    configured[dev] = true;
   }
   BatchArgs b = a;
   b.tok_tile = kTokTile;

@@ -474,12 +474,15 @@ bool encode_pool(EncodeTiledFn encode, CUtensorMap* gu, CUtensorMap* dn, const v
 
 template <int H>
 cudaError_t launch_tc(const BatchArgs& a, const TcMaps& maps, int grid, cudaStream_t st) {
-  static bool configured = false;
-  if (!configured) {
+  // the dynamic shared-memory limit is a per-device attribute of the kernel
+  static bool configured[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  if (!configured[dev]) {
     cudaError_t e = cudaFuncSetAttribute(ffn_batched_tc_kernel<H>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)TcGeo<H>::kSmem);
     if (e != cudaSuccess) return e;
-    configured = true;
+    configured[dev] = true;
   }
   BatchArgs b = a;
   b.tok_tile = kTcTokTile;

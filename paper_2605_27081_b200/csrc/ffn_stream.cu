@@ -320,12 +320,15 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const float* __restrict__ 
 template <int WB, int H>
 cudaError_t launch_one(const FfnArgs& a, int grid, cudaStream_t st) {
   const Layout lay = make_layout(H, WB);
-  static bool configured = false;
-  if (!configured) {
+  // the dynamic shared-memory limit is a per-device attribute of the kernel
+  static bool configured[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  if (!configured[dev]) {
     cudaError_t e = cudaFuncSetAttribute(ffn_stream_kernel<WB, H>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)lay.total);
     if (e != cudaSuccess) return e;
-    configured = true;
+    configured[dev] = true;
   }
   ffn_stream_kernel<WB, H><<<grid, kThreads, lay.total, st>>>(a);
   return cudaGetLastError();
