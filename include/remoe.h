@@ -64,7 +64,8 @@ typedef struct {
                          /* REMOE_FP8_E4M3: expert blocks are OCP FP8 E4M3 bytes, value =  */
                          /* byte * 2^-8; router and shared gate bf16; H multiple of 512;   */
                          /* batch 1 only (halves the bytes a miss moves over the host link)*/
-  int32_t batch;         /* B sequences per step                                           */
+  int32_t batch;         /* B sequences per step; B > 1 needs bf16 weights and I, I_shared  */
+                         /* multiples of 8, B * K <= 1024                                   */
 } remoe_shape;
 
 /* Counters of App. E.2.3-E.2.4, summed over steps since creation or the last reset. */
@@ -116,6 +117,10 @@ int remoe_load_experts_host(remoe_stack*, int32_t layer, int32_t first_expert, i
  * least recently used) on the copy stream while resident experts are already computed.
  * The call blocks only until the step's miss list is known; on return the remaining work
  * is enqueued and the outputs are complete once the stack's stream has drained.
+ * With B > 1 the cache is shared by the batch: the step's distinct requests U = Unique(R)
+ * (App. E.2.3) are resolved together, tokens are grouped per expert and the experts run as a
+ * tensor-core grouped GEMM (activations rounded to bf16, fp32 accumulation); if U has more
+ * experts than there are slots, slots are handed on within the step in request order.
  * Errors: ARG, NOT_LOADED, CUDA, DEVICE_FLAG.
  */
 int remoe_decode_step(remoe_stack*, const float* hidden_in_dev, float* hidden_out_dev,
