@@ -172,13 +172,13 @@ int remoe_reuse_stats(remoe_stack*, int32_t layer, uint64_t* overlap_sum,
  * [L, B] or [B], may be NULL) = m_t of the most recent step, -1 where t = 1. */
 int remoe_reuse_mass(remoe_stack*, int32_t layer, double* mass_sum, uint64_t* pairs, float* last_mass);
 
-/* Per-step aggregates over all layers since the last reset (App. E.2.5): for steps first ..
+/* Per-step aggregates over all layers since the last reset (App. E.2.6): for steps first ..
  * first+count-1, umiss[i] = #uMiss^(all) of the step and tok_hits[i] = H_tok^(all) (either may be
  * NULL); n_steps receives how many steps are recorded.  Host-side bookkeeping, no device work. */
 int remoe_step_history(remoe_stack*, int32_t first, int32_t count, uint32_t* umiss, uint32_t* tok_hits,
                        int32_t* n_steps);
 
-/* I/O-time and TPOT proxy of App. E.2.5 / E.3: io_ms[i] = umiss[i] * expert_bytes / bandwidth * 1000
+/* I/O-time and TPOT proxy of App. E.2.6 / F.1: io_ms[i] = umiss[i] * expert_bytes / bandwidth * 1000
  * with bandwidth_gbps in 10^9 bytes/s, TPOT_i = tpot_compute_ms + io_ms[i] / batch.  io_ms ([n], may
  * be NULL) receives the per-step I/O time, tpot_p50_p95_p99 ([3], may be NULL) the percentiles of
  * TPOT over the n steps (linear interpolation between order statistics).  Pure host arithmetic. */

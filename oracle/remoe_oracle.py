@@ -42,8 +42,9 @@ counting definition and constructed ties, LRU/FIFO/LFU against hand-worked slot 
 against the set characterisation "the C most recently used distinct experts" recomputed from
 the whole history, the exact identity misses(t) = K - |E_t n E_{t-1}| when C = K (App. A.3
 "Tightness"), both fetch bounds, Belady against exhaustive search, counters against their
-totals and against the uHR / #uMiss table the paper prints (App. E.3), the TPOT proxy against
-the slope of the paper's TPOT table, the FFN against a hand example and a library matmul in the
+totals and against the uHR / #uMiss table the paper prints (App. F.1), the TPOT proxy against
+the slope of the paper's TPOT table, the load entropy and CV against closed forms and the
+(entropy, CV) pairs the paper prints, the FFN against a hand example and a library matmul in the
 N = K = 1 case, dense-and-mask against selected-only, linearity in the gate weights, the
 chained mode against its telescoping sum and hand-run one-layer stacks.  Every function has at
 least one such pin, so none is "parity unpinned"; but the paper prints no worked numeric
@@ -111,12 +112,12 @@ def reuse_mass(p_t, e_prev, k):
 
 
 def io_ms_step(umiss, expert_bytes, bandwidth_gbps):
-    """IO_ms_step = #uMiss * expert_bytes / bandwidth * 1000, bandwidth in 1e9 bytes/s (App. E.2.5)."""
+    """IO_ms_step = #uMiss * expert_bytes / bandwidth * 1000, bandwidth in 1e9 bytes/s (App. E.2.6)."""
     return np.asarray(umiss, dtype=F64) * float(expert_bytes) / (float(bandwidth_gbps) * 1e9) * 1000.0
 
 
 def tpot_proxy(umiss, expert_bytes, bandwidth_gbps, batch=1, tpot_compute_ms=0.0):
-    """TPOT ~ TPOT_compute + IO_step / B per step (App. E.3), and its P50/P95/P99 over the steps
+    """TPOT ~ TPOT_compute + IO_step / B per step (App. F.1), and its P50/P95/P99 over the steps
     (linear interpolation between order statistics; the paper does not say which rule it uses)."""
     tpot = tpot_compute_ms + io_ms_step(umiss, expert_bytes, bandwidth_gbps) / batch
     srt = sorted(float(x) for x in tpot)
@@ -127,6 +128,35 @@ def tpot_proxy(umiss, expert_bytes, bandwidth_gbps, batch=1, tpot_compute_ms=0.0
         hi = min(lo + 1, len(srt) - 1)
         out.append(srt[lo] + (pos - lo) * (srt[hi] - srt[lo]))
     return tpot, out
+
+
+def load_entropy(counts):
+    """Normalised routing entropy: H(p) / log N of the empirical load distribution p_e = n_e / sum n,
+    n_e = how often expert e was selected (Sec. 4.4 "Routing imbalance"; Sec. 5.2, table of routing
+    metrics).  The
+    paper prints the numbers without a formula; this reading is the one its own (entropy, CV) pairs
+    satisfy: near balance H / log N = 1 - CV^2 / (2 log N) + O(CV^3).  1 = perfectly even load."""
+    n = np.asarray(counts, dtype=F64)
+    tot = float(n.sum())
+    if tot <= 0.0 or n.size < 2:
+        return 1.0
+    h = 0.0
+    for v in n:                                   # 0 log 0 = 0
+        if v > 0.0:
+            q = float(v) / tot
+            h -= q * np.log(q)
+    return float(h / np.log(float(n.size)))
+
+
+def load_cv(counts):
+    """Load-balance coefficient of variation: population standard deviation of the per-expert
+    selection counts over their mean (Sec. 4.4 "Routing imbalance"; Sec. 5.2).  0 = perfectly even load."""
+    n = np.asarray(counts, dtype=F64)
+    mean = float(n.sum()) / n.size
+    if mean <= 0.0:
+        return 0.0
+    var = float(((n - mean) ** 2).sum()) / n.size
+    return float(np.sqrt(var) / mean)
 
 
 def reuse_overlap(e_t, e_prev):
@@ -314,7 +344,8 @@ class OracleStack:
         self.overlap_sum = [0] * L
         self.pairs_counted = [0] * L
         self.mass_sum = [0.0] * L
-        self.hist_umiss = []          # per step, summed over layers (App. E.2.5)
+        self.load = [[0] * self.s.n_routed for _ in range(L)]   # selections per expert (token level)
+        self.hist_umiss = []          # per step, summed over layers (App. E.2.6)
         self.hist_tok_hits = []
         self.steps = 0
 
@@ -376,6 +407,8 @@ class OracleStack:
                 ids, g, margin, _, p = self.route(l, hl[b], ov)
                 res["ids"][l, b], res["gates"][l, b], res["margin"][l, b] = ids, g, margin
                 flat.extend(int(e) for e in ids)
+                for e in ids:
+                    self.load[l][int(e)] += 1
                 if self.prev[l][b] is not None:                       # Eq. (1), t >= 2
                     ov_n = reuse_overlap(ids, self.prev[l][b])
                     res["overlap"][l, b] = ov_n
@@ -429,6 +462,21 @@ class OracleStack:
         h = sum(self.tok_hits[l] for l in ls)
         m = sum(self.tok_misses[l] for l in ls)
         return h / (h + m) if h + m else 0.0
+
+    def routing_entropy(self, layer=None):
+        """Normalised load entropy of one layer, or its mean over the layers."""
+        ls = range(self.s.n_layers) if layer is None else [layer]
+        return sum(load_entropy(self.load[l]) for l in ls) / len(ls)
+
+    def routing_cv(self, layer=None):
+        """Load-balance CV of one layer, or its mean over the layers."""
+        ls = range(self.s.n_layers) if layer is None else [layer]
+        return sum(load_cv(self.load[l]) for l in ls) / len(ls)
+
+    def experts_visited(self, layer=None):
+        """Distinct experts selected at least once in one layer, or the mean over the layers."""
+        ls = range(self.s.n_layers) if layer is None else [layer]
+        return sum(sum(1 for v in self.load[l] if v > 0) for l in ls) / len(ls)
 
     def eor(self, layer=None):
         ls = range(self.s.n_layers) if layer is None else [layer]

@@ -248,7 +248,7 @@ int decode_step_batched(remoe_stack* s, const float* hin, float* hout, int32_t* 
   if (check_device_flag(s) != REMOE_OK) return REMOE_E_DEVICE_FLAG;
 
   {
-    // per-step all-layer aggregates (App. E.2.5)
+    // per-step all-layer aggregates (App. E.2.6)
     const int* th = trace_tok_hits(s->host_block + 1, d.L, s->BK);
     const int* nu = trace_n_unique(s->host_block + 1);
     const int* hh = trace_hit(s->host_block + 1, d.L, s->BK);
@@ -570,7 +570,7 @@ int remoe_decode_step(remoe_stack* s, const float* hin, float* hout, int32_t* id
   if (check_device_flag(s) != REMOE_OK) return REMOE_E_DEVICE_FLAG;
 
   {
-    // per-step all-layer aggregates (App. E.2.5)
+    // per-step all-layer aggregates (App. E.2.6)
     const int* th = trace_tok_hits(s->host_block + 1, d.L, s->BK);
     const int* nu = trace_n_unique(s->host_block + 1);
     const int* hh = trace_hit(s->host_block + 1, d.L, s->BK);

@@ -158,7 +158,7 @@ class StepChecker:
             assert (ov, pairs) == (o.overlap_sum[l], o.pairs_counted[l])
         ov, pairs = st.reuse_stats(-1)
         assert (ov, pairs) == (sum(o.overlap_sum), sum(o.pairs_counted))
-        # reporting: reuse mass (Eq. 2), per-step aggregates and the TPOT proxy (App. E.2.5)
+        # reporting: reuse mass (Eq. 2), per-step aggregates and the TPOT proxy (App. E.2.6)
         from paper_2605_27081_b200 import binding as B
         m, p = st.reuse_mass(-1)
         assert p == sum(o.pairs_counted) and abs(m - sum(o.mass_sum)) <= 1e-5 * max(1.0, p)

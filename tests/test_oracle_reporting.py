@@ -1,5 +1,5 @@
 """Pins for the reporting pieces: reuse mass (Eq. 2), #uMiss/uHR aggregates (App. E.2.4), the I/O-time
-and TPOT proxy (App. E.2.5, E.3)."""
+and TPOT proxy (App. E.2.6, F.1), routing entropy and load-balance CV (Sec. 4.4, 5.2)."""
 import os
 
 import numpy as np
@@ -11,6 +11,15 @@ GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "paper_cache_tables.t
 TOTAL_REQUESTS = 128 * 64 * 26 * 6
 
 
+def _balance_rows():
+    rows = []
+    for line in open(GOLDEN):
+        c = [x.strip() for x in line.strip().split("|")]
+        if c[0] == "balance":
+            rows.append((int(c[1]), float(c[2]), float(c[3])))
+    return rows
+
+
 def _tables():
     cache, tpot = {}, {}
     for line in open(GOLDEN):
@@ -18,6 +27,8 @@ def _tables():
         if not line or line.startswith("#"):
             continue
         c = [x.strip() for x in line.split("|")]
+        if c[0] == "balance":
+            continue
         if c[0] == "tpot50":
             tpot[int(c[1])] = (float(c[2]), float(c[3]))
         else:
@@ -97,3 +108,67 @@ def test_stack_tracks_mass_and_history():
         prev = r["ids"].copy()
     assert len(st.hist_umiss) == 12 and sum(st.hist_umiss) == sum(st.uniq_misses)
     assert sum(st.hist_tok_hits) == sum(st.tok_hits)
+
+
+def test_load_entropy_and_cv_closed_forms():
+    n = 64
+    assert abs(orc.load_entropy([7] * n) - 1.0) < 1e-12 and orc.load_cv([7] * n) == 0.0
+    one_hot = [0] * n
+    one_hot[5] = 123
+    assert abs(orc.load_entropy(one_hot)) < 1e-15
+    assert abs(orc.load_cv(one_hot) - np.sqrt(n - 1)) < 1e-12
+    # m of N experts share the load evenly: entropy log m / log N, CV sqrt(N / m - 1)
+    for m in (2, 16, 48):
+        c = [3] * m + [0] * (n - m)
+        assert abs(orc.load_entropy(c) - np.log(m) / np.log(n)) < 1e-12
+        assert abs(orc.load_cv(c) - np.sqrt(n / m - 1)) < 1e-12
+    # half the experts at mean * (1 + c), half at mean * (1 - c): CV = c exactly and
+    # H = log N - ((1 + c) log(1 + c) + (1 - c) log(1 - c)) / 2
+    for c in (0.0409, 0.1608, 0.5):
+        counts = [round(1e6 * (1 + c))] * 32 + [round(1e6 * (1 - c))] * 32
+        assert abs(orc.load_cv(counts) - c) < 1e-9
+        h = 1.0 - ((1 + c) * np.log(1 + c) + (1 - c) * np.log(1 - c)) / (2 * np.log(64))
+        assert abs(orc.load_entropy(counts) - h) < 1e-9
+    # invariances: scale of the counts, order of the experts
+    rng = np.random.default_rng(3)
+    v = rng.integers(1, 1000, size=60)
+    assert abs(orc.load_entropy(v) - orc.load_entropy(3 * v)) < 1e-12
+    assert abs(orc.load_cv(v) - orc.load_cv(rng.permutation(v) * 5)) < 1e-12
+    assert abs(orc.load_cv(v) - np.std(v) / np.mean(v)) < 1e-12
+    assert orc.load_entropy([0] * 8) == 1.0 and orc.load_cv([0] * 8) == 0.0        # nothing routed yet
+
+
+def test_entropy_and_cv_readings_fit_the_pairs_the_paper_prints():
+    """The paper prints entropy and CV without formulas.  With entropy read as H(load) / log N and CV
+    as std / mean of the per-expert load, the two are tied near balance by
+    H / log N = 1 - CV^2 / (2 log N) + O(CV^3); every printed pair obeys that to its last digit or
+    two, for both expert counts.  (A per-token softmax entropy, an unnormalised entropy or a CV of
+    something other than the load would not.)"""
+    rows = _balance_rows()
+    assert len(rows) == 8
+    for n, ent, cv in rows:
+        assert abs(ent - (1.0 - cv * cv / (2.0 * np.log(n)))) < (6e-5 if cv < 0.06 else 4e-4)
+    # and the oracle's own functions obey the same relation on a mildly perturbed load
+    rng = np.random.default_rng(7)
+    counts = np.round(1e5 * (1 + 0.1 * rng.standard_normal(64))).astype(np.int64)
+    cv = orc.load_cv(counts)
+    assert abs(orc.load_entropy(counts) - (1.0 - cv * cv / (2 * np.log(64)))) < 2e-4
+
+
+def test_stack_counts_the_load_per_expert():
+    shape = synth.Shape(2, 64, 16, 3, 8, batch=2)
+    routers = [synth.gen_router(0, shape, l) for l in range(2)]
+    st = orc.OracleStack(shape, 6, routers)
+    hs = synth.HiddenStream(0, shape, 0.6)
+    tally = np.zeros((2, 16), np.int64)
+    for t in range(20):
+        r = st.step(hs.step(), ffn=None)
+        for l in range(2):
+            for e in r["ids"][l].reshape(-1):
+                tally[l, e] += 1
+    assert (np.asarray(st.load) == tally).all() and tally.sum() == 20 * 2 * 2 * 3
+    assert abs(st.routing_entropy() - (orc.load_entropy(tally[0]) + orc.load_entropy(tally[1])) / 2) < 1e-15
+    assert abs(st.routing_cv(1) - np.std(tally[1]) / np.mean(tally[1])) < 1e-12
+    assert st.experts_visited(0) == (tally[0] > 0).sum()
+    st.reset()
+    assert np.asarray(st.load).sum() == 0
