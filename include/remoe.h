@@ -127,18 +127,19 @@ int remoe_decode_step(remoe_stack*, const float* hidden_in_dev, float* hidden_ou
                       int32_t* selected_ids_dev, float* gate_weights_dev);
 
 /*
- * Chained variant of the step (batch 1): the layers feed each other through a pre-norm residual
- * connection as in a decoder stack, x_l = h_l / sqrt(mean(h_l^2) + 1e-6), h_{l+1} = h_l + MoE_l(x_l),
- * instead of each reading its own stream (the paper treats layers independently, App. A.5;
- * chaining is how they sit in a model; without the norm a randomly initialised stack diverges).
- *   hidden_in    dev [H]        h_0
- *   hidden_out   dev [H]        h_L
- *   layer_inputs dev [L, H]     residual stream h_0 .. h_{L-1} (may be NULL)
- *   selected_ids dev [L, K], gate_weights dev [L, K]
+ * Chained variant of the step: the layers feed each other through a pre-norm residual connection as
+ * in a decoder stack, x_l = h_l / sqrt(mean(h_l^2) + 1e-6), h_{l+1} = h_l + MoE_l(x_l), instead of
+ * each reading its own stream (the paper treats layers independently, App. A.5; chaining is how they
+ * sit in a model; without the norm a randomly initialised stack diverges).
+ *   hidden_in    dev [B, H]        h_0
+ *   hidden_out   dev [B, H]        h_L
+ *   layer_inputs dev [L, B, H]     residual stream h_0 .. h_{L-1} (may be NULL)
+ *   selected_ids dev [L, B, K], gate_weights dev [L, B, K]
  * Routing of layer l+1 depends on layer l's output, so the host waits for one small trace per
  * layer instead of one per step, and a layer's fetches cannot start before the layer above it
- * has finished.  Cache, counters and reuse statistics behave exactly as in remoe_decode_step.
- * Errors: ARG, NOT_LOADED, UNSUPPORTED (batch > 1), CUDA, DEVICE_FLAG.
+ * has finished.  With B > 1 the sequences move through the layers together and share each layer's
+ * cache as in remoe_decode_step.  Cache, counters and reuse statistics behave exactly as in
+ * remoe_decode_step.  Errors: ARG, NOT_LOADED, CUDA, DEVICE_FLAG.
  */
 int remoe_decode_step_chained(remoe_stack*, const float* hidden_in_dev, float* hidden_out_dev,
                               float* layer_inputs_dev, int32_t* selected_ids_dev, float* gate_weights_dev);
@@ -171,6 +172,18 @@ int remoe_reuse_stats(remoe_stack*, int32_t layer, uint64_t* overlap_sum,
  * sequence) pairs of the layer (layer = -1: all layers), pairs = their number, last_mass (host,
  * [L, B] or [B], may be NULL) = m_t of the most recent step, -1 where t = 1. */
 int remoe_reuse_mass(remoe_stack*, int32_t layer, double* mass_sum, uint64_t* pairs, float* last_mass);
+
+/* Expert load since the last reset (Sec. 4.4 "Routing imbalance"; Sec. 5.2 reports entropy and CV of
+ * the routing).  counts (host, [N] for one layer, [L, N] for layer = -1, may be NULL) receives how
+ * often each routed expert was selected (token level: B*K selections per layer-step).  From them,
+ * per layer: the normalised entropy H(p) / log N of the load distribution p_e = n_e / sum n (1 = even
+ * load), the coefficient of variation std(n) / mean(n) with the population standard deviation (0 =
+ * even load), and the number of experts selected at least once.  With layer = -1 the three figures
+ * are means over the layers (visited rounded down).  Before any step: entropy 1, cv 0, visited 0.
+ * The paper prints entropy and CV without formulas; these definitions reproduce the relation its
+ * printed pairs obey.  Any output may be NULL.  Waits for the stack's stream. */
+int remoe_expert_load(remoe_stack*, int32_t layer, uint64_t* counts, double* norm_entropy, double* cv,
+                      int32_t* experts_visited);
 
 /* Per-step aggregates over all layers since the last reset (App. E.2.6): for steps first ..
  * first+count-1, umiss[i] = #uMiss^(all) of the step and tok_hits[i] = H_tok^(all) (either may be

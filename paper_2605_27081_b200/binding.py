@@ -26,6 +26,7 @@ EXPORTS = [
     "remoe_reuse_stats", "remoe_cache_reset", "remoe_set_policy", "remoe_set_reroute_beta",
     "remoe_set_profiling", "remoe_kernel_time", "remoe_launch_count", "remoe_last_cuda_error", "remoe_stack_destroy",
     "remoe_strerror", "remoe_expert_ffn_static", "remoe_reuse_mass", "remoe_step_history", "remoe_tpot_proxy", "remoe_decode_step_chained",
+    "remoe_expert_load",
 ]
 
 
@@ -79,6 +80,7 @@ def lib():
                                               vp, vp, vp]
         L.remoe_reuse_mass.argtypes = [vp, i32, C.POINTER(C.c_double), C.POINTER(C.c_uint64), vp]
         L.remoe_step_history.argtypes = [vp, i32, i32, vp, vp, C.POINTER(i32)]
+        L.remoe_expert_load.argtypes = [vp, i32, vp, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(i32)]
         L.remoe_tpot_proxy.argtypes = [vp, i32, C.c_uint64, C.c_double, i32, C.c_double, vp, vp]
         L.remoe_last_cuda_error.argtypes = [vp]
         L.remoe_last_cuda_error.restype = C.c_char_p
@@ -215,6 +217,12 @@ def remoe_reuse_mass(h, layer=-1, last_mass=None):
     return rc, float(m.value), int(p.value)
 
 
+def remoe_expert_load(h, layer=-1, counts=None):
+    ent, cv, seen = C.c_double(), C.c_double(), C.c_int32()
+    rc = lib().remoe_expert_load(h, int(layer), _ptr(counts), C.byref(ent), C.byref(cv), C.byref(seen))
+    return rc, float(ent.value), float(cv.value), int(seen.value)
+
+
 def remoe_step_history(h, first=0, count=None):
     n = C.c_int32()
     rc = lib().remoe_step_history(h, 0, 0, None, None, C.byref(n))
@@ -304,6 +312,14 @@ class Stack:
         rc, m, p = remoe_reuse_mass(self.h, layer, last)
         self._ck(rc, "remoe_reuse_mass")
         return (m, p, last) if want_last else (m, p)
+
+    def expert_load(self, layer=-1):
+        """(counts [L, N] or [N] uint64, normalised entropy, CV, experts visited)."""
+        n = self.shape.n_routed * (self.shape.n_layers if layer < 0 else 1)
+        counts = np.zeros(n, np.uint64)
+        rc, ent, cv, seen = remoe_expert_load(self.h, layer, counts)
+        self._ck(rc, "remoe_expert_load")
+        return (counts.reshape(-1, self.shape.n_routed) if layer < 0 else counts), ent, cv, seen
 
     def step_history(self, first=0, count=None):
         rc, um, th = remoe_step_history(self.h, first, count)

@@ -15,6 +15,7 @@
 #include "remoe_internal.cuh"
 
 #include <algorithm>
+#include <cmath>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -129,6 +130,7 @@ int reset_state(remoe_stack* s) {
   CK(cudaMemsetAsync(d.clock, 0, L * sizeof(unsigned long long), s->stream));
   CK(cudaMemsetAsync(d.prev_mask, 0, L * d.B * kMaskWords * sizeof(unsigned), s->stream));
   CK(cudaMemsetAsync(d.counters, 0, L * kCounters * sizeof(unsigned long long), s->stream));
+  CK(cudaMemsetAsync(d.load, 0, L * d.N * sizeof(unsigned long long), s->stream));
   CK(cudaMemsetAsync(d.last_overlap, 0xff, L * d.B * sizeof(int), s->stream));
   CK(cudaMemsetAsync(d.last_mass, 0, L * d.B * sizeof(float), s->stream));
   CK(cudaMemsetAsync(d.mass_sum, 0, L * d.B * sizeof(double), s->stream));
@@ -209,12 +211,101 @@ cudaError_t launch_batched(remoe_stack* s, const BatchArgs& a) {
                    : launch_ffn_batched(a, s->grid, s->stream);
 }
 
+// Validates the trace of layers [l0, l1) and runs their miss waves: copies queued depth by depth, layer
+// by layer; each (depth, layer) group computed once its copies have landed.  The resident-phase launch
+// covering these layers must already be enqueued with ev_resident recorded behind it.  Adds the
+// algorithmic bytes of that launch to *resident_bytes.
+int batched_waves(remoe_stack* s, BatchArgs& a, int l0, int l1, uint64_t* resident_bytes) {
+  DevStack& d = s->d;
+  const int BK = s->BK;
+  int* tr = s->host_block + 1;
+  const int* t_nu = trace_n_unique(tr);
+  const int* t_req = trace_requests(tr, d.L, BK);
+  const int* t_hit = trace_hit(tr, d.L, BK);
+  const int* t_slot = trace_slot(tr, d.L, BK);
+  const int* t_depth = trace_depth(tr, d.L, BK);
+  int max_depth = -1;
+  for (int l = l0; l < l1; ++l) {
+    if (t_nu[l] < 0 || t_nu[l] > BK) return REMOE_E_DEVICE_FLAG;
+    for (int i = 0; i < t_nu[l]; ++i) {
+      const int j = l * BK + i;
+      if (t_hit[j]) { *resident_bytes += d.slot_bytes; continue; }
+      if (t_req[j] < 0 || t_req[j] >= d.N || t_slot[j] < 0 || t_slot[j] >= d.C || t_depth[j] < 0)
+        return REMOE_E_DEVICE_FLAG;
+      if (t_depth[j] > max_depth) max_depth = t_depth[j];
+    }
+    *resident_bytes += (uint64_t)d.S * d.shared_bytes;   // algorithmic: once, although every token tile streams it
+  }
+
+  // events: [depth][layer] copy-done and compute-done
+  const size_t need = (size_t)2 * (max_depth + 1) * d.L;
+  while (s->ev_pool.size() < need) {
+    cudaEvent_t e;
+    CK(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+    s->ev_pool.push_back(e);
+  }
+  auto ev_copy = [&](int dep, int l) { return s->ev_pool[((size_t)dep * d.L + l) * 2]; };
+  auto ev_comp = [&](int dep, int l) { return s->ev_pool[((size_t)dep * d.L + l) * 2 + 1]; };
+  std::vector<char> had(((size_t)max_depth + 2) * d.L, 0);
+
+  if (max_depth >= 0) CK(cudaStreamWaitEvent(s->copy_stream, s->ev_trace, 0));
+  for (int dep = 0; dep <= max_depth; ++dep) {
+    if (dep == 1) CK(cudaStreamWaitEvent(s->copy_stream, s->ev_resident, 0));   // displaced hits are done
+    for (int l = l0; l < l1; ++l) {
+      int misses = 0;
+      for (int i = 0; i < t_nu[l]; ++i) {
+        const int j = l * BK + i;
+        if (t_hit[j] || t_depth[j] != dep) continue;
+        if (!misses && dep >= 1 && had[(size_t)(dep - 1) * d.L + l])
+          CK(cudaStreamWaitEvent(s->copy_stream, ev_comp(dep - 1, l), 0));        // displaced misses are done
+        CK(cudaMemcpyAsync(d.slots + ((size_t)l * d.C + t_slot[j]) * d.slot_bytes,
+                           s->host_ptrs[(size_t)l * d.N + t_req[j]], d.slot_bytes, cudaMemcpyHostToDevice,
+                           s->copy_stream));
+        ++misses;
+      }
+      if (!misses) continue;
+      had[(size_t)dep * d.L + l] = 1;
+      s->h2d_bytes[l] += (uint64_t)misses * d.slot_bytes;
+      CK(cudaEventRecord(ev_copy(dep, l), s->copy_stream));
+    }
+    for (int l = l0; l < l1; ++l) {
+      if (!had[(size_t)dep * d.L + l]) continue;
+      CK(cudaStreamWaitEvent(s->stream, ev_copy(dep, l), 0));
+      a.phase = 1;
+      a.layer = l;
+      a.depth = dep;
+      uint64_t bytes = 0;
+      for (int i = 0; i < t_nu[l]; ++i)
+        if (!t_hit[l * BK + i] && t_depth[l * BK + i] == dep) bytes += d.slot_bytes;
+      int rc = prof_begin(s, s->stream, bytes, 1);
+      if (rc != REMOE_OK) return rc;
+      CK(launch_batched(s, a));
+      s->kernel_launches += 2;
+      rc = prof_end(s, s->stream);
+      if (rc != REMOE_OK) return rc;
+      CK(cudaEventRecord(ev_comp(dep, l), s->stream));
+    }
+  }
+  return REMOE_OK;
+}
+
+// #uMiss and token-level hits of layers [l0, l1) of the step whose trace is in the host block.
+void trace_totals(const remoe_stack* s, int l0, int l1, uint32_t* umiss, uint32_t* tok_hits) {
+  const int L = s->d.L, BK = s->BK;
+  const int* th = trace_tok_hits(s->host_block + 1, L, BK);
+  const int* nu = trace_n_unique(s->host_block + 1);
+  const int* hh = trace_hit(s->host_block + 1, L, BK);
+  for (int l = l0; l < l1; ++l) {
+    *tok_hits += (uint32_t)th[l];
+    for (int i = 0; i < nu[l] && i < BK; ++i) *umiss += hh[l * BK + i] ? 0u : 1u;
+  }
+}
+
 int decode_step_batched(remoe_stack* s, const float* hin, float* hout, int32_t* ids, float* gates) {
   DevStack& d = s->d;
   d.has_prev = s->steps_since_reset > 0 ? 1 : 0;
   d.policy = s->policy;
   d.beta = s->beta;
-  const int BK = s->BK;
 
   CK(launch_route(d, hin, ids, gates, s->contrib, 0, d.L, s->stream));
   s->kernel_launches += 2;
@@ -247,92 +338,71 @@ int decode_step_batched(remoe_stack* s, const float* hin, float* hout, int32_t* 
   s->steps_since_reset += 1;
   if (check_device_flag(s) != REMOE_OK) return REMOE_E_DEVICE_FLAG;
 
-  {
-    // per-step all-layer aggregates (App. E.2.6)
-    const int* th = trace_tok_hits(s->host_block + 1, d.L, s->BK);
-    const int* nu = trace_n_unique(s->host_block + 1);
-    const int* hh = trace_hit(s->host_block + 1, d.L, s->BK);
-    uint32_t um = 0, tk = 0;
-    for (int l = 0; l < d.L; ++l) {
-      tk += (uint32_t)th[l];
-      for (int i = 0; i < nu[l] && i < s->BK; ++i) um += hh[l * s->BK + i] ? 0u : 1u;
-    }
-    s->hist_umiss.push_back(um);
-    s->hist_tok_hits.push_back(tk);
-  }
+  uint32_t um = 0, tk = 0;                     // per-step all-layer aggregates (App. E.2.6)
+  trace_totals(s, 0, d.L, &um, &tk);
+  s->hist_umiss.push_back(um);
+  s->hist_tok_hits.push_back(tk);
 
-  int* tr = s->host_block + 1;
-  const int* t_nu = trace_n_unique(tr);
-  const int* t_req = trace_requests(tr, d.L, BK);
-  const int* t_hit = trace_hit(tr, d.L, BK);
-  const int* t_slot = trace_slot(tr, d.L, BK);
-  const int* t_depth = trace_depth(tr, d.L, BK);
-  int max_depth = -1;
   uint64_t resident_bytes = 0;
-  for (int l = 0; l < d.L; ++l) {
-    if (t_nu[l] < 0 || t_nu[l] > BK) return REMOE_E_DEVICE_FLAG;
-    for (int i = 0; i < t_nu[l]; ++i) {
-      const int j = l * BK + i;
-      if (t_hit[j]) { resident_bytes += d.slot_bytes; continue; }
-      if (t_req[j] < 0 || t_req[j] >= d.N || t_slot[j] < 0 || t_slot[j] >= d.C || t_depth[j] < 0)
-        return REMOE_E_DEVICE_FLAG;
-      if (t_depth[j] > max_depth) max_depth = t_depth[j];
-    }
-    resident_bytes += (uint64_t)d.S * d.shared_bytes;   // algorithmic: once, although every token tile streams it
-  }
+  rc = batched_waves(s, a, 0, d.L, &resident_bytes);
+  if (rc != REMOE_OK) return rc;
   if (s->profiling) s->ev_used[prof_slot].bytes = resident_bytes;
-
-  // events: [depth][layer] copy-done and compute-done
-  const size_t need = (size_t)2 * (max_depth + 1) * d.L;
-  while (s->ev_pool.size() < need) {
-    cudaEvent_t e;
-    CK(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
-    s->ev_pool.push_back(e);
-  }
-  auto ev_copy = [&](int dep, int l) { return s->ev_pool[((size_t)dep * d.L + l) * 2]; };
-  auto ev_comp = [&](int dep, int l) { return s->ev_pool[((size_t)dep * d.L + l) * 2 + 1]; };
-  std::vector<char> had(((size_t)max_depth + 2) * d.L, 0);
-
-  if (max_depth >= 0) CK(cudaStreamWaitEvent(s->copy_stream, s->ev_trace, 0));
-  for (int dep = 0; dep <= max_depth; ++dep) {
-    if (dep == 1) CK(cudaStreamWaitEvent(s->copy_stream, s->ev_resident, 0));   // displaced hits are done
-    for (int l = 0; l < d.L; ++l) {
-      int misses = 0;
-      for (int i = 0; i < t_nu[l]; ++i) {
-        const int j = l * BK + i;
-        if (t_hit[j] || t_depth[j] != dep) continue;
-        if (!misses && dep >= 1 && had[(size_t)(dep - 1) * d.L + l])
-          CK(cudaStreamWaitEvent(s->copy_stream, ev_comp(dep - 1, l), 0));        // displaced misses are done
-        CK(cudaMemcpyAsync(d.slots + ((size_t)l * d.C + t_slot[j]) * d.slot_bytes,
-                           s->host_ptrs[(size_t)l * d.N + t_req[j]], d.slot_bytes, cudaMemcpyHostToDevice,
-                           s->copy_stream));
-        ++misses;
-      }
-      if (!misses) continue;
-      had[(size_t)dep * d.L + l] = 1;
-      s->h2d_bytes[l] += (uint64_t)misses * d.slot_bytes;
-      CK(cudaEventRecord(ev_copy(dep, l), s->copy_stream));
-    }
-    for (int l = 0; l < d.L; ++l) {
-      if (!had[(size_t)dep * d.L + l]) continue;
-      CK(cudaStreamWaitEvent(s->stream, ev_copy(dep, l), 0));
-      a.phase = 1;
-      a.layer = l;
-      a.depth = dep;
-      uint64_t bytes = 0;
-      for (int i = 0; i < t_nu[l]; ++i)
-        if (!t_hit[l * BK + i] && t_depth[l * BK + i] == dep) bytes += d.slot_bytes;
-      rc = prof_begin(s, s->stream, bytes, 1);
-      if (rc != REMOE_OK) return rc;
-      CK(launch_batched(s, a));
-      s->kernel_launches += 2;
-      rc = prof_end(s, s->stream);
-      if (rc != REMOE_OK) return rc;
-      CK(cudaEventRecord(ev_comp(dep, l), s->stream));
-    }
-  }
-  CK(launch_combine_batched(a, hout, s->stream));
+  CK(launch_combine_batched(a, hout, 0, d.L, nullptr, s->stream));
   s->kernel_launches += 1;
+  return REMOE_OK;
+}
+
+// Chained step for B > 1: every layer has its own norm -> route -> trace -> waves -> combine round trip,
+// the B sequences moving through the layers together (they share each layer's cache).
+int decode_step_chained_batched(remoe_stack* s, const float* hin, float* hout, float* layer_inputs, int32_t* ids,
+                                float* gates) {
+  DevStack& d = s->d;
+  d.has_prev = s->steps_since_reset > 0 ? 1 : 0;
+  d.policy = s->policy;
+  d.beta = s->beta;
+  const size_t rows = (size_t)d.B * d.H;
+  CK(cudaMemcpyAsync(s->chain_in, hin, rows * sizeof(float), cudaMemcpyDeviceToDevice, s->stream));
+
+  BatchArgs a{};
+  a.d = d;
+  a.hidden_in = s->chain_x;
+  a.gates = gates;
+  a.part = s->part;
+  a.flags = s->flags;
+  a.plan = s->plan;
+  a.max_items = s->max_items;
+  a.step_id = ++s->step_serial;
+  uint32_t um = 0, tk = 0;
+  for (int l = 0; l < d.L; ++l) {
+    CK(launch_rmsnorm(s->chain_in + l * rows, s->chain_x + l * rows, d.H, d.B, s->stream));
+    CK(launch_route(d, s->chain_x, ids, gates, s->contrib, l, 1, s->stream));
+    s->kernel_launches += 3;
+    CK(cudaMemcpyAsync(s->host_block, s->dev_block, s->block_ints * sizeof(int), cudaMemcpyDeviceToHost,
+                       s->stream));
+    CK(cudaEventRecord(s->ev_trace, s->stream));
+    a.phase = 0;
+    a.layer = l;
+    a.depth = 0;
+    CK(launch_batched(s, a));
+    s->kernel_launches += 2;
+    CK(cudaEventRecord(s->ev_resident, s->stream));
+    CK(cudaEventSynchronize(s->ev_trace));
+    if (check_device_flag(s) != REMOE_OK) return REMOE_E_DEVICE_FLAG;
+    trace_totals(s, l, l + 1, &um, &tk);
+    uint64_t unused = 0;
+    int rc = batched_waves(s, a, l, l + 1, &unused);
+    if (rc != REMOE_OK) return rc;
+    CK(launch_combine_batched(a, s->chain_out, l, 1, s->chain_in, s->stream));
+    s->kernel_launches += 1;
+  }
+  s->steps += 1;
+  s->steps_since_reset += 1;
+  s->hist_umiss.push_back(um);
+  s->hist_tok_hits.push_back(tk);
+  CK(cudaMemcpyAsync(hout, s->chain_in + d.L * rows, rows * sizeof(float), cudaMemcpyDeviceToDevice, s->stream));
+  if (layer_inputs)
+    CK(cudaMemcpyAsync(layer_inputs, s->chain_in, rows * d.L * sizeof(float), cudaMemcpyDeviceToDevice,
+                       s->stream));
   return REMOE_OK;
 }
 
@@ -436,6 +506,7 @@ int remoe_stack_create(const remoe_shape* sh, int32_t cache_slots, void* cuda_st
   TRY(dev_alloc(s, &d.clock, L));
   TRY(dev_alloc(s, &d.prev_mask, L * d.B * kMaskWords));
   TRY(dev_alloc(s, &d.counters, L * kCounters));
+  TRY(dev_alloc(s, &d.load, L * d.N));
   TRY(dev_alloc(s, &d.shared_scale, L * d.B));
   TRY(dev_alloc(s, &d.last_overlap, L * d.B));
   TRY(dev_alloc(s, &d.last_mass, L * d.B));
@@ -570,15 +641,8 @@ int remoe_decode_step(remoe_stack* s, const float* hin, float* hout, int32_t* id
   if (check_device_flag(s) != REMOE_OK) return REMOE_E_DEVICE_FLAG;
 
   {
-    // per-step all-layer aggregates (App. E.2.6)
-    const int* th = trace_tok_hits(s->host_block + 1, d.L, s->BK);
-    const int* nu = trace_n_unique(s->host_block + 1);
-    const int* hh = trace_hit(s->host_block + 1, d.L, s->BK);
-    uint32_t um = 0, tk = 0;
-    for (int l = 0; l < d.L; ++l) {
-      tk += (uint32_t)th[l];
-      for (int i = 0; i < nu[l] && i < s->BK; ++i) um += hh[l * s->BK + i] ? 0u : 1u;
-    }
+    uint32_t um = 0, tk = 0;                   // per-step all-layer aggregates (App. E.2.6)
+    trace_totals(s, 0, d.L, &um, &tk);
     s->hist_umiss.push_back(um);
     s->hist_tok_hits.push_back(tk);
   }
@@ -619,7 +683,7 @@ int remoe_decode_step(remoe_stack* s, const float* hin, float* hout, int32_t* id
       rc = prof_begin(s, s->stream, (uint64_t)misses * d.slot_bytes, 1);
       if (rc != REMOE_OK) return rc;
       CK(launch_ffn_stream(a, s->grid, s->stream));
-  s->kernel_launches += 1;
+      s->kernel_launches += 1;
       rc = prof_end(s, s->stream);
       if (rc != REMOE_OK) return rc;
     }
@@ -634,7 +698,7 @@ int remoe_decode_step_chained(remoe_stack* s, const float* hin, float* hout, flo
                               float* gates) {
   if (!s || !hin || !hout || !ids || !gates) return REMOE_E_ARG;
   if (!everything_loaded(s)) return REMOE_E_NOT_LOADED;
-  if (s->d.B != 1) return REMOE_E_UNSUPPORTED;
+  if (s->d.B != 1) return decode_step_chained_batched(s, hin, hout, layer_inputs, ids, gates);
   DevStack& d = s->d;
   d.has_prev = s->steps_since_reset > 0 ? 1 : 0;
   d.policy = s->policy;
@@ -653,7 +717,7 @@ int remoe_decode_step_chained(remoe_stack* s, const float* hin, float* hout, flo
   for (int l = 0; l < d.L; ++l) {
     // The layer's input exists only once the previous layer is done, so every layer has its own
     // norm -> route -> trace -> fetch -> compute round trip.
-    CK(launch_rmsnorm(s->chain_in + (size_t)l * d.H, s->chain_x + (size_t)l * d.H, d.H, s->stream));
+    CK(launch_rmsnorm(s->chain_in + (size_t)l * d.H, s->chain_x + (size_t)l * d.H, d.H, 1, s->stream));
     CK(launch_route(d, s->chain_x, ids, gates, s->contrib, l, 1, s->stream));
     s->kernel_launches += 1;
     CK(cudaMemcpyAsync(s->host_block, s->dev_block, s->block_ints * sizeof(int), cudaMemcpyDeviceToHost, s->stream));
@@ -805,6 +869,38 @@ int remoe_reuse_mass(remoe_stack* s, int32_t layer, double* mass_sum, uint64_t* 
   }
   if (mass_sum) *mass_sum = tot;
   if (pairs) *pairs = p;
+  return REMOE_OK;
+}
+
+int remoe_expert_load(remoe_stack* s, int32_t layer, uint64_t* counts, double* entropy, double* cv,
+                      int32_t* visited) {
+  if (!s || layer < -1 || layer >= s->d.L) return REMOE_E_ARG;
+  CK(cudaStreamSynchronize(s->stream));
+  const int N = s->d.N;
+  std::vector<unsigned long long> c((size_t)s->d.L * N);
+  CK(cudaMemcpy(c.data(), s->d.load, c.size() * sizeof(unsigned long long), cudaMemcpyDeviceToHost));
+  const int l0 = layer < 0 ? 0 : layer, l1 = layer < 0 ? s->d.L : layer + 1;
+  double ent_sum = 0.0, cv_sum = 0.0;
+  long seen_sum = 0;
+  for (int l = l0; l < l1; ++l) {
+    const unsigned long long* n = c.data() + (size_t)l * N;
+    if (counts) for (int e = 0; e < N; ++e) counts[(size_t)(l - l0) * N + e] = n[e];
+    double tot = 0.0;
+    for (int e = 0; e < N; ++e) { tot += (double)n[e]; seen_sum += n[e] ? 1 : 0; }
+    if (tot <= 0.0 || N < 2) { ent_sum += 1.0; continue; }        // nothing routed yet: even by convention
+    double h = 0.0, var = 0.0;
+    const double mean = tot / N;
+    for (int e = 0; e < N; ++e) {
+      if (n[e]) { const double q = (double)n[e] / tot; h -= q * std::log(q); }
+      var += ((double)n[e] - mean) * ((double)n[e] - mean);
+    }
+    ent_sum += h / std::log((double)N);
+    cv_sum += std::sqrt(var / N) / mean;
+  }
+  const int nl = l1 - l0;
+  if (entropy) *entropy = ent_sum / nl;
+  if (cv) *cv = cv_sum / nl;
+  if (visited) *visited = (int32_t)(seen_sum / nl);
   return REMOE_OK;
 }
 

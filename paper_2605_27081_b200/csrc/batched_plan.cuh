@@ -22,7 +22,7 @@ constexpr int kPlanHeader = 8;                        // ints: n_items, n_units,
 __device__ __forceinline__ int cand_tiles(const BatchArgs& a, int l, int c) {
   const DevStack& d = a.d;
   const int BK = d.B * d.K;
-  if (a.phase != 0 && l != a.layer) return 0;
+  if (a.layer >= 0 && l != a.layer) return 0;
   if (c >= BK) return a.phase == 0 ? (d.B + a.tok_tile - 1) / a.tok_tile : 0;
   if (c >= trace_n_unique(d.trace)[l]) return 0;
   const int hit = trace_hit(d.trace, d.L, BK)[l * BK + c];

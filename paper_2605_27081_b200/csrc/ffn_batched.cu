@@ -259,9 +259,10 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_kernel(const __grid_c
   }
 }
 
-__global__ void __launch_bounds__(256) combine_batched_kernel(BatchArgs a, float* __restrict__ hidden_out) {
+__global__ void __launch_bounds__(256) combine_batched_kernel(BatchArgs a, float* __restrict__ hidden_out,
+                                                              int layer0, float* __restrict__ chain_in) {
   const DevStack& d = a.d;
-  const int lb = blockIdx.y;
+  const int lb = layer0 * d.B + blockIdx.y;
   const int c = blockIdx.x * 256 + threadIdx.x;
   if (c >= d.H) return;
   const int P = d.K + d.S;
@@ -272,6 +273,7 @@ __global__ void __launch_bounds__(256) combine_batched_kernel(BatchArgs a, float
       if (a.flags[row] == a.step_id) t += a.part[row * d.H + c];
     }
   hidden_out[(size_t)lb * d.H + c] = t;
+  if (chain_in) chain_in[((size_t)lb + d.B) * d.H + c] = chain_in[(size_t)lb * d.H + c] + t;
 }
 
 template <int H>
@@ -315,9 +317,10 @@ cudaError_t launch_ffn_batched(const BatchArgs& a, int grid, cudaStream_t st) {
   return cudaErrorInvalidValue;
 }
 
-cudaError_t launch_combine_batched(const BatchArgs& a, float* hidden_out, cudaStream_t st) {
-  dim3 grid((a.d.H + 255) / 256, a.d.L * a.d.B);
-  combine_batched_kernel<<<grid, 256, 0, st>>>(a, hidden_out);
+cudaError_t launch_combine_batched(const BatchArgs& a, float* hidden_out, int layer0, int n_layers,
+                                   float* chain_in, cudaStream_t st) {
+  dim3 grid((a.d.H + 255) / 256, n_layers * a.d.B);
+  combine_batched_kernel<<<grid, 256, 0, st>>>(a, hidden_out, layer0, chain_in);
   return cudaGetLastError();
 }
 

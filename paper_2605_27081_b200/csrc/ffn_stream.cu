@@ -298,10 +298,13 @@ __global__ void __launch_bounds__(256) combine_kernel(FfnArgs a, float* __restri
   if (chain_in) chain_in[(size_t)(l + 1) * d.H + c] = chain_in[(size_t)l * d.H + c] + t;
 }
 
-__global__ void __launch_bounds__(256) rmsnorm_kernel(const float* __restrict__ h, float* __restrict__ x, int H) {
+__global__ void __launch_bounds__(256) rmsnorm_kernel(const float* __restrict__ h_all, float* __restrict__ x_all,
+                                                      int H) {
   __shared__ float warp_ss[8];
   __shared__ float s_scale;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const float* h = h_all + (size_t)blockIdx.x * H;
+  float* x = x_all + (size_t)blockIdx.x * H;
   float ss = 0.f;
   for (int c = tid; c < H; c += 256) ss = fmaf(h[c], h[c], ss);
 #pragma unroll
@@ -375,8 +378,8 @@ cudaError_t launch_ffn_stream(const FfnArgs& a, int grid, cudaStream_t st) {
   return cudaErrorInvalidValue;
 }
 
-cudaError_t launch_rmsnorm(const float* h, float* x, int H, cudaStream_t st) {
-  rmsnorm_kernel<<<1, 256, 0, st>>>(h, x, H);
+cudaError_t launch_rmsnorm(const float* h, float* x, int H, int rows, cudaStream_t st) {
+  rmsnorm_kernel<<<rows, 256, 0, st>>>(h, x, H);
   return cudaGetLastError();
 }
 

@@ -46,6 +46,7 @@ struct DevStack {
   unsigned long long* clock;           // [L]
   unsigned* prev_mask;                 // [L][B][kMaskWords]
   unsigned long long* counters;        // [L][kCounters]
+  unsigned long long* load;            // [L][N]   selections per expert since the last reset
 
   float* shared_scale;                 // [L][B]
   int* last_overlap;                   // [L][B]   -1 when not counted
@@ -92,8 +93,8 @@ struct BatchArgs {
   DevStack d;
   const float* hidden_in;              // [L][B][H]
   const float* gates;                  // [L][B][K]
-  int phase;                           // 0: cache hits + shared experts of all layers; 1: misses
-  int layer, depth;                    // phase 1: which layer, which depth
+  int phase;                           // 0: cache hits + shared experts; 1: misses
+  int layer, depth;                    // phase 0: -1 = all layers, else only this one; phase 1: which layer, which depth
   int step_id;                         // stamps the partial rows written in this step
   float* part;                         // [L][B][K+S][kUnitsPerItem][H]
   int* flags;                          // [L][B][K+S][kUnitsPerItem]
@@ -103,7 +104,10 @@ struct BatchArgs {
 };
 bool ffn_batched_supported(const DevStack& d);
 cudaError_t launch_ffn_batched(const BatchArgs& a, int grid, cudaStream_t st);
-cudaError_t launch_combine_batched(const BatchArgs& a, float* hidden_out, cudaStream_t st);
+// Adds the stamped partial rows of layers [layer0, layer0 + n_layers) into hidden_out[L, B, H]; with
+// `chain_in` ([L + 1, B, H]) also writes chain_in[l + 1] = chain_in[l] + out[l] (residual chaining).
+cudaError_t launch_combine_batched(const BatchArgs& a, float* hidden_out, int layer0, int n_layers,
+                                   float* chain_in, cudaStream_t st);
 // tcgen05 / TMEM variant (needs I and I_shared multiples of 64); `maps` is an opaque, 64-byte aligned
 // block of ffn_batched_tc_maps_bytes() bytes filled once per stack by ffn_batched_tc_init.
 bool ffn_batched_tc_supported(const DevStack& d);
@@ -119,8 +123,9 @@ cudaError_t launch_ffn_stream(const FfnArgs& a, int grid, cudaStream_t st);
 // ([L + 1, 1, H]) also writes chain_in[l + 1] = chain_in[l] + out[l] (residual chaining).
 cudaError_t launch_combine(const FfnArgs& a, float* hidden_out, int layer0, int n_layers, float* chain_in,
                            cudaStream_t st);
-// x = h / sqrt(mean(h^2) + 1e-6) for one [H] vector (pre-norm of the chained mode), fixed summation order.
-cudaError_t launch_rmsnorm(const float* h, float* x, int H, cudaStream_t st);
+// x = h / sqrt(mean(h^2) + 1e-6) for each of `rows` [H] vectors (pre-norm of the chained mode), fixed
+// summation order.
+cudaError_t launch_rmsnorm(const float* h, float* x, int H, int rows, cudaStream_t st);
 size_t ffn_stream_smem_bytes(int H, int wbytes, int* stages_out);
 bool ffn_stream_supported(int H, int wbytes);
 

@@ -100,6 +100,7 @@ __device__ void resolve_layer(const DevStack& d, int l, const int* flat, int n_f
     int e = valid ? flat[i] : -1 - lane;
     if (valid && (e < 0 || e >= N)) { atomicCAS(d.err, kErrNone, kErrBadIndex); e = 0; }
     const bool resident = valid && sm.soe[e] >= 0;
+    if (valid) atomicAdd(d.load + (size_t)l * N + e, 1ull);     // expert load (integer: order-free)
     tok_h += __popc(__ballot_sync(kFull, resident));
     const unsigned same = __match_any_sync(kFull, e);
     const bool first_here = valid && (__ffs(same) - 1 == lane);

@@ -58,3 +58,25 @@ def test_batched_tensor_core_path(shape, c, rho):
 
 def test_batched_other_policy():
     _run(synth.Shape(2, 256, 16, 2, 64, 0, 0, 0, 0, 1, 6), 5, 0.4, steps=30, seed=4, dense_steps=0, policy=2)
+
+
+@pytest.mark.parametrize("shape,c", [
+    (synth.Shape(4, 512, 24, 3, 64, 1, 64, 0, 0, 1, 12), 8),       # tcgen05 kernel, union above capacity
+    (synth.Shape(3, 256, 16, 2, 40, 2, 24, 1, 0, 1, 5), 16),       # mma.sync kernel, sigmoid gate, all resident
+])
+def test_chained_batched_stack(shape, c):
+    """Batched sequences moving through residual-chained layers that share each layer's cache."""
+    import torch
+    from paper_2605_27081_b200.loader import LoadedWorkload
+    from parity_util import StepChecker, oracle_for
+
+    wl = LoadedWorkload(shape, c, seed=9)
+    try:
+        chk = StepChecker(wl, oracle_for(wl), torch)
+        hs = synth.HiddenStream(9, synth.Shape(**{**shape.asdict(), "n_layers": 1}), 0.7)
+        for t in range(8):
+            chk.step_chained_batched(hs.step()[0])
+        chk.check_counters()
+        assert chk.max_out_err <= 2e-2
+    finally:
+        wl.close()
