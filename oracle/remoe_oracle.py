@@ -387,7 +387,8 @@ class OracleStack:
         h = np.asarray(h)
         res = dict(
             ids=np.zeros((L, B, K), np.int64), gates=np.zeros((L, B, K), F64),
-            margin=np.zeros((L, B), F64), overlap=np.full((L, B), -1, np.int64),
+            margin=np.zeros((L, B), F64), logits=np.zeros((L, B, s.n_routed), F64),
+            overlap=np.full((L, B), -1, np.int64),
             mass=np.full((L, B), -1.0, F64),
             requests=[], hit=[], slot=[], evicted=[], tok_hits=[],
             out=None if ffn is None else np.zeros((L, B, s.hidden), F64),
@@ -404,8 +405,9 @@ class OracleStack:
             flat = []
             for b in range(B):
                 ov = None if id_override is None else id_override.get((l, b))
-                ids, g, margin, _, p = self.route(l, hl[b], ov)
+                ids, g, margin, z, p = self.route(l, hl[b], ov)
                 res["ids"][l, b], res["gates"][l, b], res["margin"][l, b] = ids, g, margin
+                res["logits"][l, b] = z
                 flat.extend(int(e) for e in ids)
                 for e in ids:
                     self.load[l][int(e)] += 1

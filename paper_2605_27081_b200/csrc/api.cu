@@ -57,7 +57,12 @@ struct remoe_stack {
   int max_items = 0;
   int step_serial = 0;                    // never reset: stamps partial rows
   cudaEvent_t ev_resident = nullptr;
-  bool use_tc = false;                     // batched experts on tcgen05 / TMEM
+  bool use_tc = false;                     // batched experts on tcgen05 / TMEM, slots in operand-tile order
+  char* stage_pool = nullptr;              // [2][C] channel-major landing area of fetched blocks (use_tc)
+  size_t stage_bytes = 0;
+  cudaEvent_t ev_stage[2] = {nullptr, nullptr};   // retile of the group that last used a half is enqueued
+  bool stage_used[2] = {false, false};
+  uint64_t stage_group = 0;                // running (depth, layer) group number: picks the half
   alignas(64) unsigned char tc_maps[1024];
   std::vector<cudaEvent_t> ev_pool;        // copy-done / compute-done events of the waves
   uint64_t steps = 0, steps_since_reset = 0;
@@ -207,8 +212,7 @@ int check_device_flag(remoe_stack* s) {
 // depth by depth, layer by layer, so the copy engine stays busy; each (depth, layer) group is
 // computed as soon as its copies have landed.
 cudaError_t launch_batched(remoe_stack* s, const BatchArgs& a) {
-  return s->use_tc ? launch_ffn_batched_tc(a, s->tc_maps, s->grid, s->stream)
-                   : launch_ffn_batched(a, s->grid, s->stream);
+  return s->use_tc ? launch_ffn_batched_tc(a, s->grid, s->stream) : launch_ffn_batched(a, s->grid, s->stream);
 }
 
 // Validates the trace of layers [l0, l1) and runs their miss waves: copies queued depth by depth, layer
@@ -248,18 +252,41 @@ int batched_waves(remoe_stack* s, BatchArgs& a, int l0, int l1, uint64_t* reside
   auto ev_comp = [&](int dep, int l) { return s->ev_pool[((size_t)dep * d.L + l) * 2 + 1]; };
   std::vector<char> had(((size_t)max_depth + 2) * d.L, 0);
 
-  if (max_depth >= 0) CK(cudaStreamWaitEvent(s->copy_stream, s->ev_trace, 0));
+  // Channel-major slots (mma.sync kernel): a copy writes the slot itself, so it waits for every reader
+  // of the slot's previous occupant.  Operand-tile-order slots (tcgen05 kernel): a copy lands in one
+  // half of the staging pool and the retile kernel, on the compute stream behind those readers, writes
+  // the slot; the copy engine then only ever waits for a staging half to be free.
+  const bool staged = s->use_tc;
+  if (max_depth >= 0 && !staged) CK(cudaStreamWaitEvent(s->copy_stream, s->ev_trace, 0));
+  std::vector<size_t> src_off;
+  std::vector<char*> dst_ptr;
   for (int dep = 0; dep <= max_depth; ++dep) {
-    if (dep == 1) CK(cudaStreamWaitEvent(s->copy_stream, s->ev_resident, 0));   // displaced hits are done
+    if (dep == 1 && !staged) CK(cudaStreamWaitEvent(s->copy_stream, s->ev_resident, 0));   // displaced hits are done
     for (int l = l0; l < l1; ++l) {
-      int misses = 0;
+      // one (depth, layer) group: its copies, then (enqueued at once, run when they have landed) its
+      // retile and compute launches.  Streams keep the order depth-major, layer-minor.
+      int misses = 0, half = 0;
+      src_off.clear();
+      dst_ptr.clear();
       for (int i = 0; i < t_nu[l]; ++i) {
         const int j = l * BK + i;
         if (t_hit[j] || t_depth[j] != dep) continue;
-        if (!misses && dep >= 1 && had[(size_t)(dep - 1) * d.L + l])
+        char* slot = d.slots + ((size_t)l * d.C + t_slot[j]) * d.slot_bytes;
+        char* land = slot;
+        if (staged) {
+          if (!misses) {
+            // the half's previous user is the group before last: its retile is already enqueued
+            half = (int)(s->stage_group++ & 1);
+            if (s->stage_used[half]) CK(cudaStreamWaitEvent(s->copy_stream, s->ev_stage[half], 0));
+          }
+          if (misses >= d.C) return REMOE_E_DEVICE_FLAG;         // more misses of one depth than slots: bad trace
+          src_off.push_back(((size_t)half * d.C + misses) * d.slot_bytes);
+          dst_ptr.push_back(slot);
+          land = s->stage_pool + src_off.back();
+        } else if (!misses && dep >= 1 && had[(size_t)(dep - 1) * d.L + l]) {
           CK(cudaStreamWaitEvent(s->copy_stream, ev_comp(dep - 1, l), 0));        // displaced misses are done
-        CK(cudaMemcpyAsync(d.slots + ((size_t)l * d.C + t_slot[j]) * d.slot_bytes,
-                           s->host_ptrs[(size_t)l * d.N + t_req[j]], d.slot_bytes, cudaMemcpyHostToDevice,
+        }
+        CK(cudaMemcpyAsync(land, s->host_ptrs[(size_t)l * d.N + t_req[j]], d.slot_bytes, cudaMemcpyHostToDevice,
                            s->copy_stream));
         ++misses;
       }
@@ -267,17 +294,18 @@ int batched_waves(remoe_stack* s, BatchArgs& a, int l0, int l1, uint64_t* reside
       had[(size_t)dep * d.L + l] = 1;
       s->h2d_bytes[l] += (uint64_t)misses * d.slot_bytes;
       CK(cudaEventRecord(ev_copy(dep, l), s->copy_stream));
-    }
-    for (int l = l0; l < l1; ++l) {
-      if (!had[(size_t)dep * d.L + l]) continue;
+
       CK(cudaStreamWaitEvent(s->stream, ev_copy(dep, l), 0));
+      if (staged) {
+        CK(launch_retile_tc(d, s->tc_maps, misses, src_off.data(), dst_ptr.data(), d.I, s->stream));
+        s->kernel_launches += (misses + 63) / 64;
+        CK(cudaEventRecord(s->ev_stage[half], s->stream));
+        s->stage_used[half] = true;
+      }
       a.phase = 1;
       a.layer = l;
       a.depth = dep;
-      uint64_t bytes = 0;
-      for (int i = 0; i < t_nu[l]; ++i)
-        if (!t_hit[l * BK + i] && t_depth[l * BK + i] == dep) bytes += d.slot_bytes;
-      int rc = prof_begin(s, s->stream, bytes, 1);
+      int rc = prof_begin(s, s->stream, (uint64_t)misses * d.slot_bytes, 1);
       if (rc != REMOE_OK) return rc;
       CK(launch_batched(s, a));
       s->kernel_launches += 2;
@@ -439,6 +467,7 @@ void remoe_stack_destroy(remoe_stack* s) {
   for (EvPair& p : s->ev_free) { cudaEventDestroy(p.a); cudaEventDestroy(p.b); }
   if (s->ev_trace) cudaEventDestroy(s->ev_trace);
   if (s->ev_resident) cudaEventDestroy(s->ev_resident);
+  for (cudaEvent_t e : s->ev_stage) if (e) cudaEventDestroy(e);
   for (cudaEvent_t e : s->ev_pool) cudaEventDestroy(e);
   for (cudaEvent_t e : s->ev_layer) cudaEventDestroy(e);
   for (void* p : s->dev_allocs) cudaFree(p);
@@ -537,7 +566,11 @@ int remoe_stack_create(const remoe_shape* sh, int32_t cache_slots, void* cuda_st
     const char* pick = std::getenv("REMOE_BATCHED_KERNEL");      // "mma" forces the mma.sync kernel
     if (ffn_batched_tc_supported(d) && ffn_batched_tc_maps_bytes() <= sizeof(s->tc_maps) &&
         !(pick && std::strcmp(pick, "mma") == 0)) {
-      if (ffn_batched_tc_init(d, s->tc_maps) != cudaSuccess) return bail(REMOE_E_CUDA);
+      s->stage_bytes = std::max((size_t)2 * d.C * d.slot_bytes, d.shared_bytes);
+      TRY(dev_alloc(s, &s->stage_pool, s->stage_bytes));
+      for (cudaEvent_t& e : s->ev_stage)
+        if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return bail(REMOE_E_CUDA);
+      if (ffn_batched_tc_init(d, s->stage_pool, s->stage_bytes, s->tc_maps) != cudaSuccess) return bail(REMOE_E_CUDA);
       s->use_tc = true;
     }
   }
@@ -577,8 +610,18 @@ int remoe_load_router(remoe_stack* s, int32_t layer, const void* w, const void* 
 
 int remoe_load_shared(remoe_stack* s, int32_t layer, int32_t idx, const void* block) {
   if (!s || !block || layer < 0 || layer >= s->d.L || idx < 0 || idx >= s->d.S) return REMOE_E_ARG;
-  CK(cudaMemcpyAsync(const_cast<char*>(s->d.shared_blocks) + ((size_t)layer * s->d.S + idx) * s->d.shared_bytes,
-                     block, s->d.shared_bytes, cudaMemcpyHostToDevice, s->stream));
+  char* dst = const_cast<char*>(s->d.shared_blocks) + ((size_t)layer * s->d.S + idx) * s->d.shared_bytes;
+  if (s->use_tc) {
+    // such a stack keeps its blocks in operand-tile order: land in the staging pool, then retile
+    CK(cudaStreamSynchronize(s->copy_stream));
+    CK(cudaStreamSynchronize(s->stream));
+    CK(cudaMemcpyAsync(s->stage_pool, block, s->d.shared_bytes, cudaMemcpyHostToDevice, s->stream));
+    const size_t off = 0;
+    CK(launch_retile_tc(s->d, s->tc_maps, 1, &off, &dst, s->d.Is, s->stream));
+    s->kernel_launches += 1;
+  } else {
+    CK(cudaMemcpyAsync(dst, block, s->d.shared_bytes, cudaMemcpyHostToDevice, s->stream));
+  }
   CK(cudaStreamSynchronize(s->stream));
   s->shared_loaded[(size_t)layer * s->d.S + idx] = 1;
   return REMOE_OK;

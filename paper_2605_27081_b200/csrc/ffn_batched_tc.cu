@@ -2,10 +2,15 @@
 //
 // Same work list as ffn_batched.cu, with a work item of (layer, expert, tile of up to 16 tokens)
 // and channel blocks of 64.  Per CTA (one per SM, 192 threads):
-//   warp 4   TMA producer: tiled tensor-map loads (cp.async.bulk.tensor, 128-byte swizzle, no
-//            multicast) of 16 KB operand tiles into a shared-memory ring:
+//   warp 4   TMA producer: one bulk copy (cp.async.bulk, no multicast) per 16 KB operand tile into a
+//            shared-memory ring.  Slots and shared blocks of such a stack are kept in OPERAND-TILE
+//            ORDER: per 64-channel group the H/64 A1 tiles, then the H/128 A2 tiles, each stored as
+//            the 128-byte-swizzled image the tensor cores read, so a tile is one contiguous 16 KB run
+//            in HBM (row pieces of 128 bytes at a 4 KB pitch cost about 5 % of the DRAM rate):
 //              A1 tile  = [64 channels x {gate, up}] x 64 columns of H   (K-major, 128 rows)
-//              A2 tile  = 64 channels x 128 columns of W_down             (MN-major, two boxes)
+//              A2 tile  = 64 channels x 128 columns of W_down             (MN-major, two halves)
+//            retile_kernel below produces that order from a freshly fetched channel-major block with
+//            tensor-map loads (cp.async.bulk.tensor, 128-byte swizzle) and bulk stores.
 //   warp 5   one elected thread issues tcgen05.mma (M = 128, N = 16, K = 16, bf16 -> fp32):
 //              D1[128 x 16]        += A1(kc) . X^T(kc)        for the H/64 column chunks
 //              D2[ht][128 x 16]    += A2(ht)^T . a            for the H/128 output tiles
@@ -101,8 +106,10 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return r;
 }
 
+// Tensor maps over the staging pool (channel-major blocks as fetched), viewed as [H, 3, channel rows]:
+// box {64, 2, 64} = gate/up rows of 64 channels x 64 columns, box {64, 1, 64} = W_down rows.
 struct TcMaps {
-  CUtensorMap slots_gu, slots_d, shared_gu, shared_d;
+  CUtensorMap stage_gu, stage_d;
 };
 
 // Walks the 64-channel groups of a CTA's unit range in order, piece by piece.
@@ -148,7 +155,7 @@ struct TcGeo {
 
 template <int H>
 __global__ void __launch_bounds__(kTcThreads, 1)
-ffn_batched_tc_kernel(const __grid_constant__ BatchArgs a, const __grid_constant__ TcMaps maps) {
+ffn_batched_tc_kernel(const __grid_constant__ BatchArgs a) {
   using G = TcGeo<H>;
   constexpr int NS = G::kStages;
   extern __shared__ unsigned char smem_raw[];
@@ -212,11 +219,8 @@ ffn_batched_tc_kernel(const __grid_constant__ BatchArgs a, const __grid_constant
       int n = 0;
       bool ok = true;
       auto emit = [&](const GroupRec& g, bool second) {
-        const CUtensorMap* map = g.p.shared ? (second ? &maps.shared_d : &maps.shared_gu)
-                                            : (second ? &maps.slots_d : &maps.slots_gu);
-        const char* pool = g.p.shared ? d.shared_blocks : d.slots;
-        // channel row of this group's first channel within the pool's tensor
-        const int row = (int)((g.p.base - pool) / ((size_t)3 * H * 2)) + g.blk * kTcBlockCh;
+        // tiles of this group in the block: A1 tiles first, then the A2 tiles
+        const char* src = g.p.base + ((size_t)g.blk * (G::kChunks + G::kTiles) + (second ? G::kChunks : 0)) * kTileBytes;
         const int tiles = second ? G::kTiles : G::kChunks;
         for (int t = 0; t < tiles && ok; ++t, ++n) {
           const int s = n % NS;
@@ -225,14 +229,8 @@ ffn_batched_tc_kernel(const __grid_constant__ BatchArgs a, const __grid_constant
             ok = false;
             break;
           }
-          unsigned char* dst = ring + (size_t)s * kTileBytes;
           mbar_expect_tx(full + s, kTileBytes);
-          if (!second) {
-            tma_load_3d(dst, map, t * 64, 0, row, full + s);
-          } else {
-            tma_load_3d(dst, map, t * 128, 2, row, full + s);
-            tma_load_3d(dst + kTileBytes / 2, map, t * 128 + 64, 2, row, full + s);
-          }
+          bulk_g2s(ring + (size_t)s * kTileBytes, src + (size_t)t * kTileBytes, kTileBytes, full + s);
         }
       };
       GroupWalk walk(a, n_items, ua, ub, j0);
@@ -449,17 +447,78 @@ ffn_batched_tc_kernel(const __grid_constant__ BatchArgs a, const __grid_constant
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
 }
 
+// ------------------------------------------------------------------------------------ retile
+// Channel-major block (as fetched from the host) -> operand-tile order.  One CTA per (64-channel
+// group, block): its 48 tiles (H = 2048) are loaded through the staging pool's tensor maps into a
+// small ring, swizzled by the TMA unit, and written out as contiguous 16 KB runs with bulk stores.
+constexpr int kRetileStages = 6;
+constexpr int kRetileJobs = 64;
+struct RetileArgs {
+  int n, inter;                     // jobs in this launch; intermediate size of the blocks
+  int src_row[kRetileJobs];         // first channel row of the block within the staging pool
+  char* dst[kRetileJobs];           // destination block (slot or shared block)
+  int* err;
+};
+__device__ __forceinline__ void bulk_s2g(void* dst, const void* src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(__cvta_generic_to_global(dst)),
+               "r"(smem_u32(src)), "r"(bytes)
+               : "memory");
+}
+
+template <int H>
+__global__ void __launch_bounds__(32) retile_kernel(const __grid_constant__ TcMaps maps,
+                                                    const __grid_constant__ RetileArgs r) {
+  using G = TcGeo<H>;
+  constexpr int NS = kRetileStages, T = G::kChunks + G::kTiles;
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* ring = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* full = reinterpret_cast<uint64_t*>(ring + (size_t)NS * kTileBytes);
+  if (threadIdx.x != 0) return;
+  for (int s = 0; s < NS; ++s) mbar_init(full + s, 1);
+  mbar_fence_init();
+  const int row = r.src_row[blockIdx.y] + (int)blockIdx.x * kTcBlockCh;
+  char* dst = r.dst[blockIdx.y] + (size_t)blockIdx.x * T * kTileBytes;
+  auto issue = [&](int t) {
+    const int s = t % NS;
+    unsigned char* st = ring + (size_t)s * kTileBytes;
+    mbar_expect_tx(full + s, kTileBytes);
+    if (t < G::kChunks) {
+      tma_load_3d(st, &maps.stage_gu, t * 64, 0, row, full + s);
+    } else {
+      const int ht = t - G::kChunks;
+      tma_load_3d(st, &maps.stage_d, ht * 128, 2, row, full + s);
+      tma_load_3d(st + kTileBytes / 2, &maps.stage_d, ht * 128 + 64, 2, row, full + s);
+    }
+  };
+  int issued = 0;
+  for (; issued < NS && issued < T; ++issued) issue(issued);
+  bool ok = true;
+  for (int t = 0; t < T; ++t) {
+    const int s = t % NS;
+    if (!mbar_wait(full + s, (t / NS) & 1)) { ok = false; break; }
+    proxy_fence();
+    bulk_s2g(dst + (size_t)t * kTileBytes, ring + (size_t)s * kTileBytes, kTileBytes);
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+    if (issued < T) {
+      asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");     // the stage has been read out
+      issue(issued++);
+    }
+  }
+  asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+  if (!ok) {
+    atomicCAS(r.err, kErrNone, kErrWaitFull);
+    // loads still in flight must land before the CTA's shared memory is given up
+    for (int t = max(0, issued - NS); t < issued; ++t)
+      if (!mbar_wait(full + (t % NS), (t / NS) & 1)) atomicCAS(r.err, kErrNone, kErrDrain);
+  }
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-// A pool of expert blocks as a 3-D bf16 tensor (H columns, 3 row kinds, channel rows of all blocks).
+// A pool of channel-major expert blocks as a 3-D bf16 tensor (H columns, 3 row kinds, channel rows).
 bool encode_pool(EncodeTiledFn encode, CUtensorMap* gu, CUtensorMap* dn, const void* base, int H, size_t rows) {
-  if (rows == 0) {
-    std::memset(gu, 0, sizeof(*gu));
-    std::memset(dn, 0, sizeof(*dn));
-    return true;
-  }
   cuuint64_t dims[3] = {(cuuint64_t)H, 3, (cuuint64_t)rows};
   cuuint64_t strides[2] = {(cuuint64_t)H * 2, (cuuint64_t)3 * H * 2};
   cuuint32_t box_gu[3] = {64, 2, 64}, box_d[3] = {64, 1, 64}, estr[3] = {1, 1, 1};
@@ -472,25 +531,39 @@ bool encode_pool(EncodeTiledFn encode, CUtensorMap* gu, CUtensorMap* dn, const v
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int H>
-cudaError_t launch_tc(const BatchArgs& a, const TcMaps& maps, int grid, cudaStream_t st) {
-  // the dynamic shared-memory limit is a per-device attribute of the kernel
-  static bool configured[64] = {};
+// the dynamic shared-memory limit is a per-device attribute of a kernel
+template <typename K>
+cudaError_t allow_smem(K kernel, size_t bytes, bool* configured) {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-  if (!configured[dev]) {
-    cudaError_t e = cudaFuncSetAttribute(ffn_batched_tc_kernel<H>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)TcGeo<H>::kSmem);
-    if (e != cudaSuccess) return e;
-    configured[dev] = true;
-  }
+  if (configured[dev]) return cudaSuccess;
+  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+  if (e == cudaSuccess) configured[dev] = true;
+  return e;
+}
+
+template <int H>
+cudaError_t launch_tc(const BatchArgs& a, int grid, cudaStream_t st) {
+  static bool configured[64] = {};
+  cudaError_t e = allow_smem(ffn_batched_tc_kernel<H>, TcGeo<H>::kSmem, configured);
+  if (e != cudaSuccess) return e;
   BatchArgs b = a;
   b.tok_tile = kTcTokTile;
   b.blk_ch = kTcBlockCh;
   plan_kernel<<<1, 1024, 0, st>>>(b);
-  cudaError_t e = cudaGetLastError();
+  e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  ffn_batched_tc_kernel<H><<<grid, kTcThreads, TcGeo<H>::kSmem, st>>>(b, maps);
+  ffn_batched_tc_kernel<H><<<grid, kTcThreads, TcGeo<H>::kSmem, st>>>(b);
+  return cudaGetLastError();
+}
+
+template <int H>
+cudaError_t launch_retile(const TcMaps& maps, const RetileArgs& r, cudaStream_t st) {
+  constexpr size_t kSmem = 1024 + (size_t)kRetileStages * kTileBytes + 64;
+  static bool configured[64] = {};
+  cudaError_t e = allow_smem(retile_kernel<H>, kSmem, configured);
+  if (e != cudaSuccess) return e;
+  retile_kernel<H><<<dim3(r.inter / kTcBlockCh, r.n), 32, kSmem, st>>>(maps, r);
   return cudaGetLastError();
 }
 
@@ -505,29 +578,54 @@ bool ffn_batched_tc_supported(const DevStack& d) {
 
 size_t ffn_batched_tc_maps_bytes() { return sizeof(TcMaps); }
 
-cudaError_t ffn_batched_tc_init(const DevStack& d, void* maps_out) {
+cudaError_t ffn_batched_tc_init(const DevStack& d, const void* stage_pool, size_t stage_bytes, void* maps_out) {
   void* fn = nullptr;
   cudaDriverEntryPointQueryResult qres;
   cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
   if (e != cudaSuccess) return e;
   if (!fn) return cudaErrorNotSupported;
   TcMaps* m = static_cast<TcMaps*>(maps_out);
-  EncodeTiledFn encode = reinterpret_cast<EncodeTiledFn>(fn);
-  if (!encode_pool(encode, &m->slots_gu, &m->slots_d, d.slots, d.H, (size_t)d.L * d.C * d.I)) return cudaErrorInvalidValue;
-  if (!encode_pool(encode, &m->shared_gu, &m->shared_d, d.shared_blocks, d.H, (size_t)d.L * d.S * d.Is))
+  const size_t rows = stage_bytes / ((size_t)3 * d.H * 2);
+  if (rows < (size_t)kTcBlockCh || rows > 0x7fffffffu) return cudaErrorInvalidValue;
+  if (!encode_pool(reinterpret_cast<EncodeTiledFn>(fn), &m->stage_gu, &m->stage_d, stage_pool, d.H, rows))
     return cudaErrorInvalidValue;
   return cudaSuccess;
 }
 
-cudaError_t launch_ffn_batched_tc(const BatchArgs& a, const void* maps, int grid, cudaStream_t st) {
-  const TcMaps& m = *static_cast<const TcMaps*>(maps);
+cudaError_t launch_ffn_batched_tc(const BatchArgs& a, int grid, cudaStream_t st) {
   switch (a.d.H) {
-    case 256: return launch_tc<256>(a, m, grid, st);
-    case 512: return launch_tc<512>(a, m, grid, st);
-    case 1024: return launch_tc<1024>(a, m, grid, st);
-    case 2048: return launch_tc<2048>(a, m, grid, st);
+    case 256: return launch_tc<256>(a, grid, st);
+    case 512: return launch_tc<512>(a, grid, st);
+    case 1024: return launch_tc<1024>(a, grid, st);
+    case 2048: return launch_tc<2048>(a, grid, st);
   }
   return cudaErrorInvalidValue;
+}
+
+cudaError_t launch_retile_tc(const DevStack& d, const void* maps, int n, const size_t* src_offsets,
+                             char* const* dst, int inter, cudaStream_t st) {
+  const TcMaps& m = *static_cast<const TcMaps*>(maps);
+  const size_t row_bytes = (size_t)3 * d.H * 2;
+  for (int i0 = 0; i0 < n; i0 += kRetileJobs) {
+    RetileArgs r{};
+    r.n = n - i0 < kRetileJobs ? n - i0 : kRetileJobs;
+    r.inter = inter;
+    r.err = d.err;
+    for (int i = 0; i < r.n; ++i) {
+      if (src_offsets[i0 + i] % row_bytes) return cudaErrorInvalidValue;
+      r.src_row[i] = (int)(src_offsets[i0 + i] / row_bytes);
+      r.dst[i] = dst[i0 + i];
+    }
+    cudaError_t e = cudaErrorInvalidValue;
+    switch (d.H) {
+      case 256: e = launch_retile<256>(m, r, st); break;
+      case 512: e = launch_retile<512>(m, r, st); break;
+      case 1024: e = launch_retile<1024>(m, r, st); break;
+      case 2048: e = launch_retile<2048>(m, r, st); break;
+    }
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
 }
 
 }  // namespace remoe

@@ -108,12 +108,18 @@ cudaError_t launch_ffn_batched(const BatchArgs& a, int grid, cudaStream_t st);
 // `chain_in` ([L + 1, B, H]) also writes chain_in[l + 1] = chain_in[l] + out[l] (residual chaining).
 cudaError_t launch_combine_batched(const BatchArgs& a, float* hidden_out, int layer0, int n_layers,
                                    float* chain_in, cudaStream_t st);
-// tcgen05 / TMEM variant (needs I and I_shared multiples of 64); `maps` is an opaque, 64-byte aligned
-// block of ffn_batched_tc_maps_bytes() bytes filled once per stack by ffn_batched_tc_init.
+// tcgen05 / TMEM variant (needs I and I_shared multiples of 64).  Its stacks keep slots and shared blocks
+// in operand-tile order: a fetched block lands channel-major in a staging pool and launch_retile_tc
+// rewrites it into its slot.  `maps` is an opaque, 64-byte aligned block of ffn_batched_tc_maps_bytes()
+// bytes describing the staging pool, filled once per stack by ffn_batched_tc_init.
 bool ffn_batched_tc_supported(const DevStack& d);
 size_t ffn_batched_tc_maps_bytes();
-cudaError_t ffn_batched_tc_init(const DevStack& d, void* maps_out);
-cudaError_t launch_ffn_batched_tc(const BatchArgs& a, const void* maps, int grid, cudaStream_t st);
+cudaError_t ffn_batched_tc_init(const DevStack& d, const void* stage_pool, size_t stage_bytes, void* maps_out);
+cudaError_t launch_ffn_batched_tc(const BatchArgs& a, int grid, cudaStream_t st);
+// Rewrites n channel-major blocks of intermediate size `inter` at byte offsets src_offsets[i] of the
+// staging pool (multiples of 3 * H * 2) into dst[i] in operand-tile order.  Host arrays.
+cudaError_t launch_retile_tc(const DevStack& d, const void* maps, int n, const size_t* src_offsets,
+                             char* const* dst, int inter, cudaStream_t st);
 
 // Routes layers [layer0, layer0 + n_layers); `hidden_in`, `ids`, `gates` are the full [L, B, .] arrays.
 cudaError_t launch_route(const DevStack& d, const float* hidden_in, int* ids, float* gates,

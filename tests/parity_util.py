@@ -7,7 +7,15 @@ import synth
 from oracle import remoe_oracle as orc
 
 TOL = {0: 1e-4, 1: 2e-2, 2: 2e-2}  # max|d| / max|ref| : float32, bf16, fp8 weights (fp32 accumulate)
-NEAR_TIE = 1e-5                   # logit margin below which selected ids may differ
+NEAR_TIE = 1e-5                   # logit gap below which the selected list may differ
+
+
+def near_tie_only(z, o_ids, ids):
+    """True if the library's list `ids` differs from the oracle's `o_ids` only by near-ties: at every
+    rank the two lists hold experts whose oracle logits are within NEAR_TIE of each other.  That covers
+    the boundary case (rank K against rank K+1) and two selected experts swapping ranks; both can only
+    happen when fp32 rounding of the logits meets a gap that small (Top-K stability, App. C)."""
+    return all(abs(float(z[int(a)]) - float(z[int(b)])) < NEAR_TIE for a, b in zip(o_ids, ids))
 
 
 def widen(shape, a, router=False):
@@ -39,9 +47,10 @@ def rel_err(got, ref):
 class StepChecker:
     """Feeds one step to both sides and compares ids, gates, cache trace and outputs.
 
-    Where the oracle's top-K margin is below NEAR_TIE and the library picked a different
-    (equally defensible) set, the difference is counted and the oracle is re-run for that
-    (layer, sequence) with the library's ids so that later cache states stay comparable.
+    Where two of the oracle's logits are closer than NEAR_TIE and the library therefore picked a
+    different (equally defensible) set, or the same set with two ranks swapped, the difference is
+    counted and the oracle is re-run for that (layer, sequence) with the library's list so that
+    later cache states stay comparable.
     """
 
     def __init__(self, wl, oracle, torch, device="cuda:0"):
@@ -80,10 +89,11 @@ class StepChecker:
         override = {}
         for l in range(self.L):
             for b in range(self.B):
-                o_ids, _, margin, _, _ = self.o.route(l, h[l, b])
+                o_ids, _, margin, z, _ = self.o.route(l, h[l, b])
                 if list(o_ids) != list(ids[l, b]):
-                    assert margin < NEAR_TIE, (
-                        f"ids differ at layer {l} seq {b} with margin {margin}: {list(o_ids)} vs {list(ids[l, b])}")
+                    assert near_tie_only(z, o_ids, ids[l, b]), (
+                        f"ids differ at layer {l} seq {b} beyond near-ties (boundary margin {margin}): "
+                        f"{[int(e) for e in o_ids]} vs {[int(e) for e in ids[l, b]]}")
                     self.near_ties += 1
                     override[(l, b)] = [int(e) for e in ids[l, b]]
         r = self.o.step(h, ffn=ffn, id_override=override or None, ffn_layers=ffn_layers)
@@ -152,7 +162,8 @@ class StepChecker:
             if not bad:
                 break
             l = bad[0]
-            assert trial["margin"][l, 0] < NEAR_TIE, f"chained ids differ at layer {l}, margin {trial['margin'][l, 0]}"
+            assert near_tie_only(trial["logits"][l, 0], trial["ids"][l, 0], ids[l, 0]), (
+                f"chained ids differ at layer {l} beyond near-ties, boundary margin {trial['margin'][l, 0]}")
             self.near_ties += 1
             override[(l, 0)] = [int(e) for e in ids[l, 0]]
         r = self.o.step(np.asarray(h0).reshape(1, H), ffn="selected", chained=True, id_override=override or None)

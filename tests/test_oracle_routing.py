@@ -111,3 +111,18 @@ def test_unique_in_order_and_overlap():
     assert orc.reuse_overlap([1, 2, 3], [3, 4, 1]) == 2
     assert orc.reuse_overlap([1, 2], [3, 4]) == 0
     assert orc.reuse_overlap([7, 8], [8, 7]) == 2
+
+
+def test_near_tie_rule_of_the_parity_harness():
+    """What the GPU parity tests accept as a near-tie: lists that differ only where two oracle logits
+    are closer than 1e-5 (boundary flip or two ranks swapped), nothing else."""
+    from parity_util import near_tie_only
+    z = np.array([3.0, 2.0, 2.0 - 4e-6, 1.0, 1.0 - 2e-6, -5.0])
+    ids, _ = orc.topk_select(z, 4)
+    assert list(ids) == [0, 1, 2, 3]
+    assert near_tie_only(z, ids, [0, 2, 1, 3])            # ranks 2 and 3 swapped across a 4e-6 gap
+    assert near_tie_only(z, ids, [0, 1, 2, 4])            # boundary: expert 4 instead of 3, 2e-6 apart
+    assert near_tie_only(z, ids, [0, 2, 1, 4])
+    assert not near_tie_only(z, ids, [1, 0, 2, 3])        # a gap of 1.0 is not a tie
+    assert not near_tie_only(z, ids, [0, 1, 2, 5])
+    assert not near_tie_only(z, ids, [0, 1, 3, 2])        # 2 and 3 are 1.0 apart
