@@ -38,6 +38,16 @@ CLOCK_QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.ac
                "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
 
+def kernel_name(shape):
+    """The expert kernel a stack of this shape runs (the library picks it the same way)."""
+    if shape.batch == 1:
+        return f"ffn_stream_kernel<{DTYPE_NAME[shape.weight_dtype]},{shape.hidden}>"
+    tc = shape.inter_routed % 64 == 0 and (shape.n_shared == 0 or shape.inter_shared % 64 == 0)
+    if tc and os.environ.get("REMOE_BATCHED_KERNEL") != "mma":
+        return f"ffn_batched_tc_kernel<{shape.hidden}>"
+    return f"ffn_batched_kernel<{shape.hidden}>"
+
+
 def measured_peaks():
     try:
         with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
@@ -387,8 +397,7 @@ def run_ours(args, rank, world, local_rank):
     roofline = {"bound": "hbm", "achieved": ach, "peak": peak_hbm, "unit": "GB/s", "frac": ach / peak_hbm,
                 "traffic": (kr_b / max(1, kr_n) * TRAFFIC_RATIO[(args.workload, shape.weight_dtype)]
                             if TRAFFIC_RATIO.get((args.workload, shape.weight_dtype)) and not args.layers else None),
-                "peak_kind": f"of {peak_kind}", "kernel": (f"ffn_stream_kernel<{DTYPE_NAME[shape.weight_dtype]},{shape.hidden}>" if shape.batch == 1
-                           else f"ffn_batched_kernel<{shape.hidden}>") + " resident phase",
+                "peak_kind": f"of {peak_kind}", "kernel": kernel_name(shape) + " resident phase",
                 "launches": kr_n, "avg_launch_ms": kr_ms / max(1, kr_n), "bytes_per_launch": kr_b / max(1, kr_n),
                 "frac_of_nominal_8TBs": ach / NOMINAL_HBM_GBS}
     miss_phase = {"launches": km_n, "avg_launch_us": km_ms * 1e3 / max(1, km_n),
