@@ -141,6 +141,7 @@ int reset_state(remoe_stack* s) {
   CK(cudaMemsetAsync(d.mass_sum, 0, L * d.B * sizeof(double), s->stream));
   CK(cudaMemsetAsync(s->dev_block, 0, s->block_ints * sizeof(int), s->stream));
   CK(cudaStreamSynchronize(s->stream));
+  std::memset(s->host_block, 0, s->block_ints * sizeof(int));
   s->steps = 0;
   s->steps_since_reset = 0;
   std::fill(s->h2d_bytes.begin(), s->h2d_bytes.end(), 0);
@@ -337,8 +338,7 @@ int decode_step_batched(remoe_stack* s, const float* hin, float* hout, int32_t* 
 
   CK(launch_route(d, hin, ids, gates, s->contrib, 0, d.L, s->stream));
   s->kernel_launches += 2;
-  CK(cudaMemcpyAsync(s->host_block, s->dev_block, s->block_ints * sizeof(int), cudaMemcpyDeviceToHost, s->stream));
-  CK(cudaEventRecord(s->ev_trace, s->stream));
+  CK(cudaEventRecord(s->ev_trace, s->stream));      // the route kernel has written the trace to the host mirror
 
   BatchArgs a{};
   a.d = d;
@@ -405,8 +405,6 @@ int decode_step_chained_batched(remoe_stack* s, const float* hin, float* hout, f
     CK(launch_rmsnorm(s->chain_in + l * rows, s->chain_x + l * rows, d.H, d.B, s->stream));
     CK(launch_route(d, s->chain_x, ids, gates, s->contrib, l, 1, s->stream));
     s->kernel_launches += 3;
-    CK(cudaMemcpyAsync(s->host_block, s->dev_block, s->block_ints * sizeof(int), cudaMemcpyDeviceToHost,
-                       s->stream));
     CK(cudaEventRecord(s->ev_trace, s->stream));
     a.phase = 0;
     a.layer = l;
@@ -486,7 +484,7 @@ int remoe_stack_create(const remoe_shape* sh, int32_t cache_slots, void* cuda_st
   const int wbytes = sh->weight_dtype == REMOE_BF16 ? 2 : (sh->weight_dtype == REMOE_FP8_E4M3 ? 1 : 4);
   const int rbytes = sh->weight_dtype == REMOE_F32 ? 4 : 2;
   const long pairs = (long)sh->n_layers * (sh->top_k + sh->n_shared);
-  if (sh->n_routed > kMaxRouted || sh->top_k > 32 || cache_slots > kMaxSlots || cache_slots > sh->n_routed ||
+  if (sh->hidden > kMaxHidden || sh->n_routed > kMaxRouted || sh->top_k > 32 || cache_slots > kMaxSlots || cache_slots > sh->n_routed ||
       (long)sh->batch * sh->top_k > kMaxRequests || !ffn_stream_supported(sh->hidden, wbytes))
     return REMOE_E_UNSUPPORTED;
   if (sh->batch == 1 && pairs > kMaxPairs) return REMOE_E_UNSUPPORTED;
@@ -546,6 +544,11 @@ int remoe_stack_create(const remoe_shape* sh, int32_t cache_slots, void* cuda_st
   std::memset(s->host_block, 0, s->block_ints * sizeof(int));
   d.err = s->dev_block;
   d.trace = s->dev_block + 1;
+  {
+    void* dp = nullptr;
+    if (cudaHostGetDevicePointer(&dp, s->host_block, 0) != cudaSuccess || !dp) return bail(REMOE_E_CUDA);
+    d.host_mirror = static_cast<int*>(dp);
+  }
   TRY(dev_alloc(s, &s->partial, (size_t)2 * L * s->grid * d.H));
   TRY(dev_alloc(s, &s->contrib, (size_t)2 * L * 2));
   TRY(dev_alloc(s, &s->chain_in, (L + 1) * d.B * d.H));
@@ -657,8 +660,7 @@ int remoe_decode_step(remoe_stack* s, const float* hin, float* hout, int32_t* id
 
   CK(launch_route(d, hin, ids, gates, s->contrib, 0, d.L, s->stream));
   s->kernel_launches += d.B > 1 ? 2 : 1;
-  CK(cudaMemcpyAsync(s->host_block, s->dev_block, s->block_ints * sizeof(int), cudaMemcpyDeviceToHost, s->stream));
-  CK(cudaEventRecord(s->ev_trace, s->stream));
+  CK(cudaEventRecord(s->ev_trace, s->stream));      // the route kernel has written the trace to the host mirror
 
   FfnArgs a{};
   a.d = d;
@@ -763,7 +765,6 @@ int remoe_decode_step_chained(remoe_stack* s, const float* hin, float* hout, flo
     CK(launch_rmsnorm(s->chain_in + (size_t)l * d.H, s->chain_x + (size_t)l * d.H, d.H, 1, s->stream));
     CK(launch_route(d, s->chain_x, ids, gates, s->contrib, l, 1, s->stream));
     s->kernel_launches += 1;
-    CK(cudaMemcpyAsync(s->host_block, s->dev_block, s->block_ints * sizeof(int), cudaMemcpyDeviceToHost, s->stream));
     CK(cudaEventRecord(s->ev_trace, s->stream));
     a.phase = 0;
     a.layer = l;

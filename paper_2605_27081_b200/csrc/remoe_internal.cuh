@@ -8,6 +8,7 @@
 
 namespace remoe {
 
+constexpr int kMaxHidden = 2048;       // H limit: a row is at most 8 x 32 16-byte pieces; h staged in shared memory
 constexpr int kMaxRouted = 256;        // N_r limit: 8 logits per lane in the top-K warp
 constexpr int kMaskWords = kMaxRouted / 32;
 constexpr int kMaxSlots = 256;         // C limit of the shared-memory directory image
@@ -59,6 +60,9 @@ struct DevStack {
   // step (0 unless the step asks for more distinct experts than there are slots).
   int* trace;
   int* err;
+  // Mirror of [err | trace] in mapped page-locked host memory: the resolve warp writes its layer's part
+  // there as well, so the host has the miss list when the route kernel ends, with no copy on the stream.
+  int* host_mirror;
   // Token groups per distinct request (batch > 1): which sequences selected it, at which rank.
   int* grp_count;                      // [L][B*K]
   int* grp_tok;                        // [L][B*K][B]

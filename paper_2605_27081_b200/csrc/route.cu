@@ -29,36 +29,49 @@ __device__ __forceinline__ float warp_max(float v) {
   return v;
 }
 
-// Dot product of one weight row (H elements, 16-byte aligned) with h, by one warp.
+// Dot product of one weight row (H <= 2048 elements, 16-byte aligned) with h (staged in shared memory),
+// by one warp.  All of a lane's 16-byte pieces of the row (at most 8) are requested before the first is
+// used, so a row costs one memory round trip instead of one per piece.
+constexpr int kRowPieces = 8;
 __device__ __forceinline__ float row_dot(const char* row, const float* __restrict__ h, int H,
                                          int wbytes, int lane) {
   float acc = 0.f;
+  const uint4* r4 = reinterpret_cast<const uint4*>(row);
+  const float4* h4 = reinterpret_cast<const float4*>(h);
+  const int n = H * wbytes / 16;                     // 16-byte pieces in the row: <= 256
+  uint4 w[kRowPieces];
+#pragma unroll
+  for (int i = 0; i < kRowPieces; ++i) {
+    const int c = lane + 32 * i;
+    w[i] = c < n ? __ldg(r4 + c) : make_uint4(0u, 0u, 0u, 0u);
+  }
   if (wbytes == 4) {
-    const float4* r4 = reinterpret_cast<const float4*>(row);
-    const float4* h4 = reinterpret_cast<const float4*>(h);
-    for (int c = lane; c < H / 4; c += 32) {
-      float4 w = __ldg(r4 + c);
-      float4 x = __ldg(h4 + c);
-      acc = fmaf(w.x, x.x, acc);
-      acc = fmaf(w.y, x.y, acc);
-      acc = fmaf(w.z, x.z, acc);
-      acc = fmaf(w.w, x.w, acc);
+#pragma unroll
+    for (int i = 0; i < kRowPieces; ++i) {
+      const int c = lane + 32 * i;
+      if (c < n) {
+        const float4 x = h4[c];
+        acc = fmaf(__uint_as_float(w[i].x), x.x, acc);
+        acc = fmaf(__uint_as_float(w[i].y), x.y, acc);
+        acc = fmaf(__uint_as_float(w[i].z), x.z, acc);
+        acc = fmaf(__uint_as_float(w[i].w), x.w, acc);
+      }
     }
   } else {
-    const uint4* r4 = reinterpret_cast<const uint4*>(row);
-    const float4* h4 = reinterpret_cast<const float4*>(h);
-    for (int c = lane; c < H / 8; c += 32) {
-      uint4 w = __ldg(r4 + c);
-      float4 x0 = __ldg(h4 + 2 * c);
-      float4 x1 = __ldg(h4 + 2 * c + 1);
-      acc = fmaf(__uint_as_float(w.x << 16), x0.x, acc);
-      acc = fmaf(__uint_as_float(w.x & 0xffff0000u), x0.y, acc);
-      acc = fmaf(__uint_as_float(w.y << 16), x0.z, acc);
-      acc = fmaf(__uint_as_float(w.y & 0xffff0000u), x0.w, acc);
-      acc = fmaf(__uint_as_float(w.z << 16), x1.x, acc);
-      acc = fmaf(__uint_as_float(w.z & 0xffff0000u), x1.y, acc);
-      acc = fmaf(__uint_as_float(w.w << 16), x1.z, acc);
-      acc = fmaf(__uint_as_float(w.w & 0xffff0000u), x1.w, acc);
+#pragma unroll
+    for (int i = 0; i < kRowPieces; ++i) {
+      const int c = lane + 32 * i;
+      if (c < n) {
+        const float4 x0 = h4[2 * c], x1 = h4[2 * c + 1];
+        acc = fmaf(__uint_as_float(w[i].x << 16), x0.x, acc);
+        acc = fmaf(__uint_as_float(w[i].x & 0xffff0000u), x0.y, acc);
+        acc = fmaf(__uint_as_float(w[i].y << 16), x0.z, acc);
+        acc = fmaf(__uint_as_float(w[i].y & 0xffff0000u), x0.w, acc);
+        acc = fmaf(__uint_as_float(w[i].z << 16), x1.x, acc);
+        acc = fmaf(__uint_as_float(w[i].z & 0xffff0000u), x1.y, acc);
+        acc = fmaf(__uint_as_float(w[i].w << 16), x1.z, acc);
+        acc = fmaf(__uint_as_float(w[i].w & 0xffff0000u), x1.w, acc);
+      }
     }
   }
   return warp_sum(acc);
@@ -233,6 +246,25 @@ __device__ void resolve_layer(const DevStack& d, int l, const int* flat, int n_f
     contrib[(d.L + l) * 2 + 0] = 1;      // no miss-phase contribution yet for this layer
     contrib[(d.L + l) * 2 + 1] = 0;
   }
+  if (d.host_mirror) {
+    // this layer's part of the trace, and the error word if set, straight to mapped host memory
+    __syncwarp();
+    int* ht = d.host_mirror + 1;
+    for (int i = lane; i < BK; i += 32) {
+      trace_requests(ht, d.L, BK)[l * BK + i] = t_req[i];
+      trace_hit(ht, d.L, BK)[l * BK + i] = t_hit[i];
+      trace_slot(ht, d.L, BK)[l * BK + i] = t_slot[i];
+      trace_evicted(ht, d.L, BK)[l * BK + i] = t_ev[i];
+      trace_depth(ht, d.L, BK)[l * BK + i] = t_depth[i];
+    }
+    if (lane == 0) {
+      trace_n_unique(ht)[l] = n_u;
+      trace_tok_hits(ht, d.L, BK)[l] = tok_h;
+      const int e = *(volatile int*)d.err;
+      if (e != kErrNone) d.host_mirror[0] = e;
+    }
+    __threadfence_system();
+  }
 }
 
 __global__ void __launch_bounds__(1024) route_kernel(DevStack d, const float* __restrict__ hidden_in,
@@ -241,13 +273,16 @@ __global__ void __launch_bounds__(1024) route_kernel(DevStack d, const float* __
   __shared__ float z[kMaxRouted];
   __shared__ int s_ids[32];
   __shared__ float s_g[32];
+  __shared__ __align__(16) float h[kMaxHidden];
   __shared__ DirSmem dir;
 
   const int lb = layer0 * d.B + blockIdx.x;
   const int l = lb / d.B;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const float* h = hidden_in + (size_t)lb * d.H;
   const size_t row_bytes = (size_t)d.H * d.rbytes;
+  for (int c = threadIdx.x; c < d.H / 4; c += blockDim.x)
+    reinterpret_cast<float4*>(h)[c] = __ldg(reinterpret_cast<const float4*>(hidden_in + (size_t)lb * d.H) + c);
+  __syncthreads();
 
   const int n_warps = blockDim.x >> 5;
   for (int e = warp; e < d.N; e += n_warps) {
