@@ -14,8 +14,9 @@
  *   - "dev" pointers are CUDA device pointers owned by the caller; "host" pointers are host
  *     memory owned by the caller.  The handle is owned by the library.
  *   - All tensors are dense, row-major, layer-major: [L, B, ...].
- *   - One stack belongs to one device (the one current at creation) and one stream.
- *     Calls on one stack must not overlap in time.
+ *   - One stack belongs to one device (the one current at creation) and one stream.  A call
+ *     may be made with any device current: the library switches to the stack's device for
+ *     the call and restores the caller's.  Calls on one stack must not overlap in time.
  *
  * Data layouts
  *   router weights   [N, H]   one row per routed expert, element type = weight_dtype

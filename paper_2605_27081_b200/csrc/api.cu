@@ -99,6 +99,28 @@ int fail_cuda(remoe_stack* s, cudaError_t e, const char* what) {
     if (e_ != cudaSuccess) return fail_cuda(s, e_, #call);          \
   } while (0)
 
+// Makes the stack's device current for the duration of a call and puts the caller's back afterwards.
+struct DeviceGuard {
+  int prev = -1;
+  bool switched = false;
+  cudaError_t err = cudaSuccess;
+  explicit DeviceGuard(int dev) {
+    err = cudaGetDevice(&prev);
+    if (err == cudaSuccess && prev != dev) {
+      err = cudaSetDevice(dev);
+      switched = err == cudaSuccess;
+    }
+  }
+  ~DeviceGuard() {
+    if (switched) cudaSetDevice(prev);
+  }
+  DeviceGuard(const DeviceGuard&) = delete;
+  DeviceGuard& operator=(const DeviceGuard&) = delete;
+};
+#define ON_STACK_DEVICE(s)                                                       \
+  DeviceGuard device_guard_((s)->device);                                        \
+  if (device_guard_.err != cudaSuccess) return fail_cuda((s), device_guard_.err, "cudaSetDevice")
+
 template <typename T>
 int dev_alloc(remoe_stack* s, T** p, size_t count) {
   void* q = nullptr;
@@ -455,7 +477,7 @@ const char* remoe_last_cuda_error(const remoe_stack* s) { return s ? s->cuda_err
 
 void remoe_stack_destroy(remoe_stack* s) {
   if (!s) return;
-  cudaSetDevice(s->device);
+  DeviceGuard guard(s->device);
   cudaStreamSynchronize(s->stream);
   if (s->copy_stream) {
     cudaStreamSynchronize(s->copy_stream);
@@ -600,6 +622,7 @@ int remoe_stack_create(const remoe_shape* sh, int32_t cache_slots, void* cuda_st
 int remoe_load_router(remoe_stack* s, int32_t layer, const void* w, const void* wsg) {
   if (!s || !w || layer < 0 || layer >= s->d.L) return REMOE_E_ARG;
   if (s->d.shared_gate && !wsg) return REMOE_E_ARG;
+  ON_STACK_DEVICE(s);
   const size_t row = (size_t)s->d.H * s->d.rbytes;
   CK(cudaMemcpyAsync(const_cast<char*>(s->d.router) + (size_t)layer * s->d.N * row, w, s->d.N * row,
                      cudaMemcpyHostToDevice, s->stream));
@@ -613,6 +636,7 @@ int remoe_load_router(remoe_stack* s, int32_t layer, const void* w, const void* 
 
 int remoe_load_shared(remoe_stack* s, int32_t layer, int32_t idx, const void* block) {
   if (!s || !block || layer < 0 || layer >= s->d.L || idx < 0 || idx >= s->d.S) return REMOE_E_ARG;
+  ON_STACK_DEVICE(s);
   char* dst = const_cast<char*>(s->d.shared_blocks) + ((size_t)layer * s->d.S + idx) * s->d.shared_bytes;
   if (s->use_tc) {
     // such a stack keeps its blocks in operand-tile order: land in the staging pool, then retile
@@ -634,6 +658,7 @@ int remoe_load_experts_host(remoe_stack* s, int32_t layer, int32_t first, int32_
                             const void* const* ptrs) {
   if (!s || !ptrs || layer < 0 || layer >= s->d.L || first < 0 || count < 0 || first + count > s->d.N)
     return REMOE_E_ARG;
+  ON_STACK_DEVICE(s);
   for (int i = 0; i < count; ++i) {
     if (!ptrs[i] || (reinterpret_cast<uintptr_t>(ptrs[i]) & 15u)) return REMOE_E_ARG;
     cudaPointerAttributes at{};
@@ -652,6 +677,7 @@ int remoe_decode_step(remoe_stack* s, const float* hin, float* hout, int32_t* id
   if (!s || !hin || !hout || !ids || !gates) return REMOE_E_ARG;
   if ((reinterpret_cast<uintptr_t>(hin) | reinterpret_cast<uintptr_t>(hout)) & 15u) return REMOE_E_ARG;
   if (!everything_loaded(s)) return REMOE_E_NOT_LOADED;
+  ON_STACK_DEVICE(s);
   if (s->d.B != 1) return decode_step_batched(s, hin, hout, ids, gates);
   DevStack& d = s->d;
   d.has_prev = s->steps_since_reset > 0 ? 1 : 0;
@@ -743,6 +769,7 @@ int remoe_decode_step_chained(remoe_stack* s, const float* hin, float* hout, flo
                               float* gates) {
   if (!s || !hin || !hout || !ids || !gates) return REMOE_E_ARG;
   if (!everything_loaded(s)) return REMOE_E_NOT_LOADED;
+  ON_STACK_DEVICE(s);
   if (s->d.B != 1) return decode_step_chained_batched(s, hin, hout, layer_inputs, ids, gates);
   DevStack& d = s->d;
   d.has_prev = s->steps_since_reset > 0 ? 1 : 0;
@@ -815,6 +842,7 @@ int remoe_decode_step_chained(remoe_stack* s, const float* hin, float* hout, flo
 
 int remoe_decode_step_host(remoe_stack* s, const float* hin, float* hout, int32_t* ids, float* gates) {
   if (!s || !hin || !hout || !ids || !gates) return REMOE_E_ARG;
+  ON_STACK_DEVICE(s);
   const size_t io = (size_t)s->d.L * s->d.B * s->d.H, kk = (size_t)s->d.L * s->BK;
   std::memcpy(s->st_in_h, hin, io * sizeof(float));
   CK(cudaMemcpyAsync(s->st_in_d, s->st_in_h, io * sizeof(float), cudaMemcpyHostToDevice, s->stream));
@@ -833,6 +861,7 @@ int remoe_decode_step_host(remoe_stack* s, const float* hin, float* hout, int32_
 int remoe_last_step_trace(remoe_stack* s, int32_t* req, int32_t* hit, int32_t* slot, int32_t* ev, int32_t* nu) {
   if (!s) return REMOE_E_ARG;
   if (s->steps == 0) return REMOE_E_ARG;
+  ON_STACK_DEVICE(s);
   CK(cudaStreamSynchronize(s->stream));
   CK(cudaMemcpy(s->host_block, s->dev_block, s->block_ints * sizeof(int), cudaMemcpyDeviceToHost));
   int* tr = s->host_block + 1;
@@ -847,6 +876,7 @@ int remoe_last_step_trace(remoe_stack* s, int32_t* req, int32_t* hit, int32_t* s
 
 int remoe_cache_stats(remoe_stack* s, int32_t layer, remoe_cache_counters* out) {
   if (!s || !out || layer < -1 || layer >= s->d.L) return REMOE_E_ARG;
+  ON_STACK_DEVICE(s);
   CK(cudaStreamSynchronize(s->stream));
   std::vector<unsigned long long> c((size_t)s->d.L * kCounters);
   CK(cudaMemcpy(c.data(), s->d.counters, c.size() * sizeof(unsigned long long), cudaMemcpyDeviceToHost));
@@ -865,6 +895,7 @@ int remoe_cache_stats(remoe_stack* s, int32_t layer, remoe_cache_counters* out) 
 
 int remoe_reuse_stats(remoe_stack* s, int32_t layer, uint64_t* overlap_sum, uint64_t* pairs, float* last_ir) {
   if (!s || layer < -1 || layer >= s->d.L) return REMOE_E_ARG;
+  ON_STACK_DEVICE(s);
   CK(cudaStreamSynchronize(s->stream));
   std::vector<unsigned long long> c((size_t)s->d.L * kCounters);
   CK(cudaMemcpy(c.data(), s->d.counters, c.size() * sizeof(unsigned long long), cudaMemcpyDeviceToHost));
@@ -892,6 +923,7 @@ int remoe_reuse_stats(remoe_stack* s, int32_t layer, uint64_t* overlap_sum, uint
 
 int remoe_reuse_mass(remoe_stack* s, int32_t layer, double* mass_sum, uint64_t* pairs, float* last_mass) {
   if (!s || layer < -1 || layer >= s->d.L) return REMOE_E_ARG;
+  ON_STACK_DEVICE(s);
   CK(cudaStreamSynchronize(s->stream));
   const size_t n = (size_t)s->d.L * s->d.B;
   std::vector<double> ms(n);
@@ -919,6 +951,7 @@ int remoe_reuse_mass(remoe_stack* s, int32_t layer, double* mass_sum, uint64_t* 
 int remoe_expert_load(remoe_stack* s, int32_t layer, uint64_t* counts, double* entropy, double* cv,
                       int32_t* visited) {
   if (!s || layer < -1 || layer >= s->d.L) return REMOE_E_ARG;
+  ON_STACK_DEVICE(s);
   CK(cudaStreamSynchronize(s->stream));
   const int N = s->d.N;
   std::vector<unsigned long long> c((size_t)s->d.L * N);
@@ -984,6 +1017,7 @@ int remoe_tpot_proxy(const uint32_t* umiss, int32_t n, uint64_t expert_bytes, do
 
 int remoe_cache_reset(remoe_stack* s) {
   if (!s) return REMOE_E_ARG;
+  ON_STACK_DEVICE(s);
   CK(cudaStreamSynchronize(s->stream));
   CK(cudaStreamSynchronize(s->copy_stream));
   return reset_state(s);
@@ -1003,6 +1037,7 @@ int remoe_set_reroute_beta(remoe_stack* s, float beta) {
 
 int remoe_set_profiling(remoe_stack* s, int32_t on) {
   if (!s) return REMOE_E_ARG;
+  ON_STACK_DEVICE(s);
   int rc = prof_collect(s);
   if (rc != REMOE_OK) return rc;
   s->profiling = on != 0;
@@ -1016,6 +1051,7 @@ int remoe_set_profiling(remoe_stack* s, int32_t on) {
 
 int remoe_kernel_time(remoe_stack* s, int32_t phase, double* ms_sum, uint64_t* launches, uint64_t* bytes) {
   if (!s || phase < 0 || phase > 1) return REMOE_E_ARG;
+  ON_STACK_DEVICE(s);
   int rc = prof_collect(s);
   if (rc != REMOE_OK) return rc;
   if (ms_sum) *ms_sum = s->prof_ms[phase];
