@@ -128,6 +128,26 @@ int remoe_decode_step(remoe_stack*, const float* hidden_in_dev, float* hidden_ou
                       int32_t* selected_ids_dev, float* gate_weights_dev);
 
 /*
+ * n_steps consecutive decode steps of a batch-1 stack whose inputs are all known up front (replaying a
+ * recorded trace of hidden states, teacher-forced evaluation as in Sec. 5.2, benchmarking):
+ *   hidden_in [n_steps, L, 1, H], hidden_out [n_steps, L, 1, H], selected_ids / gate_weights
+ *   [n_steps, L, 1, K], device pointers; step t reads and writes slice t.
+ * Results, cache behaviour, counters and statistics are exactly those of n_steps calls of
+ * remoe_decode_step, bit for bit.  The difference is scheduling: a step's routing needs nothing from the
+ * previous step's fetches or expert compute (each layer reads its own input stream), so step t+1 is routed
+ * on an internal stream while step t is still fetching, and its miss list reaches the host before the copy
+ * engine runs out of work.  The host link, which bounds the step at realistic cache sizes, then stays
+ * busy across step boundaries (a single call per step leaves it idle for the time of the last expert
+ * launch, the combine, the next routing and the host hand-off: about 1 % of a step at config-2 sizes).
+ * Inputs must be complete when the stack's stream reaches the call; outputs are complete when that
+ * stream has drained.  The host blocks until the last step's miss list is known.  The first call
+ * allocates a second set of small per-step buffers.  Errors: ARG, NOT_LOADED, UNSUPPORTED (batch > 1),
+ * NOMEM, CUDA, DEVICE_FLAG.
+ */
+int remoe_decode_steps(remoe_stack*, int32_t n_steps, const float* hidden_in_dev, float* hidden_out_dev,
+                       int32_t* selected_ids_dev, float* gate_weights_dev);
+
+/*
  * Chained variant of the step: the layers feed each other through a pre-norm residual connection as
  * in a decoder stack, x_l = h_l / sqrt(mean(h_l^2) + 1e-6), h_{l+1} = h_l + MoE_l(x_l), instead of
  * each reading its own stream (the paper treats layers independently, App. A.5; chaining is how they

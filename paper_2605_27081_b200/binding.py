@@ -26,7 +26,7 @@ EXPORTS = [
     "remoe_reuse_stats", "remoe_cache_reset", "remoe_set_policy", "remoe_set_reroute_beta",
     "remoe_set_profiling", "remoe_kernel_time", "remoe_launch_count", "remoe_last_cuda_error", "remoe_stack_destroy",
     "remoe_strerror", "remoe_expert_ffn_static", "remoe_reuse_mass", "remoe_step_history", "remoe_tpot_proxy", "remoe_decode_step_chained",
-    "remoe_expert_load",
+    "remoe_expert_load", "remoe_decode_steps",
 ]
 
 
@@ -67,6 +67,7 @@ def lib():
         L.remoe_decode_step.argtypes = [vp, f32p, f32p, i32p, f32p]
         L.remoe_decode_step_host.argtypes = [vp, f32p, f32p, i32p, f32p]
         L.remoe_decode_step_chained.argtypes = [vp, f32p, f32p, f32p, i32p, f32p]
+        L.remoe_decode_steps.argtypes = [vp, i32, f32p, f32p, i32p, f32p]
         L.remoe_last_step_trace.argtypes = [vp, i32p, i32p, i32p, i32p, i32p]
         L.remoe_cache_stats.argtypes = [vp, i32, C.POINTER(remoe_cache_counters)]
         L.remoe_reuse_stats.argtypes = [vp, i32, C.POINTER(C.c_uint64), C.POINTER(C.c_uint64), vp]
@@ -144,6 +145,11 @@ def remoe_load_experts_host(h, layer, first_expert, pinned_ptrs):
 
 def remoe_decode_step(h, hidden_in, hidden_out, selected_ids, gate_weights):
     return lib().remoe_decode_step(h, _ptr(hidden_in), _ptr(hidden_out), _ptr(selected_ids), _ptr(gate_weights))
+
+
+def remoe_decode_steps(h, n_steps, hidden_in, hidden_out, selected_ids, gate_weights):
+    return lib().remoe_decode_steps(h, int(n_steps), _ptr(hidden_in), _ptr(hidden_out), _ptr(selected_ids),
+                                    _ptr(gate_weights))
 
 
 def remoe_decode_step_chained(h, hidden_in, hidden_out, layer_inputs, selected_ids, gate_weights):
@@ -278,6 +284,10 @@ class Stack:
 
     def decode_step(self, hidden_in, hidden_out, selected_ids, gate_weights):
         self._ck(remoe_decode_step(self.h, hidden_in, hidden_out, selected_ids, gate_weights), "remoe_decode_step")
+
+    def decode_steps(self, n_steps, hidden_in, hidden_out, selected_ids, gate_weights):
+        self._ck(remoe_decode_steps(self.h, n_steps, hidden_in, hidden_out, selected_ids, gate_weights),
+                 "remoe_decode_steps")
 
     def decode_step_chained(self, hidden_in, hidden_out, layer_inputs, selected_ids, gate_weights):
         self._ck(remoe_decode_step_chained(self.h, hidden_in, hidden_out, layer_inputs, selected_ids, gate_weights),

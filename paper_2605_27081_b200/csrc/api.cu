@@ -50,6 +50,17 @@ struct remoe_stack {
   float* chain_out = nullptr;              // [L][H] per-layer MoE outputs of the chained mode
   cudaEvent_t ev_trace = nullptr;
   std::vector<cudaEvent_t> ev_layer;
+  // second set of per-step buffers and the streams/events of the multi-step entry point, which routes
+  // step t+1 while step t is still fetching and computing (created on first use)
+  bool pipe_ready = false;
+  cudaStream_t route_stream = nullptr;
+  int* dev_block2 = nullptr;
+  int* host_block2 = nullptr;
+  int* contrib2 = nullptr;
+  float* shared_scale2 = nullptr;
+  cudaEvent_t ev_entry = nullptr, ev_route2[2] = {nullptr, nullptr}, ev_free2[2] = {nullptr, nullptr},
+              ev_res2[2] = {nullptr, nullptr};
+  std::vector<cudaEvent_t> ev_copy2, ev_miss2;     // [2][L]
   // batched path (B > 1)
   float* part = nullptr;
   int* flags = nullptr;
@@ -164,6 +175,7 @@ int reset_state(remoe_stack* s) {
   CK(cudaMemsetAsync(s->dev_block, 0, s->block_ints * sizeof(int), s->stream));
   CK(cudaStreamSynchronize(s->stream));
   std::memset(s->host_block, 0, s->block_ints * sizeof(int));
+  if (s->host_block2) std::memset(s->host_block2, 0, s->block_ints * sizeof(int));
   s->steps = 0;
   s->steps_since_reset = 0;
   std::fill(s->h2d_bytes.begin(), s->h2d_bytes.end(), 0);
@@ -216,13 +228,14 @@ int prof_collect(remoe_stack* s) {
   return REMOE_OK;
 }
 
-int check_device_flag(remoe_stack* s) {
-  if (s->host_block[0] == kErrNone) return REMOE_OK;
+int check_device_flag(remoe_stack* s, const int* block = nullptr) {
+  if (!block) block = s->host_block;
+  if (block[0] == kErrNone) return REMOE_OK;
   static const char* names[] = {"none", "a consumer's bounded wait for a weight row ran out",
                                 "the producer's bounded wait for a free stage ran out",
                                 "an expert id or slot index was out of range",
                                 "copies were still in flight when a kernel bailed out"};
-  const int c = s->host_block[0];
+  const int c = block[0];
   s->cuda_err = std::string("device flag ") + std::to_string(c) + ": " + (c >= 1 && c <= 4 ? names[c] : "unknown");
   return REMOE_E_DEVICE_FLAG;
 }
@@ -488,6 +501,18 @@ void remoe_stack_destroy(remoe_stack* s) {
   if (s->ev_trace) cudaEventDestroy(s->ev_trace);
   if (s->ev_resident) cudaEventDestroy(s->ev_resident);
   for (cudaEvent_t e : s->ev_stage) if (e) cudaEventDestroy(e);
+  if (s->route_stream) {
+    cudaStreamSynchronize(s->route_stream);
+    cudaStreamDestroy(s->route_stream);
+  }
+  if (s->ev_entry) cudaEventDestroy(s->ev_entry);
+  for (int p = 0; p < 2; ++p) {
+    if (s->ev_route2[p]) cudaEventDestroy(s->ev_route2[p]);
+    if (s->ev_free2[p]) cudaEventDestroy(s->ev_free2[p]);
+    if (s->ev_res2[p]) cudaEventDestroy(s->ev_res2[p]);
+  }
+  for (cudaEvent_t e : s->ev_copy2) cudaEventDestroy(e);
+  for (cudaEvent_t e : s->ev_miss2) cudaEventDestroy(e);
   for (cudaEvent_t e : s->ev_pool) cudaEventDestroy(e);
   for (cudaEvent_t e : s->ev_layer) cudaEventDestroy(e);
   for (void* p : s->dev_allocs) cudaFree(p);
@@ -762,6 +787,177 @@ int remoe_decode_step(remoe_stack* s, const float* hin, float* hout, int32_t* id
   if (s->profiling) s->ev_used[prof_slot].bytes = resident_bytes;
   CK(launch_combine(a, hout, 0, d.L, nullptr, s->stream));
   s->kernel_launches += 1;
+  return REMOE_OK;
+}
+
+// Second buffer set, route stream and events of remoe_decode_steps.
+static int pipe_setup(remoe_stack* s) {
+  if (s->pipe_ready) return REMOE_OK;
+  const DevStack& d = s->d;
+  int rc;
+  if ((rc = dev_alloc(s, &s->dev_block2, s->block_ints)) != REMOE_OK) return rc;
+  if ((rc = host_alloc(s, &s->host_block2, s->block_ints)) != REMOE_OK) return rc;
+  if ((rc = dev_alloc(s, &s->contrib2, (size_t)2 * d.L * 2)) != REMOE_OK) return rc;
+  if ((rc = dev_alloc(s, &s->shared_scale2, (size_t)d.L * d.B)) != REMOE_OK) return rc;
+  std::memset(s->host_block2, 0, s->block_ints * sizeof(int));
+  CK(cudaMemset(s->dev_block2, 0, s->block_ints * sizeof(int)));
+  if (!s->route_stream) CK(cudaStreamCreateWithFlags(&s->route_stream, cudaStreamNonBlocking));
+  auto make = [&](cudaEvent_t* e) { return *e ? cudaSuccess : cudaEventCreateWithFlags(e, cudaEventDisableTiming); };
+  CK(make(&s->ev_entry));
+  for (int p = 0; p < 2; ++p) {
+    CK(make(&s->ev_route2[p]));
+    CK(make(&s->ev_free2[p]));
+    CK(make(&s->ev_res2[p]));
+  }
+  s->ev_copy2.resize((size_t)2 * d.L, nullptr);
+  s->ev_miss2.resize((size_t)2 * d.L, nullptr);
+  for (auto& e : s->ev_copy2) CK(make(&e));
+  for (auto& e : s->ev_miss2) CK(make(&e));
+  s->pipe_ready = true;
+  return REMOE_OK;
+}
+
+int remoe_decode_steps(remoe_stack* s, int32_t n_steps, const float* hin, float* hout, int32_t* ids, float* gates) {
+  if (!s || !hin || !hout || !ids || !gates || n_steps < 0) return REMOE_E_ARG;
+  if ((reinterpret_cast<uintptr_t>(hin) | reinterpret_cast<uintptr_t>(hout)) & 15u) return REMOE_E_ARG;
+  if (!everything_loaded(s)) return REMOE_E_NOT_LOADED;
+  if (s->d.B != 1) return REMOE_E_UNSUPPORTED;
+  if (n_steps == 0) return REMOE_OK;
+  ON_STACK_DEVICE(s);
+  int rc = pipe_setup(s);
+  if (rc != REMOE_OK) return rc;
+  DevStack base = s->d;
+  base.policy = s->policy;
+  base.beta = s->beta;
+  const int L = base.L, K = base.K;
+  const size_t io = (size_t)L * base.H, kk = (size_t)L * K;
+
+  // Step t uses buffer set t & 1 (device trace + host mirror, contributor table, shared scales).  Its
+  // route kernel runs on the route stream as soon as the set is free (combine of step t-2) -- while
+  // step t-1 is still fetching and computing -- so the host has the next miss list before the copy
+  // engine runs dry.  A copy of step t into layer l waits for the kernels of step t-1 that read layer
+  // l's slots: its resident-phase launch and, if it had misses there, that miss-phase launch.
+  int* dev_blk[2] = {s->dev_block, s->dev_block2};
+  int* host_blk[2] = {s->host_block, s->host_block2};
+  int* contrib[2] = {s->contrib, s->contrib2};
+  float* scale[2] = {s->d.shared_scale, s->shared_scale2};
+  std::vector<char> missed[2] = {std::vector<char>(L, 0), std::vector<char>(L, 0)};
+
+  CK(cudaEventRecord(s->ev_entry, s->stream));          // everything before the call, the inputs included
+  CK(cudaStreamWaitEvent(s->route_stream, s->ev_entry, 0));
+  CK(cudaStreamWaitEvent(s->copy_stream, s->ev_entry, 0));
+
+  auto route = [&](int t) -> int {
+    const int p = t & 1;
+    DevStack d = base;
+    d.has_prev = (s->steps_since_reset + (uint64_t)t) > 0 ? 1 : 0;
+    d.trace = dev_blk[p] + 1;
+    d.host_mirror = host_blk[p];
+    d.shared_scale = scale[p];
+    if (t >= 2) CK(cudaStreamWaitEvent(s->route_stream, s->ev_free2[p], 0));
+    CK(launch_route(d, hin + (size_t)t * io, ids + (size_t)t * kk, gates + (size_t)t * kk, contrib[p], 0, L,
+                    s->route_stream));
+    s->kernel_launches += 1;
+    CK(cudaEventRecord(s->ev_route2[p], s->route_stream));
+    return REMOE_OK;
+  };
+
+  if ((rc = route(0)) != REMOE_OK) return rc;
+  for (int t = 0; t < n_steps; ++t) {
+    const int p = t & 1, q = p ^ 1;
+    DevStack d = base;
+    d.trace = dev_blk[p] + 1;
+    d.host_mirror = host_blk[p];
+    d.shared_scale = scale[p];
+    FfnArgs a{};
+    a.d = d;
+    a.hidden_in = hin + (size_t)t * io;
+    a.gates = gates + (size_t)t * kk;
+    a.partial = s->partial;
+    a.contrib = contrib[p];
+    a.grid_cap = s->grid;
+    a.phase = 0;
+    a.layer = -1;
+    CK(cudaStreamWaitEvent(s->stream, s->ev_route2[p], 0));
+    rc = prof_begin(s, s->stream, 0, 0);
+    if (rc != REMOE_OK) return rc;
+    CK(launch_ffn_stream(a, s->grid, s->stream));
+    s->kernel_launches += 1;
+    rc = prof_end(s, s->stream);
+    if (rc != REMOE_OK) return rc;
+    const size_t prof_slot = s->profiling ? s->ev_used.size() - 1 : 0;
+    CK(cudaEventRecord(s->ev_res2[p], s->stream));
+
+    CK(cudaEventSynchronize(s->ev_route2[p]));
+    s->steps += 1;
+    if (check_device_flag(s, host_blk[p]) != REMOE_OK) {
+      s->steps_since_reset += (uint64_t)t + 1;
+      return REMOE_E_DEVICE_FLAG;
+    }
+    // the next step's routing needs nothing from this step's fetches or compute
+    if (t + 1 < n_steps && (rc = route(t + 1)) != REMOE_OK) return rc;
+
+    int* tr = host_blk[p] + 1;
+    const int* t_req = trace_requests(tr, L, K);
+    const int* t_hit = trace_hit(tr, L, K);
+    const int* t_slot = trace_slot(tr, L, K);
+    const int* t_th = trace_tok_hits(tr, L, K);
+    uint32_t um = 0, tk = 0;
+    uint64_t resident_bytes = 0;
+    for (int l = 0; l < L; ++l) {
+      int misses = 0;
+      tk += (uint32_t)t_th[l];
+      for (int k = 0; k < K; ++k) {
+        const int i = l * K + k;
+        if (t_hit[i]) { resident_bytes += d.slot_bytes; continue; }
+        const int e = t_req[i], slot = t_slot[i];
+        if (e < 0 || e >= d.N || slot < 0 || slot >= d.C) {
+          s->cuda_err = "trace holds an expert id or slot out of range (layer " + std::to_string(l) + ")";
+          s->steps_since_reset += (uint64_t)t + 1;
+          return REMOE_E_DEVICE_FLAG;
+        }
+        if (!misses && t > 0) {
+          CK(cudaStreamWaitEvent(s->copy_stream, s->ev_res2[q], 0));
+          if (missed[q][l]) CK(cudaStreamWaitEvent(s->copy_stream, s->ev_miss2[(size_t)q * L + l], 0));
+        }
+        CK(cudaMemcpyAsync(d.slots + ((size_t)l * d.C + slot) * d.slot_bytes, s->host_ptrs[(size_t)l * d.N + e],
+                           d.slot_bytes, cudaMemcpyHostToDevice, s->copy_stream));
+        ++misses;
+      }
+      resident_bytes += (uint64_t)d.S * d.shared_bytes;
+      missed[p][l] = misses ? 1 : 0;
+      um += (uint32_t)misses;
+      if (!misses) continue;
+      s->h2d_bytes[l] += (uint64_t)misses * d.slot_bytes;
+      CK(cudaEventRecord(s->ev_copy2[(size_t)p * L + l], s->copy_stream));
+      CK(cudaStreamWaitEvent(s->stream, s->ev_copy2[(size_t)p * L + l], 0));
+      a.phase = 1;
+      a.layer = l;
+      rc = prof_begin(s, s->stream, (uint64_t)misses * d.slot_bytes, 1);
+      if (rc != REMOE_OK) return rc;
+      CK(launch_ffn_stream(a, s->grid, s->stream));
+      s->kernel_launches += 1;
+      rc = prof_end(s, s->stream);
+      if (rc != REMOE_OK) return rc;
+      CK(cudaEventRecord(s->ev_miss2[(size_t)p * L + l], s->stream));
+    }
+    if (s->profiling) s->ev_used[prof_slot].bytes = resident_bytes;
+    s->hist_umiss.push_back(um);
+    s->hist_tok_hits.push_back(tk);
+    CK(launch_combine(a, hout + (size_t)t * io, 0, L, nullptr, s->stream));
+    s->kernel_launches += 1;
+    CK(cudaEventRecord(s->ev_free2[p], s->stream));
+  }
+  s->steps_since_reset += (uint64_t)n_steps;
+  // Later calls use buffer set 0 and the stack's stream: leave the copy stream behind this call's last
+  // readers, and the device trace of the last step where remoe_last_step_trace looks for it.
+  CK(cudaStreamWaitEvent(s->copy_stream, s->ev_free2[(n_steps - 1) & 1], 0));
+  if ((n_steps - 1) & 1) {
+    CK(cudaMemcpyAsync(s->dev_block + 1, s->dev_block2 + 1, (s->block_ints - 1) * sizeof(int),
+                       cudaMemcpyDeviceToDevice, s->stream));
+    CK(cudaMemcpyAsync(s->d.shared_scale, s->shared_scale2, (size_t)L * base.B * sizeof(float),
+                       cudaMemcpyDeviceToDevice, s->stream));
+  }
   return REMOE_OK;
 }
 

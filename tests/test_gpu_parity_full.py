@@ -56,6 +56,37 @@ def test_dsv2lite_full_store_all_rhos():
     assert res[0.9][2] > res[0.5][2] > res[0.0][2]          # more temporal correlation, more hits
 
 
+def test_dsv2lite_multi_step_call_full_shape():
+    """The multi-step entry point at the benchmark's shape: bit-identical to single steps."""
+    import torch
+    from paper_2605_27081_b200.loader import LoadedWorkload
+
+    cfg = synth.config("dsv2lite")
+    shape = cfg["shape"]
+    stream = torch.cuda.Stream()
+    wl = LoadedWorkload(shape, cfg["cache_slots"], cfg["seed"], stream=stream.cuda_stream, distinct_experts=24)
+    other = wl.new_stack(cfg["cache_slots"], stream.cuda_stream)
+    try:
+        n = 40
+        L, H, K = shape.n_layers, shape.hidden, shape.top_k
+        hid = torch.from_numpy(synth.HiddenStream(cfg["seed"], shape, 0.5).take(n)).to("cuda")
+        out1 = torch.empty((n, L, 1, H), device="cuda")
+        ids1 = torch.empty((n, L, 1, K), dtype=torch.int32, device="cuda")
+        g1 = torch.empty((n, L, 1, K), device="cuda")
+        out2, ids2, g2 = torch.empty_like(out1), torch.empty_like(ids1), torch.empty_like(g1)
+        with torch.cuda.stream(stream):
+            for t in range(n):
+                wl.stack.decode_step(hid[t], out1[t], ids1[t], g1[t])
+            other.decode_steps(n, hid, out2, ids2, g2)
+        torch.cuda.synchronize()
+        assert torch.equal(ids1, ids2) and torch.equal(g1, g2) and torch.equal(out1, out2)
+        assert wl.stack.cache_stats() == other.cache_stats()
+        assert wl.stack.cache_stats()["uniq_misses"] > 30 * n
+    finally:
+        other.close()
+        wl.close()
+
+
 def test_qwen15moe_full_shape():
     res = _full("qwen15moe", 0.8, 512, distinct=16)
     print("qwen15moe:", res)

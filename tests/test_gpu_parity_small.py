@@ -216,3 +216,51 @@ def test_policy_switch_and_second_stack_share_a_store():
     finally:
         wl2.stack.close()
         wl.close()
+
+
+@pytest.mark.parametrize("shape,c,rho,n", [
+    (synth.Shape(6, 512, 24, 3, 64, 1, 32, 1, 0, 1, 1), 6, 0.6, 23),       # odd number of steps, sigmoid gate
+    (synth.Shape(3, 1024, 40, 4, 200, 2, 100, 0, 1, 1, 1), 9, 0.3, 16),    # many misses per step, renormalised
+    (synth.Shape(2, 256, 16, 2, 32, 0, 0, 0, 0, 0, 1), 2, 0.0, 9),         # float32, C = K: every slot turns over
+])
+def test_multi_step_call_equals_single_steps(shape, c, rho, n):
+    """remoe_decode_steps routes step t+1 while step t is still fetching; everything it returns must be
+    bit-identical to n calls of remoe_decode_step (itself checked against the oracle above), including
+    when single and multi-step calls are mixed on one stack."""
+    import torch
+    from paper_2605_27081_b200.loader import LoadedWorkload
+
+    wl = LoadedWorkload(shape, c, seed=11)
+    other = wl.new_stack(c)
+    try:
+        L, H, K = shape.n_layers, shape.hidden, shape.top_k
+        hid = torch.from_numpy(synth.HiddenStream(11, shape, rho).take(n + 4)).to("cuda")
+        out1 = torch.empty((n + 4, L, 1, H), device="cuda")
+        ids1 = torch.empty((n + 4, L, 1, K), dtype=torch.int32, device="cuda")
+        g1 = torch.empty((n + 4, L, 1, K), device="cuda")
+        out2, ids2, g2 = torch.empty_like(out1), torch.empty_like(ids1), torch.empty_like(g1)
+        for t in range(n + 4):
+            wl.stack.decode_step(hid[t], out1[t], ids1[t], g1[t])
+        # 2 single steps, n in one call, 1 single step, 1 in a call of its own
+        for t in range(2):
+            other.decode_step(hid[t], out2[t], ids2[t], g2[t])
+        other.decode_steps(n, hid[2:], out2[2:], ids2[2:], g2[2:])
+        other.decode_step(hid[n + 2], out2[n + 2], ids2[n + 2], g2[n + 2])
+        other.decode_steps(1, hid[n + 3:], out2[n + 3:], ids2[n + 3:], g2[n + 3:])
+        torch.cuda.synchronize()
+        assert torch.equal(ids1, ids2) and torch.equal(g1, g2)
+        assert torch.equal(out1, out2)
+        a, b = wl.stack.cache_stats(), other.cache_stats()
+        assert a == b and a["uniq_misses"] > 0
+        assert wl.stack.reuse_stats() == other.reuse_stats()
+        ta, tb = wl.stack.last_step_trace(), other.last_step_trace()
+        for k in ta:
+            assert np.array_equal(ta[k], tb[k]), k
+        ua, ha = wl.stack.step_history()
+        ub, hb = other.step_history()
+        assert list(ua) == list(ub) and list(ha) == list(hb)
+        ca, cb = wl.stack.expert_load()[0], other.expert_load()[0]
+        assert np.array_equal(ca, cb)
+    finally:
+        other.close()
+        wl.close()
