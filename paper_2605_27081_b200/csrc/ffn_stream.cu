@@ -9,7 +9,7 @@
 // linear stream of triples with no intermediate vector in memory and no dependency between
 // CTAs.  The kernel therefore treats every active (layer, expert) of the launch as one long
 // row list, cuts it into equal contiguous ranges, one per CTA, and in each CTA
-//   - a producer thread moves triples HBM -> shared memory with bulk async copies (TMA,
+//   - four lanes of a producer warp move triples HBM -> shared memory with bulk async copies (TMA,
 //     non-tensor form) into a ring of stages guarded by full/empty mbarriers;
 //   - eight consumer warps take triples round-robin; a warp owns a whole triple: two dot
 //     products by 128-bit shared loads and shuffle reduction, SiLU, then an AXPY into its
@@ -29,6 +29,7 @@ namespace {
 constexpr int kConsumerWarps = 8;
 constexpr int kThreads = (kConsumerWarps + 1) * 32;
 constexpr int kMaxStages = 16;                 // multiple of kConsumerWarps
+constexpr int kProducerLanes = 4;              // divides kConsumerWarps, hence every ring depth
 using namespace ring;
 
 // Shared-memory carve-up (dynamic): barriers | row prefix table | reduce buffer | stage ring.
@@ -135,13 +136,16 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(const __grid_co
 
   if (warp == kConsumerWarps) {
     // ------------------------------------------------------------------ producer
-    if (lane == 0) {
+    // Issuing one copy (free-stage wait, expect_tx, bulk copy) is a chain of a few hundred cycles for one
+    // thread; with small stages (FP8, narrow H) a single issuer cannot keep the ring full, so a few
+    // lanes issue side by side, lane j taking the rows whose local index is j modulo kProducerLanes.
+    if (lane < kProducerLanes) {
       int pair = 0;
       const char* base = nullptr;
       int pair_of_base = -1;
-      int issued = 0;
+      int issued = lane;                             // local index after this lane's last issued row
       bool ok = true;
-      for (int r = r0; r < r1 && ok; ++r, ++issued) {
+      for (int r = r0 + lane; r < r1 && ok; r += kProducerLanes, issued += kProducerLanes) {
         while (prefix[pair + 1] <= r) ++pair;
         if (pair != pair_of_base) {
           const int l = pair / P, p = pair % P;
@@ -170,7 +174,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(const __grid_co
       if (!ok) {
         // Let the consumers leave, then wait (bounded) for copies that are still landing.
         atomicExch(&s_abort, 1);
-        for (int n = max(0, issued - NS); n < issued; ++n)
+        for (int n = issued - kProducerLanes; n >= 0 && n >= issued - NS; n -= kProducerLanes)
           if (!mbar_wait(full + (n % NS), (n / NS) & 1)) atomicCAS(d.err, kErrNone, kErrDrain);
       }
     }

@@ -95,9 +95,9 @@ struct Elems<2> {                                   // bfloat16: the upper half 
   }
 };
 // FP8 E4M3: a stored byte q stands for q * 2^-8 (the stack-wide power-of-two scale is applied to
-// the dot products, not per element).  Decoding by cvt.e4m3x2 -> f16x2 -> f32 measured faster than
-// an integer-pipe bit construction (0.468 ms against 0.500 ms per 1.56 GB launch): at one byte per
-// weight the kernel is bound by instruction issue per element, not by HBM.
+// the dot products, not per element).  Decoding is cvt.e4m3x2 -> f16x2 -> f32; an integer-pipe bit
+// construction and packed fp32 FMAs were measured and are no faster: with several issuing producer
+// lanes the FP8 stream runs at the HBM rate, so the decode is not what bounds it.
 template <>
 struct Elems<1> {
   static constexpr int kVec = 16;
