@@ -29,9 +29,9 @@ import synth  # noqa: E402
 WORKLOAD = "dsv2lite"
 NOMINAL_HBM_GBS = 8000.0
 # DRAM bytes (read + write) per algorithmic byte of a resident-phase launch, from the ncu capture
-# summarised in profiles/ffn_stream_bf16_h2048_4layers_ncu_full.md (traffic grows in proportion to the
+# summarised in profiles/ffn_stream_{bf16,fp8}_h2048_4layers_ncu_full.md (traffic grows in proportion to the
 # blocks streamed); only valid for the kernel and shape it was taken on.
-TRAFFIC_RATIO = {("dsv2lite", 1): 1.008, ("dsv2lite_b32", 1): None}
+TRAFFIC_RATIO = {("dsv2lite", 1): 1.009, ("dsv2lite_fp8", 2): 1.018, ("dsv2lite_b32", 1): None}
 DTYPE_NAME = {0: "f32", 1: "bf16", 2: "fp8_e4m3"}      # weight storage; accumulation is always f32
 CLOCK_QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
                "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
