@@ -105,35 +105,38 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_batched_kernel(const __grid_c
 
   if (warp == kConsumerWarps) {
     // ------------------------------------------------------------------ producer
-    if (lane == 0) {
-      int n = 0;
-      bool ok = true;
-      for (int j = j0; j < n_items && ok; ++j) {
-        if (a.plan[kPlanHeader + 4 * j + 3] >= ub) break;
-        PieceInfo p;
-        if (!make_piece(a, j, ua, ub, p)) continue;
-        for (int blk = p.blk0; blk < p.blk1; ++blk, ++n) {
-          const int s = n % kStages;
-          if (n >= kStages) {
-            if (*(volatile int*)&s_abort || !mbar_wait(empty + s, ((n / kStages) - 1) & 1)) {
-              if (!*(volatile int*)&s_abort) atomicCAS(d.err, kErrNone, kErrWaitEmpty);
-              ok = false;
-              break;
-            }
+    // The whole warp walks the work list; lane 0 waits for the free stage and posts the byte count,
+    // then the stage's 24 row copies are issued by 24 lanes side by side (issued by one thread they
+    // take most of the time the stage's bytes need on the memory system).
+    int n = 0;
+    bool ok = true;
+    for (int j = j0; j < n_items && ok; ++j) {
+      if (a.plan[kPlanHeader + 4 * j + 3] >= ub) break;
+      PieceInfo p;
+      if (!make_piece(a, j, ua, ub, p)) continue;
+      for (int blk = p.blk0; blk < p.blk1; ++blk, ++n) {
+        const int s = n % kStages;
+        int go = 1;
+        if (lane == 0) {
+          if (n >= kStages && (*(volatile int*)&s_abort || !mbar_wait(empty + s, ((n / kStages) - 1) & 1))) {
+            if (!*(volatile int*)&s_abort) atomicCAS(d.err, kErrNone, kErrWaitEmpty);
+            go = 0;
+          } else {
+            mbar_expect_tx(full + s, G::kTxBytes);
           }
-          mbar_expect_tx(full + s, G::kTxBytes);
-          const char* src = p.base + (size_t)blk * (3 * kBlockCh * H * 2);
-          unsigned char* dst = stages + (size_t)s * G::kStageBytes;
-#pragma unroll 1
-          for (int r = 0; r < 3 * kBlockCh; ++r)
-            bulk_g2s(dst + r * G::kRowStride, src + (size_t)r * H * 2, H * 2, full + s);
         }
+        go = __shfl_sync(kFull, go, 0);
+        if (!go) { ok = false; break; }
+        const char* src = p.base + (size_t)blk * (3 * kBlockCh * H * 2);
+        unsigned char* dst = stages + (size_t)s * G::kStageBytes;
+        if (lane < 3 * kBlockCh) bulk_g2s(dst + lane * G::kRowStride, src + (size_t)lane * H * 2, H * 2, full + s);
       }
-      if (!ok) {
-        atomicExch(&s_abort, 1);
-        for (int m = max(0, n - kStages); m < n; ++m)
-          if (!mbar_wait(full + (m % kStages), (m / kStages) & 1)) atomicCAS(d.err, kErrNone, kErrDrain);
-      }
+    }
+    __syncwarp();
+    if (!ok && lane == 0) {
+      atomicExch(&s_abort, 1);
+      for (int m = max(0, n - kStages); m < n; ++m)
+        if (!mbar_wait(full + (m % kStages), (m / kStages) & 1)) atomicCAS(d.err, kErrNone, kErrDrain);
     }
     return;
   }
