@@ -281,16 +281,9 @@ __global__ void __launch_bounds__(256) combine_batched_kernel(BatchArgs a, float
 
 template <int H>
 cudaError_t launch_one(const BatchArgs& a, int grid, cudaStream_t st) {
-  // the dynamic shared-memory limit is a per-device attribute of the kernel
-  static bool configured[64] = {};
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-  if (!configured[dev]) {
-    cudaError_t e = cudaFuncSetAttribute(ffn_batched_kernel<H>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)Geo<H>::kSmem);
-    if (e != cudaSuccess) return e;
-    configured[dev] = true;
-  }
+  static std::atomic<bool> configured[kMaxDevices];
+  cudaError_t e0 = allow_dynamic_smem(ffn_batched_kernel<H>, Geo<H>::kSmem, configured);
+  if (e0 != cudaSuccess) return e0;
   BatchArgs b = a;
   b.tok_tile = kTokTile;
   b.blk_ch = kBlockCh;

@@ -531,21 +531,10 @@ bool encode_pool(EncodeTiledFn encode, CUtensorMap* gu, CUtensorMap* dn, const v
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// the dynamic shared-memory limit is a per-device attribute of a kernel
-template <typename K>
-cudaError_t allow_smem(K kernel, size_t bytes, bool* configured) {
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-  if (configured[dev]) return cudaSuccess;
-  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
-  if (e == cudaSuccess) configured[dev] = true;
-  return e;
-}
-
 template <int H>
 cudaError_t launch_tc(const BatchArgs& a, int grid, cudaStream_t st) {
-  static bool configured[64] = {};
-  cudaError_t e = allow_smem(ffn_batched_tc_kernel<H>, TcGeo<H>::kSmem, configured);
+  static std::atomic<bool> configured[kMaxDevices];
+  cudaError_t e = allow_dynamic_smem(ffn_batched_tc_kernel<H>, TcGeo<H>::kSmem, configured);
   if (e != cudaSuccess) return e;
   BatchArgs b = a;
   b.tok_tile = kTcTokTile;
@@ -560,8 +549,8 @@ cudaError_t launch_tc(const BatchArgs& a, int grid, cudaStream_t st) {
 template <int H>
 cudaError_t launch_retile(const TcMaps& maps, const RetileArgs& r, cudaStream_t st) {
   constexpr size_t kSmem = 1024 + (size_t)kRetileStages * kTileBytes + 64;
-  static bool configured[64] = {};
-  cudaError_t e = allow_smem(retile_kernel<H>, kSmem, configured);
+  static std::atomic<bool> configured[kMaxDevices];
+  cudaError_t e = allow_dynamic_smem(retile_kernel<H>, kSmem, configured);
   if (e != cudaSuccess) return e;
   retile_kernel<H><<<dim3(r.inter / kTcBlockCh, r.n), 32, kSmem, st>>>(maps, r);
   return cudaGetLastError();

@@ -327,16 +327,9 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const float* __restrict__ 
 template <int WB, int H>
 cudaError_t launch_one(const FfnArgs& a, int grid, cudaStream_t st) {
   const Layout lay = make_layout(H, WB);
-  // the dynamic shared-memory limit is a per-device attribute of the kernel
-  static bool configured[64] = {};
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-  if (!configured[dev]) {
-    cudaError_t e = cudaFuncSetAttribute(ffn_stream_kernel<WB, H>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)lay.total);
-    if (e != cudaSuccess) return e;
-    configured[dev] = true;
-  }
+  static std::atomic<bool> configured[kMaxDevices];
+  const cudaError_t e = allow_dynamic_smem(ffn_stream_kernel<WB, H>, lay.total, configured);
+  if (e != cudaSuccess) return e;
   ffn_stream_kernel<WB, H><<<grid, kThreads, lay.total, st>>>(a);
   return cudaGetLastError();
 }

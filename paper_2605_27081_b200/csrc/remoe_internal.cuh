@@ -4,6 +4,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "remoe.h"
 
 namespace remoe {
@@ -137,6 +139,20 @@ cudaError_t launch_combine(const FfnArgs& a, float* hidden_out, int layer0, int 
 // summation order.
 cudaError_t launch_rmsnorm(const float* h, float* x, int H, int rows, cudaStream_t st);
 size_t ffn_stream_smem_bytes(int H, int wbytes, int* stages_out);
+
+// Raises a kernel's dynamic shared-memory limit once per device (the limit is a per-device attribute of
+// the kernel).  `done` is a zero-initialised array of kMaxDevices flags owned by the caller, one array per
+// kernel; host threads may race here: the flags are atomic and setting the attribute twice is harmless.
+constexpr int kMaxDevices = 64;
+template <typename K>
+inline cudaError_t allow_dynamic_smem(K kernel, size_t bytes, std::atomic<bool>* done) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  if (done[dev].load(std::memory_order_acquire)) return cudaSuccess;
+  const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+  if (e == cudaSuccess) done[dev].store(true, std::memory_order_release);
+  return e;
+}
 bool ffn_stream_supported(int H, int wbytes);
 
 }  // namespace remoe
