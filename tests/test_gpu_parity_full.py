@@ -15,7 +15,7 @@ import synth
 pytestmark = pytest.mark.gpu
 
 
-def _full(name, rho, steps, distinct=None, sample_layers=(0, -1)):
+def _full(name, rho, steps, distinct=None, sample_layers=(0, -1), policy=None, beta=0.0):
     import torch
     from paper_2605_27081_b200.loader import LoadedWorkload
     from parity_util import StepChecker, oracle_for
@@ -27,9 +27,15 @@ def _full(name, rho, steps, distinct=None, sample_layers=(0, -1)):
     try:
         rhos = rho if isinstance(rho, (list, tuple)) else [rho]
         out = {}
+        pol_name = "lru"
+        if policy is not None:
+            wl.stack.set_policy(policy)
+            pol_name = {0: "lru", 1: "fifo", 2: "lfu"}[policy]
+        if beta:
+            wl.stack.set_reroute_beta(beta)
         for r, n in zip(rhos, steps if isinstance(steps, (list, tuple)) else [steps] * len(rhos)):
             wl.stack.cache_reset()
-            chk = StepChecker(wl, oracle_for(wl), torch)
+            chk = StepChecker(wl, oracle_for(wl, pol_name, beta), torch)
             hs = synth.HiddenStream(cfg["seed"], shape, r)
             sampled = {0, 1, n // 2, n - 1}
             layers = [l % shape.n_layers for l in sample_layers]
@@ -54,6 +60,17 @@ def test_dsv2lite_full_store_all_rhos():
     res = _full("dsv2lite", [0.9, 0.5, 0.0], [512, 512, 512])
     print("dsv2lite (near ties, max out err, uHR, EOR):", res)
     assert res[0.9][2] > res[0.5][2] > res[0.0][2]          # more temporal correlation, more hits
+
+
+@pytest.mark.parametrize("policy,beta", [(1, 0.0), (2, 0.0), (0, 0.5)])
+def test_dsv2lite_other_policies_and_rerouting_full_shape(policy, beta):
+    """FIFO, LFU (App. A.5) and the cache-aware rerouting bonus (App. F.2) at the benchmark's shape:
+    every step's ids, cache trace and counters against the oracle running the same policy."""
+    res = _full("dsv2lite", 0.5, 128, distinct=24, policy=policy, beta=beta)
+    print("dsv2lite policy", policy, "beta", beta, res)
+    if beta:
+        # the bonus keeps resident experts selected: more hits than plain LRU gets on this stream (0.46)
+        assert res[0.5][2] > 0.48
 
 
 def test_dsv2lite_multi_step_call_full_shape():
