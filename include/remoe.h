@@ -263,12 +263,13 @@ int remoe_launch_count(remoe_stack*, uint64_t* launches);
  *                          the [I, 3, H] layout above, 16-byte aligned, owned by the caller
  *   inter                  HOST array: I of each block, 1 .. REMOE_STATIC_MAX_INTER
  *   scales                 HOST array: gate weight (or shared-expert scale) of each block
- *   hidden_in_dev          DEVICE [H] float32;  hidden_out_dev  DEVICE [H] float32 (overwritten)
+ *   hidden_in_dev          DEVICE [H] float32;  hidden_out_dev  DEVICE [H] float32 (overwritten;
+ *                          may be the same buffer as hidden_in_dev)
  *
  * The host arrays are read before the call returns.  The result is complete when `cuda_stream`
- * reaches the end of the call's work.  Sizes beyond the limits above, or a hidden width the
- * kernels are not built for, are refused with REMOE_E_UNSUPPORTED before anything is launched;
- * bad pointers with REMOE_E_ARG.  The first call on each device also looks up the scratch
+ * reaches the end of the call's work.  Sizes beyond the limits above, a hidden width the kernels
+ * are not built for, or REMOE_FP8_E4M3 blocks are refused with REMOE_E_UNSUPPORTED before anything
+ * is launched; bad pointers and unknown element types with REMOE_E_ARG.  The first call on each device also looks up the scratch
  * array's device address and sets kernel attributes for that device (with that device
  * current), so make that first call outside any stream capture.  All calls on a device share
  * the one scratch array: calls whose kernels could run at the same time (different streams

@@ -18,21 +18,35 @@ class LoadedWorkload:
 
     ``distinct_experts``: generate only that many distinct routed blocks per layer and let
     the remaining expert ids alias them (saves host memory and generation time when only
-    timing matters); ``None`` generates all N blocks per layer.
+    timing matters); ``None`` generates all N blocks per layer.  ``store_of``: borrow the pinned
+    expert store of another loaded workload whose expert blocks are the same tensors (same seed,
+    layers, hidden, intermediate size and element type; e.g. the batched variant of a stack) instead
+    of generating it again; that workload must outlive this one.
     """
 
     def __init__(self, shape: synth.Shape, cache_slots: int, seed: int = 0, stream: int | None = None,
-                 distinct_experts: int | None = None, threads: int | None = None):
+                 distinct_experts: int | None = None, threads: int | None = None,
+                 store_of: "LoadedWorkload | None" = None):
         self.shape, self.cache_slots, self.seed = shape, cache_slots, seed
         L, N = shape.n_layers, shape.n_routed
-        nd = N if distinct_experts is None else min(N, int(distinct_experts))
-        self.n_distinct = nd
         elems = synth.expert_block_elems(shape.hidden, shape.inter_routed)
         np_dt = {0: np.float32, 1: np.uint16, 2: np.uint8}[shape.weight_dtype]
-        gen_shape = synth.Shape(**{**shape.asdict(), "n_routed": nd})
-        self._store_t = torch.empty(L * nd * elems * shape.elem_bytes, dtype=torch.uint8, pin_memory=True)
-        self.store = self._store_t.numpy().view(np_dt).reshape(L, nd, elems)
-        synth.fill_expert_store(seed, gen_shape, self.store, threads=threads)
+        if store_of is not None:
+            o = store_of.shape
+            same = (o.n_layers, o.hidden, o.inter_routed, o.weight_dtype, o.n_routed, store_of.seed) == \
+                   (L, shape.hidden, shape.inter_routed, shape.weight_dtype, N, seed)
+            if not same:
+                raise ValueError("store_of: the two workloads do not have the same expert blocks")
+            nd = store_of.n_distinct
+            self.n_distinct = nd
+            self._store_t, self.store = store_of._store_t, store_of.store
+        else:
+            nd = N if distinct_experts is None else min(N, int(distinct_experts))
+            self.n_distinct = nd
+            gen_shape = synth.Shape(**{**shape.asdict(), "n_routed": nd})
+            self._store_t = torch.empty(L * nd * elems * shape.elem_bytes, dtype=torch.uint8, pin_memory=True)
+            self.store = self._store_t.numpy().view(np_dt).reshape(L, nd, elems)
+            synth.fill_expert_store(seed, gen_shape, self.store, threads=threads)
         self.routers = [synth.gen_router(seed, shape, l) for l in range(L)]
         self.shared_gates = [synth.gen_shared_gate(seed, shape, l) for l in range(L)] if shape.shared_gate else None
         self.shared = [[synth.gen_shared_block(seed, shape, l, i) for i in range(shape.n_shared)] for l in range(L)]

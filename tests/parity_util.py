@@ -10,12 +10,30 @@ TOL = {0: 1e-4, 1: 2e-2, 2: 2e-2}  # max|d| / max|ref| : float32, bf16, fp8 weig
 NEAR_TIE = 1e-5                   # logit gap below which the selected list may differ
 
 
+def near_tie_kind(z, o_ids, ids):
+    """How the library's list `ids` relates to the oracle's `o_ids` for the oracle logits `z`:
+    "same", "boundary", "swap" or None (not acceptable).
+
+    A list is acceptable only if it holds K distinct expert ids inside [0, N) and, at every rank, an
+    expert whose oracle logit is within NEAR_TIE of the oracle's expert at that rank.  "boundary": the
+    selected SET differs (rank K against rank K+1 -- the case the acceptance rule names); "swap": the
+    same set with two near-tied ranks exchanged.  Both can only happen when fp32 rounding of the logits
+    meets a gap that small (Top-K stability, App. C)."""
+    o_ids = [int(e) for e in o_ids]
+    ids = [int(e) for e in ids]
+    n = len(z)
+    if len(ids) != len(o_ids) or len(set(ids)) != len(ids) or any(e < 0 or e >= n for e in ids):
+        return None
+    if ids == o_ids:
+        return "same"
+    if not all(abs(float(z[a]) - float(z[b])) < NEAR_TIE for a, b in zip(o_ids, ids)):
+        return None
+    return "swap" if set(ids) == set(o_ids) else "boundary"
+
+
 def near_tie_only(z, o_ids, ids):
-    """True if the library's list `ids` differs from the oracle's `o_ids` only by near-ties: at every
-    rank the two lists hold experts whose oracle logits are within NEAR_TIE of each other.  That covers
-    the boundary case (rank K against rank K+1) and two selected experts swapping ranks; both can only
-    happen when fp32 rounding of the logits meets a gap that small (Top-K stability, App. C)."""
-    return all(abs(float(z[int(a)]) - float(z[int(b)])) < NEAR_TIE for a, b in zip(o_ids, ids))
+    """True if `ids` is the oracle's list or differs from it only by near-ties (see near_tie_kind)."""
+    return near_tie_kind(z, o_ids, ids) is not None
 
 
 def widen(shape, a, router=False):
@@ -61,9 +79,21 @@ class StepChecker:
         self.d_out = torch.empty_like(self.d_in)
         self.d_ids = torch.empty((self.L, self.B, self.K), dtype=torch.int32, device=device)
         self.d_g = torch.empty((self.L, self.B, self.K), dtype=torch.float32, device=device)
-        self.near_ties = 0
+        self.near_ties = 0              # = boundary flips + rank swaps
+        self.boundary_flips = 0         # selected set differs across a rank-K / rank-K+1 gap below NEAR_TIE
+        self.rank_swaps = 0             # same set, two near-tied ranks exchanged
         self.max_out_err = 0.0
         self.max_gate_err = 0.0
+
+    def _count_tie(self, kind):
+        self.near_ties += 1
+        if kind == "boundary":
+            self.boundary_flips += 1
+        else:
+            self.rank_swaps += 1
+
+    def tie_report(self):
+        return f"near ties {self.near_ties} (boundary flips {self.boundary_flips}, rank swaps {self.rank_swaps})"
 
     def gpu_step(self, h, host_api=False):
         t = self.torch
@@ -84,20 +114,33 @@ class StepChecker:
 
     def compare(self, h, ids, g, out, ffn="selected", ffn_layers=None, check_trace=True):
         """Sets what the library returned for the layer inputs `h` beside the oracle's step on them."""
+        r = self.oracle_step(h, ids, ffn, ffn_layers)
+        self.check_against(r, g, out, ffn, ffn_layers, check_trace)
+        return r, (ids, g, out)
+
+    def oracle_step(self, h, ids, ffn="selected", ffn_layers=None):
+        """The oracle's step on `h`, given only the ids the library selected (needed beforehand to find
+        near-ties): selected lists are compared here, everything else in check_against."""
         # First pass of the oracle on a copy of nothing: we need margins before committing,
         # so route without touching state.
         override = {}
         for l in range(self.L):
             for b in range(self.B):
                 o_ids, _, margin, z, _ = self.o.route(l, h[l, b])
-                if list(o_ids) != list(ids[l, b]):
-                    assert near_tie_only(z, o_ids, ids[l, b]), (
-                        f"ids differ at layer {l} seq {b} beyond near-ties (boundary margin {margin}): "
-                        f"{[int(e) for e in o_ids]} vs {[int(e) for e in ids[l, b]]}")
-                    self.near_ties += 1
+                kind = near_tie_kind(z, o_ids, ids[l, b])
+                assert kind is not None, (
+                    f"ids differ at layer {l} seq {b} beyond near-ties (boundary margin {margin}): "
+                    f"{[int(e) for e in o_ids]} vs {[int(e) for e in ids[l, b]]}")
+                if kind != "same":
+                    self._count_tie(kind)
                     override[(l, b)] = [int(e) for e in ids[l, b]]
         r = self.o.step(h, ffn=ffn, id_override=override or None, ffn_layers=ffn_layers)
         assert np.array_equal(r["ids"], ids)
+        return r
+
+    def check_against(self, r, g, out, ffn="selected", ffn_layers=None, check_trace=True):
+        """Gate weights, cache trace, reuse mass and outputs of the library's last step against the
+        oracle's result `r` for the same step."""
         ge = float(np.max(np.abs(r["gates"] - g) / np.maximum(np.abs(r["gates"]), 1e-30)))
         self.max_gate_err = max(self.max_gate_err, ge)
         assert ge <= 1e-4, f"gate weights off by {ge}"
@@ -118,6 +161,24 @@ class StepChecker:
                 e = rel_err(out[l], r["out"][l])
                 self.max_out_err = max(self.max_out_err, e)
                 assert e <= tol, f"layer {l}: output error {e} > {tol}"
+
+    def step_overlapped(self, h, ffn=None, ffn_layers=None):
+        """Same checks as step(), with the oracle's share of the work done while the GPU is still busy
+        with the step: the selected ids and gate weights are final when remoe_decode_step returns (the
+        call waits for the routing kernels), so they are read on a second stream and the oracle steps on
+        the host while the library's fetches and expert kernels run.  For long host-link-bound runs."""
+        t = self.torch
+        if not hasattr(self, "side"):
+            self.side = t.cuda.Stream()
+        self.d_in.copy_(t.from_numpy(np.ascontiguousarray(h)))
+        self.wl.stack.decode_step(self.d_in, self.d_out, self.d_ids, self.d_g)
+        with t.cuda.stream(self.side):
+            ids = self.d_ids.cpu().numpy()
+            g = self.d_g.cpu().numpy()
+        r = self.oracle_step(h, ids, ffn, ffn_layers)
+        t.cuda.synchronize()
+        out = self.d_out.cpu().numpy() if ffn is not None else None
+        self.check_against(r, g, out, ffn, ffn_layers)
         return r, (ids, g, out)
 
     def step_chained_batched(self, h0):
@@ -162,9 +223,10 @@ class StepChecker:
             if not bad:
                 break
             l = bad[0]
-            assert near_tie_only(trial["logits"][l, 0], trial["ids"][l, 0], ids[l, 0]), (
+            kind = near_tie_kind(trial["logits"][l, 0], trial["ids"][l, 0], ids[l, 0])
+            assert kind is not None, (
                 f"chained ids differ at layer {l} beyond near-ties, boundary margin {trial['margin'][l, 0]}")
-            self.near_ties += 1
+            self._count_tie(kind)
             override[(l, 0)] = [int(e) for e in ids[l, 0]]
         r = self.o.step(np.asarray(h0).reshape(1, H), ffn="selected", chained=True, id_override=override or None)
         assert np.array_equal(r["ids"], ids)

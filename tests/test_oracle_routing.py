@@ -116,7 +116,7 @@ def test_unique_in_order_and_overlap():
 def test_near_tie_rule_of_the_parity_harness():
     """What the GPU parity tests accept as a near-tie: lists that differ only where two oracle logits
     are closer than 1e-5 (boundary flip or two ranks swapped), nothing else."""
-    from parity_util import near_tie_only
+    from parity_util import near_tie_kind, near_tie_only
     z = np.array([3.0, 2.0, 2.0 - 4e-6, 1.0, 1.0 - 2e-6, -5.0])
     ids, _ = orc.topk_select(z, 4)
     assert list(ids) == [0, 1, 2, 3]
@@ -126,3 +126,14 @@ def test_near_tie_rule_of_the_parity_harness():
     assert not near_tie_only(z, ids, [1, 0, 2, 3])        # a gap of 1.0 is not a tie
     assert not near_tie_only(z, ids, [0, 1, 2, 5])
     assert not near_tie_only(z, ids, [0, 1, 3, 2])        # 2 and 3 are 1.0 apart
+    # a valid list holds K distinct ids inside [0, N): near-tied logits excuse none of these
+    assert not near_tie_only(z, ids, [0, 1, 1, 3])        # expert 1 twice (1 and 2 are near-tied)
+    assert not near_tie_only(z, ids, [0, 2, 2, 3])
+    assert not near_tie_only(z, ids, [0, 1, 2, 6]) and not near_tie_only(z, ids, [0, 1, 2, -1])
+    assert not near_tie_only(z, ids, [0, 1, 2]) and not near_tie_only(z, ids, [0, 1, 2, 3, 4])
+    # and the two accepted kinds are told apart
+    assert near_tie_kind(z, ids, [0, 1, 2, 3]) == "same"
+    assert near_tie_kind(z, ids, [0, 2, 1, 3]) == "swap"
+    assert near_tie_kind(z, ids, [0, 1, 2, 4]) == "boundary"
+    assert near_tie_kind(z, ids, [0, 2, 1, 4]) == "boundary"
+    assert near_tie_kind(z, ids, [1, 0, 2, 3]) is None
