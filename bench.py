@@ -3,15 +3,20 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--rho R] [--impl ours|reference]
 
-A "step" is one decode step: one token through all MoE layers of the DeepSeek-V2-Lite-shaped
-stack (26 layers, hidden 2048, 64 routed experts top-6 + 2 shared, intermediate 1408, bf16
-weights, 16 cache slots per layer, LRU), driven by seeded AR(1) hidden states.  One JSON line
-is printed by rank 0.  With N > 1 every rank runs an independent replica (the path has no
-exchange step); the time is the maximum over ranks and the value the sum of tokens.
+A "step" is one decode step: one token (or one token of each of B sequences) through all MoE layers of
+a stack, driven by seeded AR(1) hidden states.  The line's `value` is measured on the
+DeepSeek-V2-Lite-shaped batch-1 stack (26 layers, hidden 2048, 64 routed experts top-6 + 2 shared,
+intermediate 1408, bf16 weights, 16 cache slots per layer, LRU) from device-resident inputs: cold cache,
+W warm-up steps, then exactly K timed steps; the same steps are then repeated through host buffers
+(`e2e`).  Both are run `--repeats` times on identical inputs and the median repeat is reported with the
+minimum and maximum.  One JSON line is printed by rank 0.  With N > 1 every rank runs an independent
+replica (the path has no exchange step); the time is the maximum over ranks and the value the sum of
+tokens.  The other workloads (`other_workloads` in the line) are short runs of the same protocol.
 """
 from __future__ import annotations
 
 import argparse
+import copy
 import json
 import os
 import subprocess
@@ -28,14 +33,23 @@ import synth  # noqa: E402
 
 WORKLOAD = "dsv2lite"
 NOMINAL_HBM_GBS = 8000.0
-# DRAM bytes (read + write) per algorithmic byte of a resident-phase launch, from the ncu capture
-# summarised in profiles/ffn_stream_{bf16,fp8}_h2048_4layers_ncu_full.md (traffic grows in proportion to the
-# blocks streamed); only valid for the kernel and shape it was taken on.
-TRAFFIC_RATIO = {("dsv2lite", 1): 1.009, ("dsv2lite_fp8", 2): 1.018, ("dsv2lite_b32", 1): None}
-DTYPE_NAME = {0: "f32", 1: "bf16", 2: "fp8_e4m3"}      # weight storage; accumulation is always f32
+COLD_STEPS = 32
+# DRAM bytes (read + write) per algorithmic byte of a resident-phase launch of the expert kernel, from the
+# profiler captures of that kernel on a shallower stack of the same layer shape (traffic grows in proportion
+# to the blocks streamed).  Keyed by (workload, kernel); valid only for the kernel it was taken on, so an
+# entry is dropped (None) when that kernel changes.
+TRAFFIC_RATIO = {
+    ("dsv2lite", "ffn_stream_kernel<bf16,2048>"): 1.009,
+    ("dsv2lite_fp8", "ffn_stream_kernel<fp8_e4m3,2048>"): 1.018,
+}
+DTYPE_NAME = {0: "f32", 1: "bf16", 2: "fp8_e4m3", 3: "int4_g32"}      # weight storage; accumulation is always f32
 CLOCK_QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
                "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
                "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+
+def metric_name(shape):
+    return f"decode tokens/s (batch {shape.batch}, MoE stack)"
 
 
 def kernel_name(shape):
@@ -63,7 +77,7 @@ class ClockSampler:
         self.f = open(self.path, "w")
         try:
             self.p = subprocess.Popen(["nvidia-smi", f"--id={index}", f"--query-gpu={CLOCK_QUERY}",
-                                       "--format=csv,noheader,nounits", "-lms", "200"],
+                                       "--format=csv,noheader,nounits", "-lms", "100"],
                                       stdout=self.f, stderr=subprocess.DEVNULL)
         except Exception:
             self.p = None
@@ -98,50 +112,109 @@ class ClockSampler:
                 "samples": len(sm), "power_w_max": float(max(power))}
 
 
-def oracle_sample(shape, cache_slots, seed, rho, layers, steps, warmup=0):
-    """Time the CPU oracle (as it stands) on `layers` layers for `steps` decode steps."""
+def merge_clocks(per_repeat):
+    got = [c for c in per_repeat if c and c.get("sm_mhz") is not None]
+    if not got:
+        return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "per_repeat_sm_mhz": []}
+    return {"sm_mhz": float(np.median([c["sm_mhz"] for c in got])), "sm_max_mhz": max(c["sm_max_mhz"] for c in got),
+            "reasons": sorted(set().union(*[set(c["reasons"]) for c in got])),
+            "samples": sum(c["samples"] for c in got), "power_w_max": max(c["power_w_max"] for c in got),
+            "per_repeat_sm_mhz": [c["sm_mhz"] for c in got]}
+
+
+# ------------------------------------------------------------------------------- CPU oracle legs
+
+def _blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        return max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        return 1
+
+
+def oracle_sample(shape, cache_slots, seed, rho, layers, steps, warm_steps, mode="selected", threads=None, store=None):
+    """Time the CPU oracle, as it stands, on the first `layers` layers for `steps` decode steps after
+    `warm_steps` steps that fill its caches (integer parts only).  `threads`: limit of the BLAS pool
+    (None = whatever the process has).  Returns (seconds, threads the BLAS pool had)."""
     from oracle import remoe_oracle as orc
     sub = synth.Shape(**{**shape.asdict(), "n_layers": layers})
-
-    def widen(a):
-        return synth.bf16_bits_to_f32(a) if shape.weight_dtype == 1 else a
-
-    routers = [widen(synth.gen_router(seed, shape, l)) for l in range(layers)]
+    routers = [synth.widen(shape, synth.gen_router(seed, shape, l), True) for l in range(layers)]
+    gates = [synth.widen(shape, synth.gen_shared_gate(seed, shape, l), True) for l in range(layers)] \
+        if shape.shared_gate else None
     blocks = {}
 
     def ew(l, e):
         if (l, e) not in blocks:
-            blocks[(l, e)] = widen(synth.gen_expert_block(seed, shape, l, e))
+            raw = store(l, e) if store is not None else synth.gen_expert_block(seed, shape, l, e)
+            blocks[(l, e)] = synth.widen(shape, raw)
         return synth.expert_matrices(blocks[(l, e)], shape.hidden, shape.inter_routed)
 
-    shared = {(l, i): widen(synth.gen_shared_block(seed, shape, l, i)) for l in range(layers)
+    shared = {(l, i): synth.widen(shape, synth.gen_shared_block(seed, shape, l, i)) for l in range(layers)
               for i in range(shape.n_shared)}
 
     def sw(l, i):
         return synth.expert_matrices(shared[(l, i)], shape.hidden, shape.inter_shared)
 
-    st = orc.OracleStack(sub, cache_slots, routers, ew, sw)
+    st = orc.OracleStack(sub, cache_slots, routers, ew, sw, shared_gates=gates)
     hs = synth.HiddenStream(seed, shape, rho)
-    hidden = [hs.step()[:layers] for _ in range(warmup + steps)]
-    # weights are generated before the clock starts (the GPU side also starts with its store ready)
-    for t in range(warmup + steps):
+    hidden = [hs.step()[:layers] for _ in range(warm_steps + steps)]
+    # every weight the timed steps touch is widened before the clock starts (the GPU side also starts with
+    # its store ready): a dry run of the integer parts tells which
+    for t in range(warm_steps + steps):
         r = st.step(hidden[t], ffn=None)
-        for l in range(layers):
-            for e in r["ids"][l].reshape(-1):
-                ew(l, int(e))
+        if t >= warm_steps:
+            for l in range(layers):
+                for e in (range(shape.n_routed) if mode == "dense" else r["ids"][l].reshape(-1)):
+                    ew(l, int(e))
     st.reset()
-    for t in range(warmup):
-        st.step(hidden[t], ffn="selected")
-    t0 = time.perf_counter()
-    for t in range(warmup, warmup + steps):
-        st.step(hidden[t], ffn="selected")
-    dt = time.perf_counter() - t0
-    try:
-        from threadpoolctl import threadpool_info
-        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
-    except Exception:
-        cores = 1
-    return dt, cores
+    for t in range(warm_steps):
+        st.step(hidden[t], ffn=None)
+
+    def timed():
+        t0 = time.perf_counter()
+        for t in range(warm_steps, warm_steps + steps):
+            st.step(hidden[t], ffn=mode)
+        return time.perf_counter() - t0
+
+    if threads is not None:
+        try:
+            from threadpoolctl import threadpool_limits
+            with threadpool_limits(limits=threads):
+                return timed(), threads
+        except Exception:
+            pass
+    return timed(), _blas_threads()
+
+
+def cpu_baseline_legs(shape, C, seed, rho, store):
+    """The oracle on a bounded sample of the headline workload: selected-experts-only on one thread and on
+    all host cores (the reported baseline), and dense-and-mask on the tiny configuration in full and on a
+    prefix of this one."""
+    layers, steps, warm = min(8, shape.n_layers), 8, 8
+    affinity = len(os.sched_getaffinity(0))
+    dt_all, thr_all = oracle_sample(shape, C, seed, rho, layers, steps, warm, store=store)
+    dt_one, _ = oracle_sample(shape, C, seed, rho, min(2, layers), steps, warm, threads=1, store=store)
+    per_all = dt_all / steps * shape.n_layers / layers
+    per_one = dt_one / steps * shape.n_layers / min(2, layers)
+    tiny = synth.config("tiny_fp32")
+    dt_tiny, _ = oracle_sample(tiny["shape"], tiny["cache_slots"], tiny["seed"], tiny["rhos"][0], 1, tiny["steps"], 0,
+                               mode="dense")
+    dt_dense, _ = oracle_sample(shape, C, seed, rho, 1, 8, 0, mode="dense", store=store)
+    return {
+        "value": shape.batch / per_all, "unit": "tokens/s", "cores": thr_all, "kind": "oracle",
+        "sample": (f"steps {warm + 1}..{warm + steps} of the workload (caches warm) over the first {layers} of "
+                   f"{shape.n_layers} layers, time scaled by {shape.n_layers}/{layers}; selected-experts-only fp64 "
+                   f"oracle, numpy BLAS pool of {thr_all} threads"),
+        "host_cores_sched_getaffinity": affinity,
+        "one_thread": {"value": shape.batch / per_one, "unit": "tokens/s",
+                       "sample": f"same steps over the first {min(2, layers)} layers, BLAS pool limited to 1 thread"},
+        "dense_and_mask": {
+            "tiny_fp32_full": {"steps": tiny["steps"], "seconds": dt_tiny, "tokens_per_s": tiny["steps"] / dt_tiny},
+            "headline_prefix": {"steps": 8, "layers": 1, "seconds": dt_dense,
+                                "tokens_per_s_scaled": shape.batch / (dt_dense / 8 * shape.n_layers),
+                                "note": "every routed expert evaluated and masked, first 8 steps, first layer, "
+                                        f"time scaled by {shape.n_layers}"}},
+    }
 
 
 def run_reference(args, rank, world):
@@ -156,10 +229,11 @@ def run_reference(args, rank, world):
     dt, cores = oracle_sample(shape, cfg["cache_slots"], cfg["seed"], args.rho, layers, args.steps, args.warmup)
     per_step = dt / args.steps * shape.n_layers / layers
     value = shape.batch / per_step
-    sample = (f"{args.steps} decode steps over the first {layers} of {shape.n_layers} layers, time scaled by "
-              f"{shape.n_layers}/{layers}; selected-experts-only fp64 oracle")
+    sample = (f"{args.steps} decode steps (after {args.warmup} cache-warming steps) over the first {layers} of "
+              f"{shape.n_layers} layers, time scaled by {shape.n_layers}/{layers}; selected-experts-only fp64 oracle, "
+              f"numpy BLAS pool of {cores} threads, {len(os.sched_getaffinity(0))} host cores available")
     line = {
-        "impl": "reference", "metric": "decode tokens/s (batch 1, MoE stack)", "value": value, "unit": "tokens/s",
+        "impl": "reference", "metric": metric_name(shape), "value": value, "unit": "tokens/s",
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_step * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": args.workload, "rho": args.rho, "cache_slots": cfg["cache_slots"], "batch": shape.batch},
@@ -169,73 +243,119 @@ def run_reference(args, rank, world):
     print(json.dumps(line), flush=True)
 
 
-def timed_steps(torch, wl, stream, d_hidden, d_out, d_ids, d_g, first, count):
-    """Run `count` decode steps from device-resident inputs; returns elapsed ms (CUDA events)."""
-    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.synchronize()
-    with torch.cuda.stream(stream):
-        a.record(stream)
-        for t in range(first, first + count):
-            wl.stack.decode_step(d_hidden[t], d_out, d_ids, d_g)
-        b.record(stream)
-    torch.cuda.synchronize()
-    return a.elapsed_time(b)
+# ------------------------------------------------------------------------------- GPU legs
 
+class Leg:
+    """Device buffers and counters for timed legs on one stack."""
 
-def run_rho(torch, wl, stream, shape, seed, rho, steps, warmup, with_e2e, prewarm_iid=0):
-    """Cold cache -> warm-up -> K timed steps (device inputs) [-> K timed steps through host buffers]."""
-    L, H, K, B = shape.n_layers, shape.hidden, shape.top_k, shape.batch
-    n = warmup + steps * (2 if with_e2e else 1)
-    hidden = synth.HiddenStream(seed, shape, rho).take(n)
-    h_pinned = torch.from_numpy(hidden).pin_memory()
-    d_hidden = h_pinned.to("cuda", non_blocking=False)
-    d_out = torch.empty((L, B, H), dtype=torch.float32, device="cuda")
-    d_ids = torch.empty((L, B, K), dtype=torch.int32, device="cuda")
-    d_g = torch.empty((L, B, K), dtype=torch.float32, device="cuda")
-    st = wl.stack
-    st.cache_reset()
-    st.set_profiling(False)
-    torch.cuda.synchronize()
-    if prewarm_iid:
-        # independent hidden states touch every expert quickly, so a cache as large as the expert
-        # set ends up holding all of them before the measured stream starts
-        d_pre = torch.from_numpy(synth.HiddenStream(seed + 1, shape, 0.0).take(prewarm_iid)).to("cuda")
-        timed_steps(torch, wl, stream, d_pre, d_out, d_ids, d_g, 0, prewarm_iid)
-    timed_steps(torch, wl, stream, d_hidden, d_out, d_ids, d_g, 0, warmup)
-    c0, l0 = st.cache_stats(), st.launch_count()
-    ov0 = st.reuse_stats()
-    st.set_profiling(True)
-    ms = timed_steps(torch, wl, stream, d_hidden, d_out, d_ids, d_g, warmup, steps)
-    c1, l1 = st.cache_stats(), st.launch_count()
-    ov1 = st.reuse_stats()
-    k_res = st.kernel_time(0)
-    k_miss = st.kernel_time(1)
-    st.set_profiling(False)
-    res = {
-        "ms": ms, "launches": l1 - l0,
-        "uniq_hits": c1["uniq_hits"] - c0["uniq_hits"], "uniq_misses": c1["uniq_misses"] - c0["uniq_misses"],
-        "h2d_bytes": c1["h2d_bytes"] - c0["h2d_bytes"],
-        "overlap": ov1[0] - ov0[0], "pairs": ov1[1] - ov0[1],
-        "kernel_resident": k_res, "kernel_miss": k_miss,
-    }
-    if with_e2e:
-        out_h = torch.empty((L, B, H), dtype=torch.float32).pin_memory().numpy()
-        ids_h = torch.empty((L, B, K), dtype=torch.int32).pin_memory().numpy()
-        g_h = torch.empty((L, B, K), dtype=torch.float32).pin_memory().numpy()
-        hp = h_pinned.numpy()
+    def __init__(self, torch, wl, stream, shape):
+        self.torch, self.wl, self.stream, self.shape = torch, wl, stream, shape
+        L, H, K, B = shape.n_layers, shape.hidden, shape.top_k, shape.batch
+        self.d_out = torch.empty((L, B, H), dtype=torch.float32, device="cuda")
+        self.d_ids = torch.empty((L, B, K), dtype=torch.int32, device="cuda")
+        self.d_g = torch.empty((L, B, K), dtype=torch.float32, device="cuda")
+        self.out_h = torch.empty((L, B, H), dtype=torch.float32).pin_memory().numpy()
+        self.ids_h = torch.empty((L, B, K), dtype=torch.int32).pin_memory().numpy()
+        self.g_h = torch.empty((L, B, K), dtype=torch.float32).pin_memory().numpy()
+
+    def snapshot(self):
+        st = self.wl.stack
+        c = st.cache_stats()
+        ov = st.reuse_stats()
+        return dict(c, overlap=ov[0], pairs=ov[1], launches=st.launch_count())
+
+    @staticmethod
+    def delta(a, b):
+        return {k: b[k] - a[k] for k in ("uniq_hits", "uniq_misses", "h2d_bytes", "overlap", "pairs", "launches")}
+
+    def device_steps(self, d_hidden, first, count):
+        """`count` decode steps from device-resident inputs; elapsed ms (CUDA events on the stack's stream)."""
+        torch = self.torch
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        with torch.cuda.stream(self.stream):
+            a.record(self.stream)
+            for t in range(first, first + count):
+                self.wl.stack.decode_step(d_hidden[t], self.d_out, self.d_ids, self.d_g)
+            b.record(self.stream)
+        torch.cuda.synchronize()
+        return a.elapsed_time(b)
+
+    def host_steps(self, h_hidden, first, count):
+        """The same steps through host buffers: inputs copied in, outputs read back, every step."""
+        torch = self.torch
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.synchronize()
         t0 = time.perf_counter()
-        a.record(stream)
-        for t in range(warmup + steps, warmup + 2 * steps):
-            st.decode_step_host(hp[t], out_h, ids_h, g_h)
-        b.record(stream)
+        a.record(self.stream)
+        for t in range(first, first + count):
+            self.wl.stack.decode_step_host(h_hidden[t], self.out_h, self.ids_h, self.g_h)
+        b.record(self.stream)
         torch.cuda.synchronize()
         wall = (time.perf_counter() - t0) * 1e3
-        res["e2e_ms"] = max(a.elapsed_time(b), wall)
-        res["e2e_in_bytes"] = hp[0].nbytes
-        res["e2e_out_bytes"] = out_h.nbytes + ids_h.nbytes + g_h.nbytes
-    return res
+        return max(a.elapsed_time(b), wall)
+
+
+def run_protocol(torch, wl, stream, shape, seed, rho, steps, warmup, repeats, with_e2e, with_cold, local_rank=None,
+                 prewarm_iid=0):
+    """Per repeat, all from the same hidden states: [cold cache -> COLD_STEPS timed steps]; cold cache -> W
+    warm-up steps -> K timed steps from device inputs; [cold cache -> W warm-up steps -> the same K steps
+    through host buffers].  Returns the list of per-repeat results."""
+    n = max(warmup + steps, COLD_STEPS if with_cold else 0)
+    hidden = synth.HiddenStream(seed, shape, rho).take(n)
+    h_pinned = torch.from_numpy(hidden).pin_memory()
+    d_hidden = h_pinned.to("cuda", non_blocking=False)
+    hp = h_pinned.numpy()
+    st = wl.stack
+    leg = Leg(torch, wl, stream, shape)
+    st.set_profiling(False)
+    d_pre = None
+    if prewarm_iid:
+        # independent hidden states touch every expert quickly, so a cache as large as the expert set ends
+        # up holding all of them before the measured stream starts
+        d_pre = torch.from_numpy(synth.HiddenStream(seed + 1, shape, 0.0).take(prewarm_iid)).to("cuda")
+
+    def fresh():
+        st.cache_reset()
+        torch.cuda.synchronize()
+        if d_pre is not None:
+            leg.device_steps(d_pre, 0, prewarm_iid)
+
+    reps = []
+    for rep in range(repeats):
+        sampler = ClockSampler(local_rank) if local_rank is not None else None
+        res = {}
+        if with_cold:
+            fresh()
+            s0 = leg.snapshot()
+            ms = leg.device_steps(d_hidden, 0, COLD_STEPS)
+            res["cold"] = dict(Leg.delta(s0, leg.snapshot()), ms=ms, steps=COLD_STEPS)
+        fresh()
+        leg.device_steps(d_hidden, 0, warmup)
+        s0 = leg.snapshot()
+        st.set_profiling(True)
+        res["ms"] = leg.device_steps(d_hidden, warmup, steps)
+        res.update(Leg.delta(s0, leg.snapshot()))
+        res["kernel_resident"] = st.kernel_time(0)
+        res["kernel_miss"] = st.kernel_time(1)
+        st.set_profiling(False)
+        if with_e2e:
+            fresh()
+            for t in range(warmup):
+                st.decode_step_host(hp[t], leg.out_h, leg.ids_h, leg.g_h)
+            s0 = leg.snapshot()
+            ms = leg.host_steps(hp, warmup, steps)
+            res["e2e"] = dict(Leg.delta(s0, leg.snapshot()), ms=ms, in_bytes=hp[0].nbytes,
+                              out_bytes=leg.out_h.nbytes + leg.ids_h.nbytes + leg.g_h.nbytes)
+        if sampler is not None:
+            res["clocks"] = sampler.stop()
+        reps.append(res)
+    return reps
+
+
+def median_rep(reps, key="ms"):
+    order = sorted(range(len(reps)), key=lambda i: reps[i][key] if key == "ms" else reps[i][key]["ms"])
+    return reps[order[len(order) // 2]]
 
 
 def measure_h2d(torch, nbytes, reps=12):
@@ -281,6 +401,78 @@ def reduce_over_ranks(dist, maxima: dict, sums: dict, device):
     return out
 
 
+def step_roofline(shape, r, steps, peak_hbm, h2d_peak):
+    """bytes one step must move: resident experts + shared + router from HBM, misses over the host link"""
+    S_e = synth.expert_block_bytes(shape)
+    router = shape.n_layers * shape.n_routed * shape.hidden * (4 if shape.weight_dtype == 0 else 2)
+    hbm = (r["uniq_hits"] + r["uniq_misses"]) * S_e / steps + shape.n_layers * shape.n_shared * \
+        synth.expert_block_bytes(shape, shared=True) + router
+    t_hbm = hbm / (peak_hbm * 1e9)
+    t_h2d = r["h2d_bytes"] / steps / (h2d_peak * 1e9)
+    t_roof = max(t_hbm, t_h2d)
+    return {"t_hbm_ms": t_hbm * 1e3, "t_h2d_ms": t_h2d * 1e3, "t_step_ms": r["ms"] / steps,
+            "frac": t_roof / (r["ms"] / steps / 1e3), "bound": "h2d" if t_h2d > t_hbm else "hbm",
+            "h2d_achieved_gbs": r["h2d_bytes"] / (r["ms"] / 1e3) / 1e9}
+
+
+def summarise(shape, r, steps, peak_hbm, h2d_peak):
+    return {"tokens_per_s": steps * shape.batch / (r["ms"] / 1e3), "ms_per_step": r["ms"] / steps,
+            "hit_rate": r["uniq_hits"] / max(1, r["uniq_hits"] + r["uniq_misses"]),
+            "eor": r["overlap"] / max(1, r["pairs"] * shape.top_k),
+            "misses_per_step": r["uniq_misses"] / steps,
+            "step_roofline": step_roofline(shape, r, steps, peak_hbm, h2d_peak)}
+
+
+def all_resident(torch, wl, stream, shape, seed, rho, steps, warmup, peak_hbm, h2d_peak):
+    """The same stream on a stack with as many slots as experts (no misses once warm): the expert kernel
+    and the whole step against HBM alone."""
+    wl_r = copy.copy(wl)
+    wl_r.stack = wl.new_stack(shape.n_routed, stream.cuda_stream)
+    try:
+        r = run_protocol(torch, wl_r, stream, shape, seed, rho, steps, warmup, 1, False, False,
+                         prewarm_iid=max(192, 3 * shape.n_routed // max(1, shape.top_k * shape.batch)))[0]
+    finally:
+        wl_r.stack.close()
+    ms_r, n_r, b_r = r["kernel_resident"]
+    gbs = b_r / (ms_r / 1e3) / 1e9 if ms_r > 0 else 0.0
+    return {"cache_slots": shape.n_routed, "tokens_per_s": steps * shape.batch / (r["ms"] / 1e3),
+            "ms_per_step": r["ms"] / steps, "misses": r["uniq_misses"], "kernel_gbs": gbs,
+            "kernel_frac_of_measured": gbs / peak_hbm, "kernel_frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS,
+            "step_frac_of_hbm_roofline": step_roofline(shape, r, steps, peak_hbm, h2d_peak)["frac"]}
+
+
+def short_run(torch, name, steps, warmup, peak_hbm, h2d_peak_of, store_of=None, budget_bytes=12e9):
+    """One of the other workloads under the same protocol, one repeat, plus its all-resident run."""
+    from paper_2605_27081_b200.loader import LoadedWorkload
+    cfg = synth.config(name)
+    shape, C, seed = cfg["shape"], cfg["cache_slots"], cfg["seed"]
+    S_e = synth.expert_block_bytes(shape)
+    distinct = None
+    if store_of is None and shape.n_layers * shape.n_routed * S_e > budget_bytes:
+        # bound the pinned store and its generation time: expert ids share this many distinct blocks per
+        # layer (a fetch moves the same bytes whichever block it reads)
+        distinct = max(C + shape.top_k + 1, int(budget_bytes / (shape.n_layers * S_e)))
+    stream = torch.cuda.Stream()
+    wl = LoadedWorkload(shape, C, seed, stream=stream.cuda_stream, distinct_experts=distinct, store_of=store_of)
+    out = {"kernel": kernel_name(shape), "dtype": DTYPE_NAME[shape.weight_dtype], "batch": shape.batch,
+           "cache_slots": C, "steps": steps, "warmup": warmup,
+           "distinct_experts_per_layer": wl.n_distinct, "blocks_aliased": wl.n_distinct < shape.n_routed}
+    try:
+        h2d_peak = h2d_peak_of(S_e)
+        out["h2d_peak_gbs"] = h2d_peak
+        runs = {}
+        for rho in cfg["rhos"]:
+            r = run_protocol(torch, wl, stream, shape, seed, rho, steps, warmup, 1, False, False)[0]
+            runs["per_sequence" if rho is None else str(rho)] = summarise(shape, r, steps, peak_hbm, h2d_peak)
+        out["runs"] = runs
+        rho0 = cfg["rhos"][0]
+        out["all_resident"] = all_resident(torch, wl, stream, shape, seed, rho0, min(steps, 64), warmup, peak_hbm,
+                                           h2d_peak)
+    finally:
+        wl.close()
+    return out
+
+
 def run_ours(args, rank, world, local_rank):
     import torch
     from paper_2605_27081_b200.loader import LoadedWorkload
@@ -308,7 +500,14 @@ def run_ours(args, rank, world, local_rank):
         distinct = max(C + shape.top_k, int(0.6 * avail / world / (shape.n_layers * S_e)))
     stream = torch.cuda.Stream()
     wl = LoadedWorkload(shape, C, seed, stream=stream.cuda_stream, distinct_experts=distinct)
-    h2d_peak = measure_h2d(torch, S_e)
+    h2d_cache = {}
+
+    def h2d_peak_of(nbytes):
+        if nbytes not in h2d_cache:
+            h2d_cache[nbytes] = measure_h2d(torch, nbytes)
+        return h2d_cache[nbytes]
+
+    h2d_peak = h2d_peak_of(S_e)
 
     def barrier():
         torch.cuda.synchronize()
@@ -316,28 +515,23 @@ def run_ours(args, rank, world, local_rank):
             dist.barrier()
         torch.cuda.synchronize()
 
-    rhos = [args.rho] + [r for r in cfg["rhos"] if r != args.rho and not args.no_sweep]
-    results = {}
-    clocks = None
-    for rho in rhos:
-        is_head = rho == args.rho
-        barrier()
-        sampler = ClockSampler(local_rank) if (is_head and rank == 0) else None
-        results[rho] = run_rho(torch, wl, stream, shape, seed, rho, args.steps, args.warmup, with_e2e=is_head)
-        barrier()
-        if sampler is not None:
-            clocks = sampler.stop()
+    # Headline coefficient: `repeats` repeats of cold start, device-input steps and host-buffer steps.
+    barrier()
+    reps = run_protocol(torch, wl, stream, shape, seed, args.rho, args.steps, args.warmup, args.repeats, True,
+                        not args.no_cold, local_rank=local_rank if rank == 0 else None)
+    barrier()
+    head = median_rep(reps)
+    head_e2e = median_rep(reps, "e2e")["e2e"]
+    results = {args.rho: head}
+    for rho in cfg["rhos"]:
+        if rho != args.rho and not args.no_sweep:
+            results[rho] = run_protocol(torch, wl, stream, shape, seed, rho, args.steps, args.warmup, 1, False, False)[0]
+    barrier()
 
-    # All-resident stack (C = N, no misses once warm): the expert-streaming kernel against HBM.
     resident = None
     if not args.no_resident and rank == 0:
-        import copy
-        wl_r = copy.copy(wl)
-        wl_r.stack = wl.new_stack(shape.n_routed, stream.cuda_stream)
-        r = run_rho(torch, wl_r, stream, shape, seed, args.rho, min(args.steps, 256), args.warmup, False,
-                    prewarm_iid=192)
-        resident = r
-        wl_r.stack.close()
+        resident = all_resident(torch, wl, stream, shape, seed, args.rho, min(args.steps, 256), args.warmup, peak_hbm,
+                                h2d_peak)
 
     # The same steps through the multi-step entry point (all inputs known up front: step t+1 is routed
     # while step t is still fetching, so the host link stays busy across step boundaries).
@@ -391,13 +585,13 @@ def run_ours(args, rank, world, local_rank):
             torch.cuda.synchronize()
         c1 = wl.stack.cache_stats()
         ms_c = ea.elapsed_time(eb)
+        h2d_c = c1["h2d_bytes"] - c0["h2d_bytes"]
         chained = {"tokens_per_s": n / (ms_c / 1e3), "ms_per_step": ms_c / n,
                    "misses_per_step": (c1["uniq_misses"] - c0["uniq_misses"]) / n,
-                   "h2d_achieved_gbs": (c1["h2d_bytes"] - c0["h2d_bytes"]) / (ms_c / 1e3) / 1e9}
+                   "h2d_achieved_gbs": h2d_c / (ms_c / 1e3) / 1e9,
+                   "frac_of_h2d_roofline": (h2d_c / (h2d_peak * 1e9)) / (ms_c / 1e3)}
 
-    head = results[args.rho]
-    red = reduce_over_ranks(dist, {"ms": head["ms"], "e2e_ms": head["e2e_ms"]}, {"launches": head["launches"]},
-                            "cuda")
+    red = reduce_over_ranks(dist, {"ms": head["ms"], "e2e_ms": head_e2e["ms"]}, {"launches": head["launches"]}, "cuda")
     ms, e2e_ms, launches = red["ms"], red["e2e_ms"], red["launches"]
     if rank != 0:
         wl.close()
@@ -406,27 +600,15 @@ def run_ours(args, rank, world, local_rank):
         return
     tokens = args.steps * world * shape.batch
     value = tokens / (ms / 1e3)
-    per_step_ms = ms / args.steps
 
-    def step_roofline(r, steps):
-        # bytes one step must move: resident experts + shared + router from HBM, misses over the host link
-        router = shape.n_layers * shape.n_routed * shape.hidden * shape.elem_bytes
-        hbm = (r["uniq_hits"] + r["uniq_misses"]) * S_e / steps + shape.n_layers * shape.n_shared * \
-            synth.expert_block_bytes(shape, shared=True) + router
-        t_hbm = hbm / (peak_hbm * 1e9)
-        t_h2d = r["h2d_bytes"] / steps / (h2d_peak * 1e9)
-        t_roof = max(t_hbm, t_h2d)
-        return {"t_hbm_ms": t_hbm * 1e3, "t_h2d_ms": t_h2d * 1e3, "t_step_ms": r["ms"] / steps,
-                "frac": t_roof / (r["ms"] / steps / 1e3), "bound": "h2d" if t_h2d > t_hbm else "hbm",
-                "h2d_achieved_gbs": r["h2d_bytes"] / (r["ms"] / 1e3) / 1e9}
-
+    kname = kernel_name(shape)
     kr_ms, kr_n, kr_b = head["kernel_resident"]
     km_ms, km_n, km_b = head["kernel_miss"]
     ach = kr_b / (kr_ms / 1e3) / 1e9 if kr_ms > 0 else 0.0
+    ratio = None if args.layers else TRAFFIC_RATIO.get((args.workload, kname))
     roofline = {"bound": "hbm", "achieved": ach, "peak": peak_hbm, "unit": "GB/s", "frac": ach / peak_hbm,
-                "traffic": (kr_b / max(1, kr_n) * TRAFFIC_RATIO[(args.workload, shape.weight_dtype)]
-                            if TRAFFIC_RATIO.get((args.workload, shape.weight_dtype)) and not args.layers else None),
-                "peak_kind": f"of {peak_kind}", "kernel": kernel_name(shape) + " resident phase",
+                "traffic": kr_b / max(1, kr_n) * ratio if ratio else None,
+                "peak_kind": f"of {peak_kind}", "kernel": kname + " resident phase",
                 "launches": kr_n, "avg_launch_ms": kr_ms / max(1, kr_n), "bytes_per_launch": kr_b / max(1, kr_n),
                 "frac_of_nominal_8TBs": ach / NOMINAL_HBM_GBS}
     miss_phase = {"launches": km_n, "avg_launch_us": km_ms * 1e3 / max(1, km_n),
@@ -435,36 +617,32 @@ def run_ours(args, rank, world, local_rank):
     # CPU baseline: the oracle on a bounded sample, rank 0 only.
     cpu = None
     if not args.no_cpu_baseline and world == 1:
-        layers, steps_cpu = 2, 3
-        dt, cores = oracle_sample(shape, C, seed, args.rho, layers, steps_cpu)
-        per = dt / steps_cpu * shape.n_layers / layers
-        cpu = {"value": shape.batch / per, "unit": "tokens/s", "cores": cores, "kind": "oracle",
-               "sample": f"first {steps_cpu} decode steps (cold cache) over the first {layers} of {shape.n_layers} "
-                         f"layers, time scaled by {shape.n_layers}/{layers}; selected-experts-only fp64 oracle"}
+        cpu = cpu_baseline_legs(shape, C, seed, args.rho, wl.expert_block)
 
-    sweep = {}
-    for rho, r in results.items():
-        sweep[str(rho)] = {
-            "tokens_per_s": args.steps * shape.batch / (r["ms"] / 1e3),
-            "hit_rate": r["uniq_hits"] / max(1, r["uniq_hits"] + r["uniq_misses"]),
-            "eor": r["overlap"] / max(1, r["pairs"] * shape.top_k),
-            "misses_per_step": r["uniq_misses"] / args.steps,
-            "step_roofline": step_roofline(r, args.steps)}
+    sweep = {str(rho): summarise(shape, r, args.steps, peak_hbm, h2d_peak) for rho, r in results.items()}
+    all_ms = sorted(r["ms"] for r in reps)
+    all_e2e = sorted(r["e2e"]["ms"] for r in reps)
     line = {
-        "metric": "decode tokens/s (batch 1, MoE stack)", "value": value, "unit": "tokens/s",
-        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_step_ms,
+        "metric": metric_name(shape), "value": value, "unit": "tokens/s",
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": DTYPE_NAME[shape.weight_dtype], "data": "synthetic",
         "config": {"workload": args.workload, "rho": args.rho, "cache_slots": C, "batch": shape.batch,
                    "layers": shape.n_layers,
                    "l2": "inputs larger than L2 (>= 1.6 GB of expert weights streamed per step)",
                    "parallelism": "replicas only" if world > 1 else "single GPU",
                    "distinct_experts_per_layer": wl.n_distinct},
-        "clocks": clocks,
+        "repeats": {"n": len(reps), "reported": "median repeat",
+                    "tokens_per_s_min_med_max": [args.steps * shape.batch / (m / 1e3) for m in (all_ms[-1], all_ms[len(all_ms) // 2], all_ms[0])],
+                    "e2e_tokens_per_s_min_med_max": [args.steps * shape.batch / (m / 1e3) for m in (all_e2e[-1], all_e2e[len(all_e2e) // 2], all_e2e[0])],
+                    "note": "every repeat: cold cache, the same warm-up steps, the same timed steps (identical miss sequence)"},
+        "clocks": merge_clocks([r.get("clocks") for r in reps]),
         "e2e": {"value": tokens / (e2e_ms / 1e3), "unit": "tokens/s",
-                "h2d_bytes_per_step": head["e2e_in_bytes"] + head["h2d_bytes"] / args.steps,
-                "d2h_bytes_per_step": head["e2e_out_bytes"],
-                "note": "remoe_decode_step_host: hidden states from pinned host memory, outputs read back; "
-                        "h2d bytes include the expert fetches"},
+                "h2d_bytes_per_step": head_e2e["in_bytes"] + head_e2e["h2d_bytes"] / args.steps,
+                "d2h_bytes_per_step": head_e2e["out_bytes"],
+                "misses_per_step": head_e2e["uniq_misses"] / args.steps,
+                "note": "remoe_decode_step_host on the same steps as `value` (same cold start, warm-up and hidden "
+                        "states): hidden states from pinned host memory, outputs read back every step; h2d bytes "
+                        "include this leg's own expert fetches"},
         "gpu_launches": int(launches),
         "roofline": roofline,
         "roofline_miss_phase": miss_phase,
@@ -474,19 +652,30 @@ def run_ours(args, rank, world, local_rank):
         "sweep": sweep,
         "cpu_baseline": cpu,
     }
+    if "cold" in head:
+        c = head["cold"]
+        line["cold_start"] = dict(summarise(shape, c, c["steps"], peak_hbm, h2d_peak), steps=c["steps"],
+                                  note="steps 1..%d from an empty cache (request-isolated start), kernels warm" % c["steps"])
     if resident is not None:
-        n = min(args.steps, 256)
-        ms_r, n_r, b_r = resident["kernel_resident"]
-        line["all_resident"] = {
-            "cache_slots": shape.n_routed, "tokens_per_s": n * shape.batch / (resident["ms"] / 1e3),
-            "ms_per_step": resident["ms"] / n, "misses": resident["uniq_misses"],
-            "kernel_gbs": b_r / (ms_r / 1e3) / 1e9 if ms_r > 0 else 0.0,
-            "kernel_frac_of_measured": (b_r / (ms_r / 1e3) / 1e9 / peak_hbm) if ms_r > 0 else 0.0,
-            "step_frac_of_hbm_roofline": step_roofline(resident, n)["frac"]}
+        line["all_resident"] = resident
     if multi is not None:
         line["multi_step"] = multi
     if chained is not None:
         line["chained"] = chained
+    wl_keep = wl
+    if not args.no_others and world == 1 and not args.layers and args.workload == WORKLOAD:
+        others = {}
+        n_o, w_o = min(args.steps, 24), min(max(args.warmup, 8), 16)
+        for name in ("tiny_fp32", "qwen15moe", "qwen3_30b", "dsv2lite_b32", "dsv2lite_fp8", "dsv2lite_int4",
+                     "dsv2lite_b32_fp8"):
+            if name not in synth.CONFIGS:
+                continue
+            try:
+                others[name] = short_run(torch, name, n_o, w_o, peak_hbm, h2d_peak_of,
+                                         store_of=wl_keep if name == "dsv2lite_b32" and wl_keep.n_distinct == shape.n_routed else None)
+            except Exception as ex:              # a workload that cannot run here must not lose the line
+                others[name] = {"error": f"{type(ex).__name__}: {ex}"}
+        line["other_workloads"] = others
     print(json.dumps(line), flush=True)
     wl.close()
     if dist is not None:
@@ -498,6 +687,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=256)
     ap.add_argument("--warmup", type=int, default=16)
+    ap.add_argument("--repeats", type=int, default=3, help="repeats of the headline protocol (median reported)")
     ap.add_argument("--rho", type=float, default=None, help="AR(1) coefficient of the headline run (default 0.9)")
     ap.add_argument("--workload", default=WORKLOAD, choices=sorted(synth.CONFIGS),
                     help="default: the DeepSeek-V2-Lite-shaped batch-1 stack the metric is quoted on")
@@ -507,10 +697,13 @@ def main():
     ap.add_argument("--no-resident", action="store_true")
     ap.add_argument("--no-chained", action="store_true")
     ap.add_argument("--no-multi", action="store_true")
+    ap.add_argument("--no-cold", action="store_true")
+    ap.add_argument("--no-others", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
+    args.repeats = max(1, args.repeats)
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))

@@ -14,6 +14,15 @@
  *   - "dev" pointers are CUDA device pointers owned by the caller; "host" pointers are host
  *     memory owned by the caller.  The handle is owned by the library.
  *   - All tensors are dense, row-major, layer-major: [L, B, ...].
+ *   - Device-side errors.  Kernels never trap: a bounded wait that runs out or an index out of range
+ *     sets an error word and the kernel returns.  The routing kernel's errors are seen by the decode
+ *     call itself; an expert or combine kernel runs after the call has returned, so its error is
+ *     reported as REMOE_E_DEVICE_FLAG by the NEXT call on the stack that synchronises: a decode call,
+ *     remoe_decode_step_host (which reports its own step), remoe_last_step_trace or one of the
+ *     statistics calls.  The outputs of that step are then finite but incomplete.
+ *   - After REMOE_E_DEVICE_FLAG or REMOE_E_CUDA from a decode call the cache directory may already hold
+ *     the step's admissions while their slots were never filled: call remoe_cache_reset() before the
+ *     next step (it also clears the error word).  Nothing else needs to be rebuilt.
  *   - One stack belongs to one device (the one current at creation) and one stream.  A call
  *     may be made with any device current: the library switches to the stack's device for
  *     the call and restores the caller's.  Calls on one stack must not overlap in time.
@@ -85,6 +94,11 @@ typedef struct remoe_stack remoe_stack;
  * `cuda_stream` is the cudaStream_t all kernels are ordered on (NULL = default stream); the
  * library also owns one copy stream.  Allocates the slot pools, directory and scratch on
  * the current device.  Errors: ARG, CAPACITY (B == 1 and C < K), UNSUPPORTED, NOMEM, CUDA.
+ * Environment read here: REMOE_BATCHED_KERNEL=mma keeps a batched stack on the mma.sync expert kernel;
+ * REMOE_FAULT_INJECT=lost_copy (failure-detection tests, batch 1) makes the first step's resident-phase
+ * expert launch run with a short wait limit and never issue the copy of its first weight row: the
+ * consumer's bounded wait runs out, the kernel sets the error word and returns, and the error surfaces as
+ * described under "Device-side errors" above.  Later launches of the stack are normal.
  */
 int remoe_stack_create(const remoe_shape* shape, int32_t cache_slots_per_layer,
                        void* cuda_stream, remoe_stack** out);
@@ -101,8 +115,8 @@ int remoe_load_shared(remoe_stack*, int32_t layer, int32_t idx, const void* bloc
 /* Register the host copies of routed experts first_expert .. first_expert+count-1 of
  * `layer`: `pinned_ptrs[i]` points at one expert block in page-locked host memory, 16-byte
  * aligned.  BORROWED: the caller keeps the memory pinned, alive and unchanged until the
- * stack is destroyed; misses are fetched from it (Sec. 3.1: "misses trigger expert
- * fetches").  Several experts may share one pointer.  Errors: ARG, NOT_PINNED. */
+ * stack is destroyed; misses are fetched from it (the cache model of Sec. 3.1).
+ * Several experts may share one pointer.  Errors: ARG, NOT_PINNED. */
 int remoe_load_experts_host(remoe_stack*, int32_t layer, int32_t first_expert, int32_t count,
                             const void* const* pinned_ptrs);
 
@@ -138,7 +152,8 @@ int remoe_decode_step(remoe_stack*, const float* hidden_in_dev, float* hidden_ou
  * on an internal stream while step t is still fetching, and its miss list reaches the host before the copy
  * engine runs out of work.  The host link, which bounds the step at realistic cache sizes, then stays
  * busy across step boundaries (a single call per step leaves it idle for the time of the last expert
- * launch, the combine, the next routing and the host hand-off: about 1 % of a step at config-2 sizes).
+ * launch, the combine, the next routing and the host hand-off: about 1 % of a step for a 26-layer stack
+ * of 17 MB experts at 28 misses per step).
  * Inputs must be complete when the stack's stream reaches the call; outputs are complete when that
  * stream has drained.  The host blocks until the last step's miss list is known.  The first call
  * allocates a second set of small per-step buffers.  Errors: ARG, NOT_LOADED, UNSUPPORTED (batch > 1),
@@ -178,7 +193,8 @@ int remoe_last_step_trace(remoe_stack*, int32_t* requests, int32_t* hit, int32_t
                           int32_t* evicted, int32_t* n_unique);
 
 /* Counters for one layer, or summed over layers with layer = -1 (App. E.2.4: #uMiss, uHR =
- * uniq_hits / (uniq_hits + uniq_misses), tHR likewise).  Waits for the stack's stream. */
+ * uniq_hits / (uniq_hits + uniq_misses), tHR likewise).  Waits for the stack's stream; like the
+ * other statistics calls it fills its outputs and returns DEVICE_FLAG if a kernel has set the error word. */
 int remoe_cache_stats(remoe_stack*, int32_t layer, remoe_cache_counters* out);
 
 /* Reuse statistic (Eq. 1): overlap_sum = sum over counted (step, sequence) pairs of

@@ -2,9 +2,10 @@
 // statistics, and the extern "C" boundary declared in remoe.h.
 //
 // Per decode step (batch 1):
-//   compute stream : route+resolve kernel -> copy of the step trace to pinned host memory
+//   compute stream : route+resolve kernel (its resolve warps also write the step trace to a mirror in
+//                    mapped page-locked host memory)
 //                    -> resident-phase streaming kernel (hits + shared experts, all layers)
-//   host           : waits only for the trace, then walks it: for each layer, one
+//   host           : waits only for the route kernel, then walks the mirrored trace: for each layer, one
 //                    cudaMemcpyAsync per missing expert from its pinned host block into the
 //                    victim slot on the copy stream, an event after the layer's last copy
 //   compute stream : per layer with misses: wait for that event, miss-phase streaming kernel
@@ -91,6 +92,9 @@ struct remoe_stack {
   uint64_t prof_launches[2] = {0, 0}, prof_bytes[2] = {0, 0};
   uint64_t kernel_launches = 0;          // every kernel this stack has launched
   std::string cuda_err;
+  // failure-detection test aid (REMOE_FAULT_INJECT=lost_copy at creation): the first resident-phase launch
+  // of the batch-1 step runs with a short wait limit and one weight row whose copy is never issued
+  bool inject_lost_copy = false;
   int policy = REMOE_POLICY_LRU;
   float beta = 0.f;
 };
@@ -238,6 +242,16 @@ int check_device_flag(remoe_stack* s, const int* block = nullptr) {
   const int c = block[0];
   s->cuda_err = std::string("device flag ") + std::to_string(c) + ": " + (c >= 1 && c <= 4 ? names[c] : "unknown");
   return REMOE_E_DEVICE_FLAG;
+}
+
+// With the stack's stream drained: the device error word, which the expert and combine kernels of the
+// last step may have set after the route kernel mirrored it to the host.
+int fetch_device_flag(remoe_stack* s) {
+  int e = kErrNone;
+  CK(cudaMemcpy(&e, s->dev_block, sizeof(int), cudaMemcpyDeviceToHost));
+  if (e == kErrNone) return REMOE_OK;
+  s->host_block[0] = e;
+  return check_device_flag(s);
 }
 
 // One decode step for B > 1.  The step's distinct requests may outnumber the slots, so a slot
@@ -558,6 +572,8 @@ int remoe_stack_create(const remoe_shape* sh, int32_t cache_slots, void* cuda_st
   for (auto& e : s->ev_layer)
     if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return bail(REMOE_E_CUDA);
 
+  if (const char* inj = std::getenv("REMOE_FAULT_INJECT"))
+    s->inject_lost_copy = std::strcmp(inj, "lost_copy") == 0 && sh->batch == 1;
   DevStack& d = s->d;
   d.L = sh->n_layers; d.H = sh->hidden; d.N = sh->n_routed; d.K = sh->top_k; d.I = sh->inter_routed;
   d.S = sh->n_shared; d.Is = sh->n_shared ? sh->inter_shared : 0; d.B = sh->batch; d.C = cache_slots;
@@ -725,7 +741,14 @@ int remoe_decode_step(remoe_stack* s, const float* hin, float* hout, int32_t* id
   // The resident phase needs no host decision: enqueue it before waiting for the trace.
   int rc = prof_begin(s, s->stream, 0, 0);
   if (rc != REMOE_OK) return rc;
+  if (s->inject_lost_copy) {
+    a.lose_row1 = 1;                 // the launch's first weight row never arrives
+    a.spin_limit = 1u << 12;         // so that the wait for it gives up quickly
+    s->inject_lost_copy = false;
+  }
   CK(launch_ffn_stream(a, s->grid, s->stream));
+  a.lose_row1 = 0;
+  a.spin_limit = 0;
   s->kernel_launches += 1;
   rc = prof_end(s, s->stream);
   if (rc != REMOE_OK) return rc;
@@ -1048,6 +1071,8 @@ int remoe_decode_step_host(remoe_stack* s, const float* hin, float* hout, int32_
   CK(cudaMemcpyAsync(s->st_ids_h, s->st_ids_d, kk * sizeof(int), cudaMemcpyDeviceToHost, s->stream));
   CK(cudaMemcpyAsync(s->st_g_h, s->st_g_d, kk * sizeof(float), cudaMemcpyDeviceToHost, s->stream));
   CK(cudaStreamSynchronize(s->stream));
+  rc = fetch_device_flag(s);                   // an expert kernel of this very step may have given up
+  if (rc != REMOE_OK) return rc;
   std::memcpy(hout, s->st_out_h, io * sizeof(float));
   std::memcpy(ids, s->st_ids_h, kk * sizeof(int));
   std::memcpy(gates, s->st_g_h, kk * sizeof(float));
@@ -1086,7 +1111,7 @@ int remoe_cache_stats(remoe_stack* s, int32_t layer, remoe_cache_counters* out) 
     out->h2d_bytes += s->h2d_bytes[l];
   }
   out->steps = s->steps;
-  return REMOE_OK;
+  return fetch_device_flag(s);
 }
 
 int remoe_reuse_stats(remoe_stack* s, int32_t layer, uint64_t* overlap_sum, uint64_t* pairs, float* last_ir) {
@@ -1114,7 +1139,7 @@ int remoe_reuse_stats(remoe_stack* s, int32_t layer, uint64_t* overlap_sum, uint
         last_ir[j++] = v < 0 ? -1.f : (float)v / (float)s->d.K;
       }
   }
-  return REMOE_OK;
+  return fetch_device_flag(s);
 }
 
 int remoe_reuse_mass(remoe_stack* s, int32_t layer, double* mass_sum, uint64_t* pairs, float* last_mass) {
@@ -1141,7 +1166,7 @@ int remoe_reuse_mass(remoe_stack* s, int32_t layer, double* mass_sum, uint64_t* 
   }
   if (mass_sum) *mass_sum = tot;
   if (pairs) *pairs = p;
-  return REMOE_OK;
+  return fetch_device_flag(s);
 }
 
 int remoe_expert_load(remoe_stack* s, int32_t layer, uint64_t* counts, double* entropy, double* cv,
@@ -1174,7 +1199,7 @@ int remoe_expert_load(remoe_stack* s, int32_t layer, uint64_t* counts, double* e
   if (entropy) *entropy = ent_sum / nl;
   if (cv) *cv = cv_sum / nl;
   if (visited) *visited = (int32_t)(seen_sum / nl);
-  return REMOE_OK;
+  return fetch_device_flag(s);
 }
 
 int remoe_step_history(remoe_stack* s, int32_t first, int32_t count, uint32_t* umiss, uint32_t* tok_hits,

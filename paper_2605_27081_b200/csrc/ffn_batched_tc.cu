@@ -2,7 +2,7 @@
 //
 // Same work list as ffn_batched.cu, with a work item of (layer, expert, tile of up to 16 tokens)
 // and channel blocks of 64.  Per CTA (one per SM, 192 threads):
-//   warp 4   TMA producer: one bulk copy (cp.async.bulk, no multicast) per 16 KB operand tile into a
+//   warp 4   TMA producer: one bulk copy (cp.async.bulk, per CTA) per 16 KB operand tile into a
 //            shared-memory ring.  Slots and shared blocks of such a stack are kept in OPERAND-TILE
 //            ORDER: per 64-channel group the H/64 A1 tiles, then the H/128 A2 tiles, each stored as
 //            the 128-byte-swizzled image the tensor cores read, so a tile is one contiguous 16 KB run

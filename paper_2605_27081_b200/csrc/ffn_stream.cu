@@ -91,6 +91,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(const __grid_co
   const DevStack& d = a.d;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int P = d.K + d.S, n_pairs = d.L * P;
+  const unsigned spin = a.spin_limit ? a.spin_limit : kSpinLimit;
 
   // Work table: exclusive prefix of rows per pair.
   for (int i = tid; i < n_pairs; i += kThreads) prefix[i + 1] = pair_rows(a, i);
@@ -162,20 +163,21 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(const __grid_co
         const int n = r - r0, s = n % NS;
         if (n >= NS) {
           if (*(volatile int*)&s_abort) { ok = false; break; }
-          if (!mbar_wait(empty + s, ((n / NS) - 1) & 1)) {
+          if (!mbar_wait(empty + s, ((n / NS) - 1) & 1, spin)) {
             atomicCAS(d.err, kErrNone, kErrWaitEmpty);
             ok = false;
             break;
           }
         }
+        if (r + 1 == a.lose_row1) continue;                // test aid: this stage is never filled
         mbar_expect_tx(full + s, kStageBytes);
         bulk_g2s(stages + (size_t)s * kStageBytes, base + (size_t)i * kStageBytes, kStageBytes, full + s);
       }
-      if (!ok) {
+      if (!ok || *(volatile int*)&s_abort) {
         // Let the consumers leave, then wait (bounded) for copies that are still landing.
         atomicExch(&s_abort, 1);
         for (int n = issued - kProducerLanes; n >= 0 && n >= issued - NS; n -= kProducerLanes)
-          if (!mbar_wait(full + (n % NS), (n / NS) & 1)) atomicCAS(d.err, kErrNone, kErrDrain);
+          if (!mbar_wait(full + (n % NS), (n / NS) & 1, spin)) atomicCAS(d.err, kErrNone, kErrDrain);
       }
     }
   } else {
@@ -220,7 +222,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(const __grid_co
         }
         const int n = r - r0, s = n % NS;
         // decided for the whole warp: the shuffles below need every lane
-        if (__any_sync(kFull, *(volatile int*)&s_abort || !mbar_wait(full + s, (n / NS) & 1))) {
+        if (__any_sync(kFull, *(volatile int*)&s_abort || !mbar_wait(full + s, (n / NS) & 1, spin))) {
           if (!*(volatile int*)&s_abort) { atomicCAS(d.err, kErrNone, kErrWaitFull); atomicExch(&s_abort, 1); }
           aborted = true;
           break;

@@ -90,6 +90,9 @@ struct FfnArgs {
   float* partial;                      // [2][L][grid][H]
   int* contrib;                        // [2][L][2]  (first CTA, last CTA) contributing; first > last = none
   int grid_cap;                        // CTAs per phase the partial buffer is laid out for
+  unsigned spin_limit;                 // polls of one bounded wait (0 = the default limit)
+  int lose_row1;                       // failure-detection test aid: the copy of row (lose_row1 - 1) of the launch's
+                                       // row list is never issued, so its consumer's bounded wait runs out; 0 = none
 };
 
 // Batched (B > 1) expert kernels: tensor-core grouped GEMM over per-expert token groups.

@@ -1,5 +1,5 @@
 // Device helpers shared by the expert-streaming kernels: mbarrier primitives with bounded waits,
-// the bulk asynchronous global->shared copy (TMA, non-tensor form, no multicast) and the decoding
+// the bulk asynchronous global->shared copy (TMA, non-tensor form, one CTA's own shared memory) and the decoding
 // of 16-byte groups of stored weights to float.
 #pragma once
 
@@ -42,8 +42,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // Bounded wait: false if the phase did not complete within the spin limit.  A parity wait cannot
 // tell "phase k done" from "phase k-2 done", so a waiter must never be a whole phase ahead of the
 // barrier: every kernel here lets a stage be consumed by the same agent every time.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
-  for (unsigned it = 0; it < kSpinLimit; ++it)
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsigned limit = kSpinLimit) {
+  for (unsigned it = 0; it < limit; ++it)
     if (mbar_try_wait(bar, parity)) return true;
   return false;
 }

@@ -189,6 +189,49 @@ def test_non_finite_input_is_reported_not_faulted():
         wl.close()
 
 
+@pytest.mark.parametrize("host_api", [False, True])
+def test_wait_that_runs_out_is_reported_and_reset_restores_service(monkeypatch, host_api):
+    """Failure detection without a fault: a stack created with REMOE_FAULT_INJECT=lost_copy runs its
+    first resident-phase expert launch with a short wait limit and never issues the copy of that launch's
+    first weight row.  The consumer's bounded wait runs out, the kernel records the error and returns (no
+    trap, no hang, the context stays usable).  The step through host buffers reports its own failure;
+    the step on device buffers has already returned when the kernel runs, so the next synchronising call
+    reports it.  A reset clears the condition and the stack then matches the oracle step for step."""
+    import torch
+    from paper_2605_27081_b200 import binding as B
+    from paper_2605_27081_b200.loader import LoadedWorkload
+    from parity_util import StepChecker, oracle_for
+
+    shape = synth.Shape(2, 256, 16, 2, 24, 1, 40, 0, 0, 1, 1)        # a shared expert: step 1 has resident rows
+    monkeypatch.setenv("REMOE_FAULT_INJECT", "lost_copy")
+    wl = LoadedWorkload(shape, 4, seed=21)
+    monkeypatch.delenv("REMOE_FAULT_INJECT")
+    try:
+        hs = synth.HiddenStream(21, shape, 0.5).take(8)
+        x = torch.from_numpy(hs[0]).to("cuda")
+        out = torch.empty_like(x)
+        ids = torch.zeros((2, 1, 2), dtype=torch.int32, device="cuda")
+        g = torch.zeros((2, 1, 2), device="cuda")
+        if host_api:
+            o_h, i_h, g_h = np.empty((2, 1, 256), np.float32), np.empty((2, 1, 2), np.int32), np.empty((2, 1, 2), np.float32)
+            assert B.remoe_decode_step_host(wl.stack.h, hs[0], o_h, i_h, g_h) == B.REMOE_E_DEVICE_FLAG
+        else:
+            assert B.remoe_decode_step(wl.stack.h, x, out, ids, g) == B.REMOE_OK
+            torch.cuda.synchronize()                                  # the kernel has returned by itself
+            rc, _ = B.remoe_cache_stats(wl.stack.h, -1)
+            assert rc == B.REMOE_E_DEVICE_FLAG
+            assert B.remoe_decode_step(wl.stack.h, x, out, ids, g) == B.REMOE_E_DEVICE_FLAG
+        assert "bounded wait" in B.remoe_last_cuda_error(wl.stack.h)
+        torch.cuda.synchronize()
+        wl.stack.cache_reset()
+        chk = StepChecker(wl, oracle_for(wl), torch)
+        for t in range(8):
+            chk.step(hs[t], host_api=(t % 2 == 1))
+        chk.check_counters()
+    finally:
+        wl.close()
+
+
 def test_policy_switch_and_second_stack_share_a_store():
     """Two stacks over the same pinned store (different capacity and policy) stay independent."""
     import torch
