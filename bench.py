@@ -403,10 +403,12 @@ def reduce_over_ranks(dist, maxima: dict, sums: dict, device):
 
 def step_roofline(shape, r, steps, peak_hbm, h2d_peak):
     """bytes one step must move: resident experts + shared + router from HBM, misses over the host link"""
-    S_e = synth.expert_block_bytes(shape)
+    # a batched stack over an FP8 store keeps bf16 blocks on the device (widened on arrival)
+    dev_elem = 2 if (shape.weight_dtype == 2 and shape.batch > 1) else shape.elem_bytes
+    S_dev = synth.expert_block_elems(shape.hidden, shape.inter_routed) * dev_elem
+    S_sh = synth.expert_block_elems(shape.hidden, shape.inter_shared) * dev_elem
     router = shape.n_layers * shape.n_routed * shape.hidden * (4 if shape.weight_dtype == 0 else 2)
-    hbm = (r["uniq_hits"] + r["uniq_misses"]) * S_e / steps + shape.n_layers * shape.n_shared * \
-        synth.expert_block_bytes(shape, shared=True) + router
+    hbm = (r["uniq_hits"] + r["uniq_misses"]) * S_dev / steps + shape.n_layers * shape.n_shared * S_sh + router
     t_hbm = hbm / (peak_hbm * 1e9)
     t_h2d = r["h2d_bytes"] / steps / (h2d_peak * 1e9)
     t_roof = max(t_hbm, t_h2d)
@@ -498,6 +500,8 @@ def run_ours(args, rank, world, local_rank):
     distinct = None
     if world * full > 0.6 * avail:
         distinct = max(C + shape.top_k, int(0.6 * avail / world / (shape.n_layers * S_e)))
+    if args.distinct:
+        distinct = args.distinct
     stream = torch.cuda.Stream()
     wl = LoadedWorkload(shape, C, seed, stream=stream.cuda_stream, distinct_experts=distinct)
     h2d_cache = {}
@@ -693,6 +697,8 @@ def main():
                     help="default: the DeepSeek-V2-Lite-shaped batch-1 stack the metric is quoted on")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layers", type=int, default=0, help="use only this many layers (profiling captures)")
+    ap.add_argument("--distinct", type=int, default=0,
+                    help="let expert ids share this many distinct host blocks per layer (quick experiments)")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-resident", action="store_true")
     ap.add_argument("--no-chained", action="store_true")

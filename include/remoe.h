@@ -56,7 +56,7 @@ enum {
   REMOE_E_NOMEM = -8         /* host or device allocation failed                          */
 };
 
-enum { REMOE_F32 = 0, REMOE_BF16 = 1, REMOE_FP8_E4M3 = 2 };
+enum { REMOE_F32 = 0, REMOE_BF16 = 1, REMOE_FP8_E4M3 = 2, REMOE_INT4_G32 = 3 };
 enum { REMOE_POLICY_LRU = 0, REMOE_POLICY_FIFO = 1, REMOE_POLICY_LFU = 2 };
 
 /* Shape of the stack.  Sec. 3.1: N_r routed experts, Top-K; shared experts always active. */
@@ -72,9 +72,18 @@ typedef struct {
   int32_t renorm_topk;   /* 1: top-K gate weights are renormalised to sum to 1             */
   int32_t weight_dtype;  /* REMOE_F32, REMOE_BF16 (router, shared gate, all experts) or    */
                          /* REMOE_FP8_E4M3: expert blocks are OCP FP8 E4M3 bytes, value =  */
-                         /* byte * 2^-8; router and shared gate bf16; H multiple of 512;   */
-                         /* batch 1 only (halves the bytes a miss moves over the host link)*/
-  int32_t batch;         /* B sequences per step; B > 1 needs bf16 weights and I, I_shared  */
+                         /* byte * 2^-8; router and shared gate bf16; H multiple of 512.   */
+                         /* Halves the bytes a miss moves over the host link.  At batch 1  */
+                         /* the slots hold the FP8 bytes; at batch > 1 (I, I_shared        */
+                         /* multiples of 64) a fetched block is widened, exactly, to bf16  */
+                         /* operand tiles on arrival and the grouped GEMM is the bf16 one. */
+                         /* REMOE_INT4_G32 (batch 1; H 1024 or 2048): 4-bit codes in groups*/
+                         /* of 32 consecutive elements of a row, value = (code - 8) * the  */
+                         /* group's bf16 scale; a stored row is H/2 bytes of codes (element*/
+                         /* 2i in the low half of byte i) then H/32 scales, so a row takes */
+                         /* 0.5625 H bytes: 3.6x fewer bytes per miss than bf16.  Router   */
+                         /* and shared gate bf16.                                          */
+  int32_t batch;         /* B sequences per step; B > 1 needs bf16 or FP8 weights and I, I_shared */
                          /* multiples of 8, B * K <= 1024                                   */
 } remoe_shape;
 

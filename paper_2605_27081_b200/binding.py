@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_PKG, "libremoe.so")
 REMOE_OK = 0
 REMOE_E_ARG, REMOE_E_CAPACITY, REMOE_E_NOT_LOADED, REMOE_E_NOT_PINNED = -1, -2, -3, -4
 REMOE_E_CUDA, REMOE_E_DEVICE_FLAG, REMOE_E_UNSUPPORTED, REMOE_E_NOMEM = -5, -6, -7, -8
-REMOE_F32, REMOE_BF16, REMOE_FP8_E4M3 = 0, 1, 2
+REMOE_F32, REMOE_BF16, REMOE_FP8_E4M3, REMOE_INT4_G32 = 0, 1, 2, 3
 REMOE_POLICY_LRU, REMOE_POLICY_FIFO, REMOE_POLICY_LFU = 0, 1, 2
 
 EXPORTS = [

@@ -70,6 +70,8 @@ struct remoe_stack {
   int step_serial = 0;                    // never reset: stamps partial rows
   cudaEvent_t ev_resident = nullptr;
   bool use_tc = false;                     // batched experts on tcgen05 / TMEM, slots in operand-tile order
+  bool widen_fp8 = false;                  // batched stack over an FP8 host store: blocks are widened to bf16 on arrival
+  size_t fetch_bytes = 0, fetch_shared_bytes = 0;   // bytes of one routed / shared expert block in HOST memory
   char* stage_pool = nullptr;              // [2][C] channel-major landing area of fetched blocks (use_tc)
   size_t stage_bytes = 0;
   cudaEvent_t ev_stage[2] = {nullptr, nullptr};   // retile of the group that last used a half is enqueued
@@ -310,6 +312,7 @@ int batched_waves(remoe_stack* s, BatchArgs& a, int l0, int l1, uint64_t* reside
   if (max_depth >= 0 && !staged) CK(cudaStreamWaitEvent(s->copy_stream, s->ev_trace, 0));
   std::vector<size_t> src_off;
   std::vector<char*> dst_ptr;
+  std::vector<const void*> src_ptr;
   for (int dep = 0; dep <= max_depth; ++dep) {
     if (dep == 1 && !staged) CK(cudaStreamWaitEvent(s->copy_stream, s->ev_resident, 0));   // displaced hits are done
     for (int l = l0; l < l1; ++l) {
@@ -330,24 +333,30 @@ int batched_waves(remoe_stack* s, BatchArgs& a, int l0, int l1, uint64_t* reside
             if (s->stage_used[half]) CK(cudaStreamWaitEvent(s->copy_stream, s->ev_stage[half], 0));
           }
           if (misses >= d.C) return REMOE_E_DEVICE_FLAG;         // more misses of one depth than slots: bad trace
-          src_off.push_back(((size_t)half * d.C + misses) * d.slot_bytes);
+          src_off.push_back(((size_t)half * d.C + misses) * s->fetch_bytes);
           dst_ptr.push_back(slot);
           land = s->stage_pool + src_off.back();
         } else if (!misses && dep >= 1 && had[(size_t)(dep - 1) * d.L + l]) {
           CK(cudaStreamWaitEvent(s->copy_stream, ev_comp(dep - 1, l), 0));        // displaced misses are done
         }
-        CK(cudaMemcpyAsync(land, s->host_ptrs[(size_t)l * d.N + t_req[j]], d.slot_bytes, cudaMemcpyHostToDevice,
+        CK(cudaMemcpyAsync(land, s->host_ptrs[(size_t)l * d.N + t_req[j]], s->fetch_bytes, cudaMemcpyHostToDevice,
                            s->copy_stream));
         ++misses;
       }
       if (!misses) continue;
       had[(size_t)dep * d.L + l] = 1;
-      s->h2d_bytes[l] += (uint64_t)misses * d.slot_bytes;
+      s->h2d_bytes[l] += (uint64_t)misses * s->fetch_bytes;
       CK(cudaEventRecord(ev_copy(dep, l), s->copy_stream));
 
       CK(cudaStreamWaitEvent(s->stream, ev_copy(dep, l), 0));
       if (staged) {
-        CK(launch_retile_tc(d, s->tc_maps, misses, src_off.data(), dst_ptr.data(), d.I, s->stream));
+        if (s->widen_fp8) {
+          src_ptr.clear();
+          for (size_t off : src_off) src_ptr.push_back(s->stage_pool + off);
+          CK(launch_widen_retile_tc(d, misses, src_ptr.data(), dst_ptr.data(), d.I, s->stream));
+        } else {
+          CK(launch_retile_tc(d, s->tc_maps, misses, src_off.data(), dst_ptr.data(), d.I, s->stream));
+        }
         s->kernel_launches += (misses + 63) / 64;
         CK(cudaEventRecord(s->ev_stage[half], s->stream));
         s->stage_used[half] = true;
@@ -539,11 +548,18 @@ int remoe_stack_create(const remoe_shape* sh, int32_t cache_slots, void* cuda_st
   *out = nullptr;
   if (sh->n_layers < 1 || sh->hidden < 1 || sh->n_routed < 1 || sh->top_k < 1 || sh->inter_routed < 1 ||
       sh->batch < 1 || sh->n_shared < 0 || cache_slots < 1 || sh->top_k > sh->n_routed ||
-      (sh->n_shared > 0 && sh->inter_shared < 1) || (sh->weight_dtype != REMOE_F32 && sh->weight_dtype != REMOE_BF16 && sh->weight_dtype != REMOE_FP8_E4M3))
+      (sh->n_shared > 0 && sh->inter_shared < 1) || (sh->weight_dtype != REMOE_F32 && sh->weight_dtype != REMOE_BF16 && sh->weight_dtype != REMOE_FP8_E4M3 &&
+       sh->weight_dtype != REMOE_INT4_G32))
     return REMOE_E_ARG;
   if (sh->batch == 1 && cache_slots < sh->top_k) return REMOE_E_CAPACITY;
-  const int wbytes = sh->weight_dtype == REMOE_BF16 ? 2 : (sh->weight_dtype == REMOE_FP8_E4M3 ? 1 : 4);
+  // host store: bytes per element, 0 tagging the 4-bit grouped format
+  const int wbytes = sh->weight_dtype == REMOE_BF16 ? 2
+                     : sh->weight_dtype == REMOE_FP8_E4M3 ? 1 : sh->weight_dtype == REMOE_INT4_G32 ? 0 : 4;
+  if (sh->weight_dtype == REMOE_INT4_G32 && sh->batch > 1) return REMOE_E_UNSUPPORTED;
   const int rbytes = sh->weight_dtype == REMOE_F32 ? 4 : 2;
+  // A batched stack over an FP8 store keeps its slots as bf16 operand tiles: fetched bytes are widened on arrival.
+  const bool widen = sh->weight_dtype == REMOE_FP8_E4M3 && sh->batch > 1;
+  const int dev_wbytes = widen ? 2 : wbytes;
   const long pairs = (long)sh->n_layers * (sh->top_k + sh->n_shared);
   if (sh->hidden > kMaxHidden || sh->n_routed > kMaxRouted || sh->top_k > 32 || cache_slots > kMaxSlots || cache_slots > sh->n_routed ||
       (long)sh->batch * sh->top_k > kMaxRequests || !ffn_stream_supported(sh->hidden, wbytes))
@@ -577,10 +593,13 @@ int remoe_stack_create(const remoe_shape* sh, int32_t cache_slots, void* cuda_st
   DevStack& d = s->d;
   d.L = sh->n_layers; d.H = sh->hidden; d.N = sh->n_routed; d.K = sh->top_k; d.I = sh->inter_routed;
   d.S = sh->n_shared; d.Is = sh->n_shared ? sh->inter_shared : 0; d.B = sh->batch; d.C = cache_slots;
-  d.shared_gate = sh->shared_gate ? 1 : 0; d.renorm = sh->renorm_topk ? 1 : 0; d.wbytes = wbytes; d.rbytes = rbytes;
+  d.shared_gate = sh->shared_gate ? 1 : 0; d.renorm = sh->renorm_topk ? 1 : 0; d.wbytes = dev_wbytes; d.rbytes = rbytes;
   d.policy = REMOE_POLICY_LRU; d.beta = 0.f; d.has_prev = 0;
-  d.slot_bytes = (size_t)3 * d.I * d.H * wbytes;
-  d.shared_bytes = (size_t)3 * d.Is * d.H * wbytes;
+  d.slot_bytes = (size_t)3 * d.I * weight_row_bytes(d.H, dev_wbytes);
+  d.shared_bytes = (size_t)3 * d.Is * weight_row_bytes(d.H, dev_wbytes);
+  s->fetch_bytes = (size_t)3 * d.I * weight_row_bytes(d.H, wbytes);
+  s->fetch_shared_bytes = (size_t)3 * d.Is * weight_row_bytes(d.H, wbytes);
+  s->widen_fp8 = widen;
   const size_t L = d.L;
   char *router = nullptr, *sgw = nullptr, *shared = nullptr, *slots = nullptr;
 #define TRY(x) do { rc = (x); if (rc != REMOE_OK) return bail(rc); } while (0)
@@ -632,13 +651,16 @@ int remoe_stack_create(const remoe_shape* sh, int32_t cache_slots, void* cuda_st
     const char* pick = std::getenv("REMOE_BATCHED_KERNEL");      // "mma" forces the mma.sync kernel
     if (ffn_batched_tc_supported(d) && ffn_batched_tc_maps_bytes() <= sizeof(s->tc_maps) &&
         !(pick && std::strcmp(pick, "mma") == 0)) {
-      s->stage_bytes = std::max((size_t)2 * d.C * d.slot_bytes, d.shared_bytes);
+      s->stage_bytes = std::max((size_t)2 * d.C * s->fetch_bytes, s->fetch_shared_bytes);
       TRY(dev_alloc(s, &s->stage_pool, s->stage_bytes));
       for (cudaEvent_t& e : s->ev_stage)
         if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return bail(REMOE_E_CUDA);
-      if (ffn_batched_tc_init(d, s->stage_pool, s->stage_bytes, s->tc_maps) != cudaSuccess) return bail(REMOE_E_CUDA);
+      // (the tensor maps describe a bf16 staging pool; FP8 blocks are rewritten by the widening kernel instead)
+      if (!widen && ffn_batched_tc_init(d, s->stage_pool, s->stage_bytes, s->tc_maps) != cudaSuccess)
+        return bail(REMOE_E_CUDA);
       s->use_tc = true;
     }
+    if (widen && !s->use_tc) return bail(REMOE_E_UNSUPPORTED);
   }
   const size_t io = L * d.B * d.H, kk = L * (size_t)s->BK;
   TRY(dev_alloc(s, &s->st_in_d, io));
@@ -683,9 +705,14 @@ int remoe_load_shared(remoe_stack* s, int32_t layer, int32_t idx, const void* bl
     // such a stack keeps its blocks in operand-tile order: land in the staging pool, then retile
     CK(cudaStreamSynchronize(s->copy_stream));
     CK(cudaStreamSynchronize(s->stream));
-    CK(cudaMemcpyAsync(s->stage_pool, block, s->d.shared_bytes, cudaMemcpyHostToDevice, s->stream));
+    CK(cudaMemcpyAsync(s->stage_pool, block, s->fetch_shared_bytes, cudaMemcpyHostToDevice, s->stream));
     const size_t off = 0;
-    CK(launch_retile_tc(s->d, s->tc_maps, 1, &off, &dst, s->d.Is, s->stream));
+    if (s->widen_fp8) {
+      const void* src = s->stage_pool;
+      CK(launch_widen_retile_tc(s->d, 1, &src, &dst, s->d.Is, s->stream));
+    } else {
+      CK(launch_retile_tc(s->d, s->tc_maps, 1, &off, &dst, s->d.Is, s->stream));
+    }
     s->kernel_launches += 1;
   } else {
     CK(cudaMemcpyAsync(dst, block, s->d.shared_bytes, cudaMemcpyHostToDevice, s->stream));

@@ -513,6 +513,45 @@ __global__ void __launch_bounds__(32) retile_kernel(const __grid_constant__ TcMa
   }
 }
 
+// ------------------------------------------------------------------------- FP8 widen + retile
+// A stack with an FP8 E4M3 host store (value = byte * 2^-8) at batch > 1 fetches FP8 bytes -- half of what
+// a bf16 block moves over the host link -- and keeps its slots as bf16 operand tiles, so the MMA kernel
+// above is the same.  This kernel does both steps at once for freshly fetched channel-major FP8 blocks:
+// every 16-byte piece of an operand tile is eight consecutive stored bytes of one row, widened exactly
+// (an E4M3 value times 2^-8 has at most 4 significant bits and fits bf16), written at the swizzled place
+// the tensor-map path would have put it.  One CTA per (64-channel group, block); plain loads and stores.
+struct WidenArgs {
+  int n, inter;
+  const unsigned char* src[kRetileJobs];   // channel-major FP8 block in the staging pool
+  char* dst[kRetileJobs];                  // destination block (slot or shared block), bf16 tile order
+};
+
+template <int H>
+__global__ void __launch_bounds__(256) widen_retile_kernel(const __grid_constant__ WidenArgs r) {
+  using G = TcGeo<H>;
+  constexpr int T = G::kChunks + G::kTiles;
+  const unsigned char* src = r.src[blockIdx.y] + (size_t)blockIdx.x * kTcBlockCh * 3 * H;
+  char* dst = r.dst[blockIdx.y] + (size_t)blockIdx.x * T * kTileBytes;
+  for (int q = threadIdx.x; q < T * 1024; q += 256) {
+    const int t = q >> 10, line = (q >> 3) & 127, pos = q & 7;
+    const int c = pos ^ (line & 7);                      // which 8 columns of the line sit at this place
+    int ch, kind, col;
+    if (t < G::kChunks) {                                // A1 tile: lines alternate gate / up of a channel
+      ch = line >> 1; kind = line & 1; col = t * 64 + c * 8;
+    } else {                                             // A2 tile: two halves of 64 channel lines
+      ch = line & 63; kind = 2; col = (t - G::kChunks) * 128 + (line >> 6) * 64 + c * 8;
+    }
+    const uint2 b = __ldg(reinterpret_cast<const uint2*>(src + ((size_t)ch * 3 + kind) * H + col));
+    float f[8];
+    Elems<1>::pair(b.x & 0xffffu, f[0], f[1]); Elems<1>::pair(b.x >> 16, f[2], f[3]);
+    Elems<1>::pair(b.y & 0xffffu, f[4], f[5]); Elems<1>::pair(b.y >> 16, f[6], f[7]);
+    constexpr float k = WScale<1>::kDot;                 // the store's power-of-two scale
+    *reinterpret_cast<uint4*>(dst + (size_t)t * kTileBytes + line * 128 + pos * 16) =
+        make_uint4(pack_bf16(f[0] * k, f[1] * k), pack_bf16(f[2] * k, f[3] * k), pack_bf16(f[4] * k, f[5] * k),
+                   pack_bf16(f[6] * k, f[7] * k));
+  }
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -589,6 +628,31 @@ cudaError_t launch_ffn_batched_tc(const BatchArgs& a, int grid, cudaStream_t st)
     case 2048: return launch_tc<2048>(a, grid, st);
   }
   return cudaErrorInvalidValue;
+}
+
+cudaError_t launch_widen_retile_tc(const DevStack& d, int n, const void* const* src, char* const* dst, int inter,
+                                   cudaStream_t st) {
+  for (int i0 = 0; i0 < n; i0 += kRetileJobs) {
+    WidenArgs r{};
+    r.n = n - i0 < kRetileJobs ? n - i0 : kRetileJobs;
+    r.inter = inter;
+    for (int i = 0; i < r.n; ++i) {
+      if (reinterpret_cast<uintptr_t>(src[i0 + i]) & 7u) return cudaErrorInvalidValue;
+      r.src[i] = static_cast<const unsigned char*>(src[i0 + i]);
+      r.dst[i] = dst[i0 + i];
+    }
+    const dim3 grid(inter / kTcBlockCh, r.n);
+    switch (d.H) {
+      case 256: widen_retile_kernel<256><<<grid, 256, 0, st>>>(r); break;
+      case 512: widen_retile_kernel<512><<<grid, 256, 0, st>>>(r); break;
+      case 1024: widen_retile_kernel<1024><<<grid, 256, 0, st>>>(r); break;
+      case 2048: widen_retile_kernel<2048><<<grid, 256, 0, st>>>(r); break;
+      default: return cudaErrorInvalidValue;
+    }
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
 }
 
 cudaError_t launch_retile_tc(const DevStack& d, const void* maps, int n, const size_t* src_offsets,

@@ -246,7 +246,7 @@ extern "C" int remoe_expert_ffn_static(int32_t hidden, int32_t weight_dtype, int
                                        void* cuda_stream) {
   if (!expert_blocks_dev || !inter || !scales || !hidden_in_dev || !hidden_out_dev || n_experts < 1)
     return REMOE_E_ARG;
-  if (weight_dtype == REMOE_FP8_E4M3) return REMOE_E_UNSUPPORTED;          // no kernel of this entry point reads FP8 blocks
+  if (weight_dtype == REMOE_FP8_E4M3 || weight_dtype == REMOE_INT4_G32) return REMOE_E_UNSUPPORTED;   // no kernel here reads these
   if (weight_dtype != REMOE_F32 && weight_dtype != REMOE_BF16) return REMOE_E_ARG;
   if (n_experts > REMOE_STATIC_MAX_EXPERTS || hidden > REMOE_STATIC_MAX_HIDDEN) return REMOE_E_UNSUPPORTED;
   const int wb = weight_dtype == REMOE_BF16 ? 2 : 4;

@@ -47,8 +47,8 @@ __host__ __device__ inline Layout make_layout(int H, int wbytes) {
   y.prefix = 2 * kMaxStages * sizeof(uint64_t);
   y.red = y.prefix + (size_t)(kMaxPairs + 1) * sizeof(int);
   y.red = (y.red + 127) / 128 * 128;
-  y.stages = y.red + (size_t)kConsumerWarps * 32 * (16 / wbytes) * sizeof(float);
-  const size_t stage = (size_t)3 * H * wbytes;
+  y.stages = y.red + (size_t)kConsumerWarps * 32 * weight_vec(wbytes) * sizeof(float);
+  const size_t stage = 3 * weight_row_bytes(H, wbytes);
   const size_t budget = 227 * 1024 - 1024;              // leave room for static shared memory
   int n = (int)((budget - y.stages) / stage);
   n = n >= kMaxStages ? kMaxStages : (n / kConsumerWarps) * kConsumerWarps;
@@ -75,8 +75,9 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(const __grid_co
   constexpr int kVec = E::kVec;
   constexpr int kIter = H / (32 * kVec);
   constexpr int kCols = kIter * kVec;                  // columns of h / out owned by one lane
-  constexpr uint32_t kStageBytes = 3u * H * WB;
-  constexpr uint32_t kRowBytes = (uint32_t)H * WB;
+  constexpr uint32_t kRowBytes = (uint32_t)weight_row_bytes(H, WB);
+  constexpr uint32_t kStageBytes = 3u * kRowBytes;
+  constexpr bool kGrouped = WB == 0;                   // per-group scales follow the codes of a row
 
   extern __shared__ __align__(128) unsigned char smem[];
   const Layout lay = make_layout(H, WB);
@@ -229,19 +230,40 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(const __grid_co
         }
         const char* st = reinterpret_cast<const char*>(stages) + (size_t)s * kStageBytes;
         float g = 0.f, u = 0.f;
+        float gs[kGrouped ? kIter : 1];                  // grouped format: this lane's group scales of the third row
+        if constexpr (kGrouped) {
 #pragma unroll
-        for (int it = 0; it < kIter; ++it) {
-          float w[kVec];
-          E::load(st + (it * 32 + lane) * 16, w);
+          for (int it = 0; it < kIter; ++it) {
+            float w[kVec], t = 0.f;
+            E::load(st + (it * 32 + lane) * 16, w);
 #pragma unroll
-          for (int j = 0; j < kVec; ++j) g = fmaf(w[j], hreg[it * kVec + j], g);
-        }
+            for (int j = 0; j < kVec; ++j) t = fmaf(w[j], hreg[it * kVec + j], t);
+            g = fmaf(E::scale(st, H, it * 32 + lane), t, g);
+          }
 #pragma unroll
-        for (int it = 0; it < kIter; ++it) {
-          float w[kVec];
-          E::load(st + kRowBytes + (it * 32 + lane) * 16, w);
+          for (int it = 0; it < kIter; ++it) {
+            float w[kVec], t = 0.f;
+            E::load(st + kRowBytes + (it * 32 + lane) * 16, w);
 #pragma unroll
-          for (int j = 0; j < kVec; ++j) u = fmaf(w[j], hreg[it * kVec + j], u);
+            for (int j = 0; j < kVec; ++j) t = fmaf(w[j], hreg[it * kVec + j], t);
+            u = fmaf(E::scale(st + kRowBytes, H, it * 32 + lane), t, u);
+            gs[it] = E::scale(st + 2 * kRowBytes, H, it * 32 + lane);
+          }
+        } else {
+#pragma unroll
+          for (int it = 0; it < kIter; ++it) {
+            float w[kVec];
+            E::load(st + (it * 32 + lane) * 16, w);
+#pragma unroll
+            for (int j = 0; j < kVec; ++j) g = fmaf(w[j], hreg[it * kVec + j], g);
+          }
+#pragma unroll
+          for (int it = 0; it < kIter; ++it) {
+            float w[kVec];
+            E::load(st + kRowBytes + (it * 32 + lane) * 16, w);
+#pragma unroll
+            for (int j = 0; j < kVec; ++j) u = fmaf(w[j], hreg[it * kVec + j], u);
+          }
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
@@ -255,8 +277,9 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(const __grid_co
         for (int it = 0; it < kIter; ++it) {
           float w[kVec];
           E::load(st + 2 * kRowBytes + (it * 32 + lane) * 16, w);
+          const float a_it = kGrouped ? av * gs[kGrouped ? it : 0] : av;
 #pragma unroll
-          for (int j = 0; j < kVec; ++j) acc[it * kVec + j] = fmaf(av, w[j], acc[it * kVec + j]);
+          for (int j = 0; j < kVec; ++j) acc[it * kVec + j] = fmaf(a_it, w[j], acc[it * kVec + j]);
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(empty + s);
@@ -339,6 +362,7 @@ cudaError_t launch_one(const FfnArgs& a, int grid, cudaStream_t st) {
 }  // namespace
 
 bool ffn_stream_supported(int H, int wbytes) {
+  if (wbytes == 0) return H == 1024 || H == 2048;
   if (wbytes == 4) return H == 128 || H == 256 || H == 512 || H == 1024;
   if (wbytes == 2) return H == 256 || H == 512 || H == 1024 || H == 2048;
   if (wbytes == 1) return H == 512 || H == 1024 || H == 2048;
@@ -367,11 +391,16 @@ cudaError_t launch_ffn_stream(const FfnArgs& a, int grid, cudaStream_t st) {
       case 1024: return launch_one<2, 1024>(a, grid, st);
       case 2048: return launch_one<2, 2048>(a, grid, st);
     }
-  } else {
+  } else if (a.d.wbytes == 1) {
     switch (H) {
       case 512: return launch_one<1, 512>(a, grid, st);
       case 1024: return launch_one<1, 1024>(a, grid, st);
       case 2048: return launch_one<1, 2048>(a, grid, st);
+    }
+  } else {
+    switch (H) {
+      case 1024: return launch_one<0, 1024>(a, grid, st);
+      case 2048: return launch_one<0, 2048>(a, grid, st);
     }
   }
   return cudaErrorInvalidValue;

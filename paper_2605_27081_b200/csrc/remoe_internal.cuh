@@ -30,7 +30,8 @@ enum : int {
 // Everything the kernels need, passed by value.
 struct DevStack {
   int L, H, N, K, I, S, Is, B, C;
-  int shared_gate, renorm, wbytes;     // wbytes: bytes per expert-block element: 4 float32, 2 bfloat16, 1 fp8 e4m3
+  int shared_gate, renorm, wbytes;     // wbytes: bytes per expert-block element: 4 float32, 2 bfloat16, 1 fp8 e4m3;
+                                       // 0 tags the 4-bit grouped format (see weight_row_bytes)
   int rbytes;                          // bytes per router / shared-gate element: 4 or 2
   int policy;
   float beta;
@@ -70,6 +71,14 @@ struct DevStack {
   int* grp_tok;                        // [L][B*K][B]
   int* grp_k;                          // [L][B*K][B]
 };
+
+// Bytes of one stored weight row of H elements: H * wbytes, or, for the 4-bit grouped format (wbytes == 0), H/2
+// bytes of packed codes followed by one bfloat16 scale per group of 32 elements.
+__host__ __device__ constexpr size_t weight_row_bytes(int H, int wbytes) {
+  return wbytes ? (size_t)H * wbytes : (size_t)H / 2 + (size_t)H / 16;
+}
+// Floats that sixteen stored bytes decode to.
+__host__ __device__ constexpr int weight_vec(int wbytes) { return wbytes ? 16 / wbytes : 32; }
 
 __host__ __device__ inline int trace_ints(int L, int BK) { return 2 * L + 5 * L * BK; }
 __host__ __device__ inline int* trace_tok_hits(int* t, int L, int BK) { return t + L + 5 * L * BK; }
@@ -129,6 +138,11 @@ cudaError_t launch_ffn_batched_tc(const BatchArgs& a, int grid, cudaStream_t st)
 // staging pool (multiples of 3 * H * 2) into dst[i] in operand-tile order.  Host arrays.
 cudaError_t launch_retile_tc(const DevStack& d, const void* maps, int n, const size_t* src_offsets,
                              char* const* dst, int inter, cudaStream_t st);
+
+// FP8 host store at batch > 1: n channel-major FP8 E4M3 blocks (value = byte * 2^-8) at src[i] (device,
+// 8-byte aligned) are widened to bf16 and written to dst[i] in operand-tile order.  Host arrays.
+cudaError_t launch_widen_retile_tc(const DevStack& d, int n, const void* const* src, char* const* dst, int inter,
+                                   cudaStream_t st);
 
 // Routes layers [layer0, layer0 + n_layers); `hidden_in`, `ids`, `gates` are the full [L, B, .] arrays.
 cudaError_t launch_route(const DevStack& d, const float* hidden_in, int* ids, float* gates,

@@ -116,6 +116,26 @@ struct Elems<1> {
     pair(v.w & 0xffffu, f[12], f[13]); pair(v.w >> 16, f[14], f[15]);
   }
 };
+// 4-bit grouped format (tag 0): sixteen stored bytes are one group of 32 codes, element 2i in the low and element
+// 2i+1 in the high half of byte i; a code c stands for (c - 8) * the group's scale, the scales (bfloat16) follow
+// the codes of a row.  load() yields the 32 integers c - 8 as floats (2^23 + c is the float with bit pattern
+// 0x4B000000 | c); the caller multiplies a group's finished partial sum by its scale.
+template <>
+struct Elems<0> {
+  static constexpr int kVec = 32;
+  __device__ static __forceinline__ void word(uint32_t w, float* f) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(((w >> (4 * i)) & 0xfu) | 0x4b000000u) - 8388616.f;
+  }
+  __device__ static __forceinline__ void load(const char* p, float* f) {
+    const uint4 v = *reinterpret_cast<const uint4*>(p);
+    word(v.x, f); word(v.y, f + 8); word(v.z, f + 16); word(v.w, f + 24);
+  }
+  // scale of 16-byte piece `piece` of the row starting at `row` (H elements)
+  __device__ static __forceinline__ float scale(const char* row, int H, int piece) {
+    return __uint_as_float((uint32_t)*reinterpret_cast<const unsigned short*>(row + H / 2 + 2 * piece) << 16);
+  }
+};
 // kDot rescales a finished dot product to its true value, kAct multiplies the activation before
 // the AXPY (FP8 weights are stored without their factor 2^-8).
 template <int WB>

@@ -29,8 +29,9 @@ class LoadedWorkload:
                  store_of: "LoadedWorkload | None" = None):
         self.shape, self.cache_slots, self.seed = shape, cache_slots, seed
         L, N = shape.n_layers, shape.n_routed
-        elems = synth.expert_block_elems(shape.hidden, shape.inter_routed)
-        np_dt = {0: np.float32, 1: np.uint16, 2: np.uint8}[shape.weight_dtype]
+        np_dt = {0: np.float32, 1: np.uint16, 2: np.uint8, 3: np.uint8}[shape.weight_dtype]
+        blk_bytes = synth.expert_block_bytes(shape)
+        elems = blk_bytes // np.dtype(np_dt).itemsize          # stored items per block
         if store_of is not None:
             o = store_of.shape
             same = (o.n_layers, o.hidden, o.inter_routed, o.weight_dtype, o.n_routed, store_of.seed) == \
@@ -44,7 +45,7 @@ class LoadedWorkload:
             nd = N if distinct_experts is None else min(N, int(distinct_experts))
             self.n_distinct = nd
             gen_shape = synth.Shape(**{**shape.asdict(), "n_routed": nd})
-            self._store_t = torch.empty(L * nd * elems * shape.elem_bytes, dtype=torch.uint8, pin_memory=True)
+            self._store_t = torch.empty(L * nd * blk_bytes, dtype=torch.uint8, pin_memory=True)
             self.store = self._store_t.numpy().view(np_dt).reshape(L, nd, elems)
             synth.fill_expert_store(seed, gen_shape, self.store, threads=threads)
         self.routers = [synth.gen_router(seed, shape, l) for l in range(L)]

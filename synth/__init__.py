@@ -16,6 +16,9 @@ from .workloads import (  # noqa: F401
     bf16_bits_to_f32,
     fp8_e4m3_round_to_bits,
     fp8_e4m3_bits_to_f32,
+    int4_g32_encode,
+    int4_g32_decode,
+    INT4_GROUP,
     widen,
     FP8_SHIFT,
     gen_router,

@@ -18,7 +18,9 @@ Element type is float32 (``weight_dtype == 0``) or bfloat16 stored as ``uint16``
 patterns (``weight_dtype == 1``), rounded to nearest-even once, at generation.  With
 ``weight_dtype == 2`` the expert blocks are OCP FP8 E4M3 bytes whose value is
 ``decode(byte) * 2**-FP8_SHIFT`` (a fixed power-of-two scale that puts N(0, 0.02^2) weights in
-the format's normal range) while the router and shared-gate weights stay bfloat16.
+the format's normal range) while the router and shared-gate weights stay bfloat16.  With
+``weight_dtype == 3`` the expert blocks are 4-bit integers in groups of 32 consecutive elements of a
+row with one bfloat16 scale per group (see ``int4_g32_encode``); router and shared gate again bfloat16.
 """
 from __future__ import annotations
 
@@ -37,6 +39,7 @@ KIND_RHO = 6
 
 EXPERT_STD = 0.02
 FP8_SHIFT = 8
+INT4_GROUP = 32
 
 
 @dataclass(frozen=True)
@@ -50,7 +53,7 @@ class Shape:
     inter_shared: int = 0
     shared_gate: int = 0      # 1: shared output scaled by sigmoid(w_sg . h)
     renorm_topk: int = 0      # 1: top-k gate weights renormalised to sum to 1
-    weight_dtype: int = 0     # 0 float32, 1 bfloat16
+    weight_dtype: int = 0     # 0 float32, 1 bfloat16, 2 fp8 e4m3, 3 int4 in groups of 32
     batch: int = 1
 
     def asdict(self):
@@ -58,8 +61,15 @@ class Shape:
 
     @property
     def elem_bytes(self) -> int:
-        """Bytes per element of an expert block."""
+        """Bytes per element of an expert block (whole-byte formats only)."""
         return {0: 4, 1: 2, 2: 1}[self.weight_dtype]
+
+    @property
+    def row_bytes(self) -> int:
+        """Bytes of one stored row of `hidden` expert-block elements."""
+        if self.weight_dtype == 3:
+            return self.hidden // 2 + 2 * (self.hidden // INT4_GROUP)
+        return self.hidden * self.elem_bytes
 
     @property
     def router_dtype(self) -> int:
@@ -85,8 +95,14 @@ CONFIGS = {
     "dsv2lite_fp8": dict(
         shape=Shape(26, 2048, 64, 6, 1408, 2, 1408, 0, 0, 2, 1),
         cache_slots=16, steps=512, rhos=(0.9, 0.5, 0.0), seed=0),
+    "dsv2lite_int4": dict(
+        shape=Shape(26, 2048, 64, 6, 1408, 2, 1408, 0, 0, 3, 1),
+        cache_slots=16, steps=512, rhos=(0.9, 0.5, 0.0), seed=0),
     "dsv2lite_b32": dict(
         shape=Shape(26, 2048, 64, 6, 1408, 2, 1408, 0, 0, 1, 32),
+        cache_slots=32, steps=1024, rhos=(None,), seed=0),
+    "dsv2lite_b32_fp8": dict(
+        shape=Shape(26, 2048, 64, 6, 1408, 2, 1408, 0, 0, 2, 32),
         cache_slots=32, steps=1024, rhos=(None,), seed=0),
 }
 
@@ -101,7 +117,7 @@ def expert_block_elems(hidden: int, inter: int) -> int:
 
 def expert_block_bytes(shape: Shape, shared: bool = False) -> int:
     inter = shape.inter_shared if shared else shape.inter_routed
-    return expert_block_elems(shape.hidden, inter) * shape.elem_bytes
+    return 3 * inter * shape.row_bytes
 
 
 def bf16_round_to_bits(x: np.ndarray) -> np.ndarray:
@@ -153,6 +169,44 @@ def fp8_e4m3_bits_to_f32(bits: np.ndarray) -> np.ndarray:
     return _FP8[np.asarray(bits, dtype=np.uint8)]
 
 
+def int4_g32_encode(x: np.ndarray, hidden: int) -> np.ndarray:
+    """float32 rows of `hidden` elements -> the 4-bit grouped storage format, as bytes.
+
+    Each row is cut into groups of 32 consecutive elements.  A group's scale is max|x| / 7 rounded to
+    bfloat16 (nearest, ties to even); its codes are q = round-half-even(x / scale) clipped to [-7, 7]
+    (all zero when the scale is zero), stored offset by 8 as unsigned nibbles, element 2i in the low and
+    element 2i+1 in the high half of byte i.  A stored row is `hidden/2` bytes of codes followed by
+    `hidden/32` bfloat16 scales (little endian); rows follow each other without padding.  The value a
+    stored element denotes is (nibble - 8) * scale."""
+    x = np.ascontiguousarray(x, dtype=np.float32).reshape(-1, hidden // INT4_GROUP, INT4_GROUP)
+    rows = x.shape[0]
+    amax = np.max(np.abs(x), axis=2)
+    s_bits = bf16_round_to_bits((amax / np.float32(7.0)).astype(np.float32))
+    s = bf16_bits_to_f32(s_bits)
+    safe = np.where(s > 0, s, np.float32(1.0))
+    q = np.clip(np.rint(x / safe[:, :, None]), -7, 7).astype(np.int16)
+    q = np.where(s[:, :, None] > 0, q, 0)
+    u = (q + 8).astype(np.uint8).reshape(rows, hidden)
+    packed = (u[:, 0::2] | (u[:, 1::2] << 4)).astype(np.uint8)
+    out = np.empty((rows, hidden // 2 + 2 * (hidden // INT4_GROUP)), dtype=np.uint8)
+    out[:, :hidden // 2] = packed
+    out[:, hidden // 2:] = s_bits.astype("<u2").view(np.uint8).reshape(rows, -1)
+    return out.reshape(-1)
+
+
+def int4_g32_decode(b: np.ndarray, hidden: int) -> np.ndarray:
+    """Bytes in the 4-bit grouped format -> the float32 values they denote (exact), flattened row by row."""
+    row = hidden // 2 + 2 * (hidden // INT4_GROUP)
+    b = np.asarray(b, dtype=np.uint8).reshape(-1, row)
+    codes = b[:, :hidden // 2]
+    u = np.empty((b.shape[0], hidden), dtype=np.int16)
+    u[:, 0::2] = codes & 0xF
+    u[:, 1::2] = codes >> 4
+    s = bf16_bits_to_f32(np.ascontiguousarray(b[:, hidden // 2:]).view("<u2").astype(np.uint16))
+    v = (u - 8).astype(np.float32).reshape(b.shape[0], -1, INT4_GROUP) * s[:, :, None]
+    return v.reshape(-1)
+
+
 def widen(shape: "Shape", a: np.ndarray, router: bool = False) -> np.ndarray:
     """Stored weights -> the float32 values they denote (router=True for router / gate tensors)."""
     dt = shape.router_dtype if router else shape.weight_dtype
@@ -160,6 +214,8 @@ def widen(shape: "Shape", a: np.ndarray, router: bool = False) -> np.ndarray:
         return bf16_bits_to_f32(a)
     if dt == 2:
         return fp8_e4m3_bits_to_f32(a) * np.float32(2.0 ** -FP8_SHIFT)
+    if dt == 3:
+        return int4_g32_decode(a, shape.hidden)
     return a
 
 
@@ -168,7 +224,13 @@ def _rng(seed: int, kind: int, a: int = 0, b: int = 0) -> np.random.Generator:
     return np.random.Generator(np.random.Philox(key=key))
 
 
-def _store(x32: np.ndarray, weight_dtype: int, out: np.ndarray | None) -> np.ndarray:
+def _store(x32: np.ndarray, weight_dtype: int, out: np.ndarray | None, hidden: int = 0) -> np.ndarray:
+    if weight_dtype == 3:
+        bits = int4_g32_encode(x32, hidden)
+        if out is None:
+            return bits
+        out[...] = bits.reshape(out.shape)
+        return out
     if weight_dtype == 2:
         bits = fp8_e4m3_round_to_bits(x32 * np.float32(2.0 ** FP8_SHIFT))
         if out is None:
@@ -210,7 +272,7 @@ def gen_expert_block(seed: int, shape: Shape, layer: int, expert: int,
     g = _rng(seed, KIND_EXPERT, layer, expert)
     x = g.standard_normal((n,), dtype=np.float32)
     x *= np.float32(EXPERT_STD)
-    return _store(x, shape.weight_dtype, out)
+    return _store(x, shape.weight_dtype, out, shape.hidden)
 
 
 def gen_shared_block(seed: int, shape: Shape, layer: int, idx: int,
@@ -220,7 +282,7 @@ def gen_shared_block(seed: int, shape: Shape, layer: int, idx: int,
     g = _rng(seed, KIND_SHARED, layer, idx)
     x = g.standard_normal((n,), dtype=np.float32)
     x *= np.float32(EXPERT_STD)
-    return _store(x, shape.weight_dtype, out)
+    return _store(x, shape.weight_dtype, out, shape.hidden)
 
 
 def fill_expert_store(seed: int, shape: Shape, store: np.ndarray, layers=None,

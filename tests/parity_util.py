@@ -6,7 +6,7 @@ import numpy as np
 import synth
 from oracle import remoe_oracle as orc
 
-TOL = {0: 1e-4, 1: 2e-2, 2: 2e-2}  # max|d| / max|ref| : float32, bf16, fp8 weights (fp32 accumulate)
+TOL = {0: 1e-4, 1: 2e-2, 2: 2e-2, 3: 2e-2}  # max|d| / max|ref| : float32, bf16, fp8, int4 weights (fp32 accumulate)
 NEAR_TIE = 1e-5                   # logit gap below which the selected list may differ
 
 

@@ -56,6 +56,24 @@ def test_batched_tensor_core_path(shape, c, rho):
     assert chk.max_out_err <= 2e-2
 
 
+@pytest.mark.parametrize("shape,c,rho", [
+    (synth.Shape(2, 512, 16, 2, 64, 1, 64, 0, 0, 2, 4), 6, 0.5),         # one block per expert, a shared expert
+    (synth.Shape(3, 512, 24, 3, 128, 2, 64, 1, 0, 2, 12), 8, None),      # union far above capacity, sigmoid gate
+    (synth.Shape(2, 2048, 64, 6, 192, 2, 192, 0, 0, 2, 32), 32, None),   # the serving configuration's layer shape
+])
+def test_batched_fp8_store(shape, c, rho):
+    """FP8 E4M3 host store under a batched stack: a miss moves half the bytes; the fetched block is widened
+    (exactly) to bf16 operand tiles on arrival, so outputs match the oracle on the FP8-denoted values."""
+    from paper_2605_27081_b200 import binding as B
+    chk, deepest = _run(shape, c, rho, steps=10, seed=6)
+    assert chk.max_out_err <= 2e-2
+    if shape.batch * shape.top_k > 2 * c:
+        assert deepest > c
+    # intermediate sizes the tensor-core path is not built for have no FP8 batched variant
+    rc, _ = B.remoe_stack_create(synth.Shape(2, 512, 16, 2, 40, 0, 0, 0, 0, 2, 4), 6)
+    assert rc == B.REMOE_E_UNSUPPORTED
+
+
 def test_batched_other_policy():
     _run(synth.Shape(2, 256, 16, 2, 64, 0, 0, 0, 0, 1, 6), 5, 0.4, steps=30, seed=4, dense_steps=0, policy=2)
 

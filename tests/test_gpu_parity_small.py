@@ -73,6 +73,23 @@ def test_fp8_expert_store(shape, c, rho):
     _run(shape, c, rho, steps=16, seed=9, dense_steps=1, host_api_every=5)
 
 
+@pytest.mark.parametrize("shape,c,rho", [
+    (synth.Shape(3, 1024, 20, 3, 72, 2, 40, 1, 0, 3, 1), 5, 0.6),       # int4 grouped blocks, bf16 router and gate
+    (synth.Shape(2, 2048, 64, 6, 44, 2, 44, 0, 1, 3, 1), 16, 0.9),      # full hidden width
+])
+def test_int4_expert_store(shape, c, rho):
+    chk = _run(shape, c, rho, steps=16, seed=10, dense_steps=1, host_api_every=5)
+    assert chk.max_out_err < 1e-4                # both sides use the exact stored values; fp32 accumulation
+
+
+def test_int4_store_limits():
+    from paper_2605_27081_b200 import binding as B
+    rc, _ = B.remoe_stack_create(synth.Shape(2, 512, 16, 2, 32, 0, 0, 0, 0, 3, 1), 4)      # H not 1024 / 2048
+    assert rc == B.REMOE_E_UNSUPPORTED
+    rc, _ = B.remoe_stack_create(synth.Shape(2, 1024, 16, 2, 64, 0, 0, 0, 0, 3, 4), 4)     # batched
+    assert rc == B.REMOE_E_UNSUPPORTED
+
+
 def test_many_layers_span_ctas():
     """Enough rows that CTAs cross expert and layer boundaries in the streaming kernel."""
     shape = synth.Shape(12, 512, 16, 4, 300, 1, 300, 0, 0, 1, 1)

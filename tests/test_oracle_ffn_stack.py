@@ -275,3 +275,56 @@ def test_fp8_storage_matches_library_cast():
     assert blk.dtype == np.uint8 and synth.gen_router(0, shape, 0).dtype == np.uint16
     w = synth.widen(shape, blk)
     assert 0.015 < w.std() < 0.025 and np.abs(w).max() < 448 / 256
+
+
+def test_int4_grouped_storage_hand_example_and_error_bound():
+    """The 4-bit grouped format against a group worked by hand and against its definition: value =
+    (code - 8) * bf16 scale, scale = bf16(max|x| / 7), codes = round-half-even(x / scale) in [-7, 7];
+    a row is H/2 code bytes (element 2i in the low half of byte i) followed by H/32 little-endian bf16
+    scales."""
+    H = 64
+    x = np.zeros((2, H), np.float32)
+    # row 0, group 0: max 3.5 -> scale 0.5 exactly; codes = x / 0.5
+    x[0, :8] = [3.5, -3.5, 0.5, -0.5, 0.25, 0.75, 1.0, -2.0]          # 0.25/0.5 = 0.5 -> 0 (ties to even); 0.75/0.5 = 1.5 -> 2
+    # row 0, group 1: all zero -> scale 0, codes 8
+    # row 1, group 0: max 7 -> scale 1; row 1, group 1: max 14 -> scale 2
+    x[1, 0], x[1, 1], x[1, 31] = 7.0, -3.0, 2.4
+    x[1, 32], x[1, 33], x[1, 63] = -14.0, 5.0, 3.0                    # 5/2 = 2.5 -> 2 ; 3/2 = 1.5 -> 2
+    b = synth.int4_g32_encode(x, H).reshape(2, H // 2 + 4)
+    want0 = [7, -7, 1, -1, 0, 2, 2, -4] + [0] * 24
+    codes0 = [(int(b[0, i // 2]) >> (4 * (i % 2))) & 15 for i in range(32)]
+    assert codes0 == [q + 8 for q in want0]
+    assert all(int(v) == 0x88 for v in b[0, 16:32])                   # the all-zero group: code 8 everywhere
+    assert list(b[0, 32:36]) == [0x00, 0x3F, 0x00, 0x00]              # bf16(0.5) = 0x3F00, then bf16(0) little endian
+    assert list(b[1, 32:36]) == [0x80, 0x3F, 0x00, 0x40]              # bf16(1.0) = 0x3F80, bf16(2.0) = 0x4000
+    v = synth.int4_g32_decode(b.reshape(-1), H).reshape(2, H)
+    assert list(v[0, :8]) == [3.5, -3.5, 0.5, -0.5, 0.0, 1.0, 1.0, -2.0] and not v[0, 8:].any()
+    assert (v[1, 0], v[1, 1], v[1, 31], v[1, 32], v[1, 33], v[1, 63]) == (7.0, -3.0, 2.0, -14.0, 4.0, 4.0)
+    # random rows: brute-force decode per element, error at most half a step of the group's stored scale,
+    # the group maximum itself reproduced to the bf16 rounding of the scale
+    rng = np.random.default_rng(1)
+    H = 256
+    y = (rng.standard_normal((5, H)) * 0.02).astype(np.float32)
+    bb = synth.int4_g32_encode(y, H)
+    assert bb.size == 5 * (H // 2 + 2 * (H // 32))
+    dec = synth.int4_g32_decode(bb, H).reshape(5, H)
+    rows = bb.reshape(5, -1)
+    for r in range(5):
+        for gidx in range(H // 32):
+            sb = int(rows[r, H // 2 + 2 * gidx]) | (int(rows[r, H // 2 + 2 * gidx + 1]) << 8)
+            scale = float(np.array([sb << 16], np.uint32).view(np.float32)[0])
+            seg = y[r, 32 * gidx:32 * gidx + 32]
+            assert abs(scale - np.abs(seg).max() / 7) <= 2.0 ** -8 * scale
+            for j in range(32):
+                byte = int(rows[r, (32 * gidx + j) // 2])
+                code = (byte >> 4) if j % 2 else (byte & 15)
+                assert 1 <= code <= 15
+                val = (code - 8) * scale
+                assert val == dec[r, 32 * gidx + j]
+                assert abs(val - seg[j]) <= 0.5 * scale * (1 + 2.0 ** -7)
+    shape = synth.Shape(1, 1024, 4, 2, 8, 0, 0, 0, 0, 3, 1)
+    blk = synth.gen_expert_block(0, shape, 0, 1)
+    assert blk.dtype == np.uint8 and blk.size == synth.expert_block_bytes(shape) == 3 * 8 * (512 + 64)
+    assert synth.gen_router(0, shape, 0).dtype == np.uint16
+    w = synth.widen(shape, blk)
+    assert w.size == 3 * 8 * 1024 and 0.015 < w.std() < 0.025
