@@ -39,7 +39,9 @@ namespace {
 constexpr int kTcTokTile = 16;
 constexpr int kTcBlockCh = 64;
 constexpr int kTcThreads = 192;
-constexpr int kTileBytes = 16384;                      // one ring stage: 128 rows x 128 B
+constexpr int kTileBytes = 16384;                      // one operand tile: 128 rows x 128 B
+constexpr int kStageTiles = 2;                         // tiles per ring stage (one bulk copy, one barrier round trip)
+constexpr int kStageBytes = kStageTiles * kTileBytes;
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kD2Col = 32;                        // D1 buffers at columns 0 and 16, D2 tiles from column 32
 
@@ -149,8 +151,9 @@ struct TcGeo {
   static constexpr int kB1Bytes = kChunks * 2048;      // X^T: 16 tokens x 128 B per chunk
   static constexpr int kB2Bytes = 2048;                // a: 16 tokens x 64 channels
   static constexpr int kFixed = kB1Bytes + kB2Bytes;
-  static constexpr int kStages = (227 * 1024 - 2048 - kFixed) / kTileBytes > 10 ? 10 : (227 * 1024 - 2048 - kFixed) / kTileBytes;
-  static constexpr size_t kSmem = 1024 + kFixed + (size_t)kStages * kTileBytes + 512;
+  static constexpr int kStages = (227 * 1024 - 2048 - kFixed) / kStageBytes > 5 ? 5 : (227 * 1024 - 2048 - kFixed) / kStageBytes;
+  static constexpr size_t kSmem = 1024 + kFixed + (size_t)kStages * kStageBytes + 512;
+  static_assert(kChunks % kStageTiles == 0 && kTiles % kStageTiles == 0, "a stage never spans two tile kinds");
 };
 
 template <int H>
@@ -163,7 +166,7 @@ ffn_batched_tc_kernel(const __grid_constant__ BatchArgs a) {
   unsigned char* b1 = smem;
   unsigned char* b2 = b1 + G::kB1Bytes;
   unsigned char* ring = b2 + G::kB2Bytes;                              // 1024-byte aligned
-  uint64_t* bars = reinterpret_cast<uint64_t*>(ring + (size_t)NS * kTileBytes);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(ring + (size_t)NS * kStageBytes);
   uint64_t *full = bars, *empty = bars + NS;
   uint64_t* x_full = bars + 2 * NS;        // X^T of a piece staged            (128 epilogue threads)
   uint64_t* x_empty = x_full + 1;          // X^T no longer read                 (commit)
@@ -221,16 +224,16 @@ ffn_batched_tc_kernel(const __grid_constant__ BatchArgs a) {
       auto emit = [&](const GroupRec& g, bool second) {
         // tiles of this group in the block: A1 tiles first, then the A2 tiles
         const char* src = g.p.base + ((size_t)g.blk * (G::kChunks + G::kTiles) + (second ? G::kChunks : 0)) * kTileBytes;
-        const int tiles = second ? G::kTiles : G::kChunks;
-        for (int t = 0; t < tiles && ok; ++t, ++n) {
+        const int stages = (second ? G::kTiles : G::kChunks) / kStageTiles;
+        for (int t = 0; t < stages && ok; ++t, ++n) {
           const int s = n % NS;
           if (n >= NS && (aborted() || !mbar_wait(empty + s, ((n / NS) - 1) & 1))) {
             if (!aborted()) fail(kErrWaitEmpty);
             ok = false;
             break;
           }
-          mbar_expect_tx(full + s, kTileBytes);
-          bulk_g2s(ring + (size_t)s * kTileBytes, src + (size_t)t * kTileBytes, kTileBytes, full + s);
+          mbar_expect_tx(full + s, kStageBytes);
+          bulk_g2s(ring + (size_t)s * kStageBytes, src + (size_t)t * kStageBytes, kStageBytes, full + s);
         }
       };
       GroupWalk walk(a, n_items, ua, ub, j0);
@@ -258,16 +261,20 @@ ffn_batched_tc_kernel(const __grid_constant__ BatchArgs a) {
         if (g.first) ok = !aborted() && mbar_wait(x_full, g.np & 1);
         if (ok && g.idx >= 2) ok = !aborted() && mbar_wait(d1_empty + (g.idx & 1), ((g.idx >> 1) - 1) & 1);
         const uint32_t dcol = tmem + (uint32_t)(g.idx & 1) * 16;
-        for (int kc = 0; kc < G::kChunks && ok; ++kc, ++n) {
+        for (int kc = 0; kc < G::kChunks && ok; kc += kStageTiles, ++n) {
           const int s = n % NS;
           ok = !aborted() && mbar_wait(full + s, (n / NS) & 1);
           if (!ok) break;
           tc_fence_after();
-          const uint32_t a_addr = smem_u32(ring + (size_t)s * kTileBytes), b_addr = smem_u32(b1 + kc * 2048);
 #pragma unroll
-          for (int k = 0; k < 4; ++k)
-            umma(dcol, smem_desc(a_addr + k * 32, 16, 1024), smem_desc(b_addr + k * 32, 16, 1024), kIdescK,
-                 (kc | k) ? 1u : 0u);
+          for (int j = 0; j < kStageTiles; ++j) {
+            const uint32_t a_addr = smem_u32(ring + (size_t)s * kStageBytes + j * kTileBytes);
+            const uint32_t b_addr = smem_u32(b1 + (kc + j) * 2048);
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+              umma(dcol, smem_desc(a_addr + k * 32, 16, 1024), smem_desc(b_addr + k * 32, 16, 1024), kIdescK,
+                   (kc | j | k) ? 1u : 0u);
+          }
           umma_commit(empty + s);
         }
         if (!ok) return;
@@ -279,16 +286,20 @@ ffn_batched_tc_kernel(const __grid_constant__ BatchArgs a) {
         ok = !aborted() && mbar_wait(b2_full, g.idx & 1);
         if (ok && g.first && g.np > 0) ok = !aborted() && mbar_wait(d2_empty, (g.np - 1) & 1);
         tc_fence_after();
-        for (int ht = 0; ht < G::kTiles && ok; ++ht, ++n) {
+        for (int ht = 0; ht < G::kTiles && ok; ht += kStageTiles, ++n) {
           const int s = n % NS;
           ok = !aborted() && mbar_wait(full + s, (n / NS) & 1);
           if (!ok) break;
           tc_fence_after();
-          const uint32_t a_addr = smem_u32(ring + (size_t)s * kTileBytes), b_addr = smem_u32(b2);
+          const uint32_t b_addr = smem_u32(b2);
 #pragma unroll
-          for (int k = 0; k < 4; ++k)
-            umma(tmem + kD2Col + ht * 16, smem_desc(a_addr + k * 2048, 8192, 1024), smem_desc(b_addr + k * 32, 16, 1024),
-                 kIdescMN, (!g.first || k) ? 1u : 0u);
+          for (int j = 0; j < kStageTiles; ++j) {
+            const uint32_t a_addr = smem_u32(ring + (size_t)s * kStageBytes + j * kTileBytes);
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+              umma(tmem + kD2Col + (ht + j) * 16, smem_desc(a_addr + k * 2048, 8192, 1024),
+                   smem_desc(b_addr + k * 32, 16, 1024), kIdescMN, (!g.first || k) ? 1u : 0u);
+          }
           umma_commit(empty + s);
         }
         if (!ok) return;
