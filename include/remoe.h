@@ -53,7 +53,9 @@ enum {
   REMOE_E_CUDA = -5,         /* a CUDA runtime call failed; see remoe_last_cuda_error()   */
   REMOE_E_DEVICE_FLAG = -6,  /* a kernel recorded an internal error (bounded wait ran out, bad index) */
   REMOE_E_UNSUPPORTED = -7,  /* shape outside what the kernels are built for              */
-  REMOE_E_NOMEM = -8         /* host or device allocation failed                          */
+  REMOE_E_NOMEM = -8,        /* host or device allocation failed                          */
+  REMOE_E_ORDER = -9         /* REMOE_CHECK_ORDER=1 only: the call enqueued a slot access whose order
+                                the streams and events do not guarantee; see remoe_last_cuda_error() */
 };
 
 enum { REMOE_F32 = 0, REMOE_BF16 = 1, REMOE_FP8_E4M3 = 2, REMOE_INT4_G32 = 3 };
@@ -104,6 +106,10 @@ typedef struct remoe_stack remoe_stack;
  * library also owns one copy stream.  Allocates the slot pools, directory and scratch on
  * the current device.  Errors: ARG, CAPACITY (B == 1 and C < K), UNSUPPORTED, NOMEM, CUDA.
  * Environment read here: REMOE_BATCHED_KERNEL=mma keeps a batched stack on the mma.sync expert kernel;
+ * REMOE_CHECK_ORDER=1 makes every decode call also replay what it enqueues on its streams (launches, copies,
+ * event records and waits, host waits) into a host-side ledger that checks, per cache slot, that each write
+ * is ordered behind the readers of the previous contents and each read behind the write that filled it; a
+ * call that fails the check returns REMOE_E_ORDER (a debugging aid: host work only, no effect on the GPU);
  * REMOE_FAULT_INJECT=lost_copy (failure-detection tests, batch 1) makes the first step's resident-phase
  * expert launch run with a short wait limit and never issue the copy of its first weight row: the
  * consumer's bounded wait runs out, the kernel sets the error word and returns, and the error surfaces as
@@ -264,6 +270,10 @@ int remoe_set_reroute_beta(remoe_stack*, float beta);
 int remoe_set_profiling(remoe_stack*, int32_t on);
 int remoe_kernel_time(remoe_stack*, int32_t phase, double* ms_sum, uint64_t* launches,
                       uint64_t* weight_bytes);
+
+/* Ordering checker of a stack created with REMOE_CHECK_ORDER=1 (see remoe_stack_create): how many pairs of
+ * operations it has compared so far and how many were found unordered; both 0 on other stacks. */
+int remoe_order_check_counts(remoe_stack*, uint64_t* comparisons, uint64_t* violations);
 
 /* Number of kernels this stack has launched since creation (all kinds). */
 int remoe_launch_count(remoe_stack*, uint64_t* launches);

@@ -16,7 +16,7 @@ LIB_PATH = os.path.join(_PKG, "libremoe.so")
 
 REMOE_OK = 0
 REMOE_E_ARG, REMOE_E_CAPACITY, REMOE_E_NOT_LOADED, REMOE_E_NOT_PINNED = -1, -2, -3, -4
-REMOE_E_CUDA, REMOE_E_DEVICE_FLAG, REMOE_E_UNSUPPORTED, REMOE_E_NOMEM = -5, -6, -7, -8
+REMOE_E_CUDA, REMOE_E_DEVICE_FLAG, REMOE_E_UNSUPPORTED, REMOE_E_NOMEM, REMOE_E_ORDER = -5, -6, -7, -8, -9
 REMOE_F32, REMOE_BF16, REMOE_FP8_E4M3, REMOE_INT4_G32 = 0, 1, 2, 3
 REMOE_POLICY_LRU, REMOE_POLICY_FIFO, REMOE_POLICY_LFU = 0, 1, 2
 
@@ -26,7 +26,7 @@ EXPORTS = [
     "remoe_reuse_stats", "remoe_cache_reset", "remoe_set_policy", "remoe_set_reroute_beta",
     "remoe_set_profiling", "remoe_kernel_time", "remoe_launch_count", "remoe_last_cuda_error", "remoe_stack_destroy",
     "remoe_strerror", "remoe_expert_ffn_static", "remoe_reuse_mass", "remoe_step_history", "remoe_tpot_proxy", "remoe_decode_step_chained",
-    "remoe_expert_load", "remoe_decode_steps",
+    "remoe_expert_load", "remoe_decode_steps", "remoe_order_check_counts",
 ]
 
 
@@ -77,6 +77,7 @@ def lib():
         L.remoe_set_profiling.argtypes = [vp, i32]
         L.remoe_kernel_time.argtypes = [vp, i32, C.POINTER(C.c_double), C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
         L.remoe_launch_count.argtypes = [vp, C.POINTER(C.c_uint64)]
+        L.remoe_order_check_counts.argtypes = [vp, C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
         L.remoe_expert_ffn_static.argtypes = [i32, i32, i32, C.POINTER(vp), C.POINTER(i32), C.POINTER(C.c_float),
                                               vp, vp, vp]
         L.remoe_reuse_mass.argtypes = [vp, i32, C.POINTER(C.c_double), C.POINTER(C.c_uint64), vp]
@@ -206,6 +207,12 @@ def remoe_launch_count(h):
     return rc, int(n.value)
 
 
+def remoe_order_check_counts(h):
+    c, v = C.c_uint64(), C.c_uint64()
+    rc = lib().remoe_order_check_counts(h, C.byref(c), C.byref(v))
+    return rc, int(c.value), int(v.value)
+
+
 def remoe_expert_ffn_static(hidden, weight_dtype, expert_blocks_dev, inter, scales, hidden_in, hidden_out,
                             cuda_stream=None):
     """Allocation-free expert sum of one layer; `expert_blocks_dev` are device tensors/addresses."""
@@ -270,7 +277,7 @@ class Stack:
 
     def _ck(self, rc, what):
         if rc != REMOE_OK:
-            raise RemoeError(rc, what, remoe_last_cuda_error(self.h) if rc in (REMOE_E_CUDA, REMOE_E_DEVICE_FLAG) else "")
+            raise RemoeError(rc, what, remoe_last_cuda_error(self.h) if rc in (REMOE_E_CUDA, REMOE_E_DEVICE_FLAG, REMOE_E_ORDER) else "")
 
     def load_router(self, layer, w_router, w_shared_gate=None):
         self._ck(remoe_load_router(self.h, layer, w_router, w_shared_gate), "remoe_load_router")
@@ -357,6 +364,11 @@ class Stack:
         rc, n = remoe_launch_count(self.h)
         self._ck(rc, "remoe_launch_count")
         return n
+
+    def order_check_counts(self):
+        rc, c, v = remoe_order_check_counts(self.h)
+        self._ck(rc, "remoe_order_check_counts")
+        return c, v
 
     def close(self):
         if self.h is not None:

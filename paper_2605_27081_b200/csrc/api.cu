@@ -14,12 +14,14 @@
 // slot except the misses of an already routed step (no speculative prefetch, which would
 // break the fetch bound of Prop. 3.1).
 #include "remoe_internal.cuh"
+#include "order_ledger.h"
 
 #include <algorithm>
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <memory>
 #include <new>
 #include <string>
 #include <vector>
@@ -97,6 +99,11 @@ struct remoe_stack {
   // failure-detection test aid (REMOE_FAULT_INJECT=lost_copy at creation): the first resident-phase launch
   // of the batch-1 step runs with a short wait limit and one weight row whose copy is never issued
   bool inject_lost_copy = false;
+  // REMOE_CHECK_ORDER=1 at creation: every decode call also replays what it enqueues (operations, event
+  // records and waits, host waits) into a ledger that checks that each write of a cache slot is ordered
+  // behind the readers of the slot's previous contents and each read behind the write that filled it
+  std::unique_ptr<OrderLedger> ledger;
+  uint64_t ledger_reported = 0;
   int policy = REMOE_POLICY_LRU;
   float beta = 0.f;
 };
@@ -137,6 +144,26 @@ struct DeviceGuard {
 #define ON_STACK_DEVICE(s)                                                       \
   DeviceGuard device_guard_((s)->device);                                        \
   if (device_guard_.err != cudaSuccess) return fail_cuda((s), device_guard_.err, "cudaSetDevice")
+
+// ---- ordering ledger hooks (no-ops unless the stack was created with REMOE_CHECK_ORDER=1)
+enum { kStCompute = 0, kStCopy = 1, kStRoute = 2 };
+using LOp = OrderLedger::Op;
+inline LOp l_op(remoe_stack* s, int st) { return s->ledger ? s->ledger->op(st) : LOp{}; }
+inline void l_record(remoe_stack* s, const void* ev, int st) { if (s->ledger) s->ledger->record(ev, st); }
+inline void l_wait(remoe_stack* s, int st, const void* ev) { if (s->ledger) s->ledger->wait(st, ev); }
+inline void l_host_wait(remoe_stack* s, const void* ev) { if (s->ledger) s->ledger->host_wait(ev); }
+inline void l_host_sync(remoe_stack* s, int st) { if (s->ledger) s->ledger->host_sync(st); }
+inline void l_read(remoe_stack* s, const LOp& o, uint64_t cell, const char* what) { if (s->ledger) s->ledger->read(o, cell, what); }
+inline void l_write(remoe_stack* s, const LOp& o, uint64_t cell, const char* what) { if (s->ledger) s->ledger->write(o, cell, what); }
+inline uint64_t slot_cell(const remoe_stack* s, int l, int slot) { return (uint64_t)l * s->d.C + slot; }
+inline uint64_t stage_cell(const remoe_stack* s, int half, int i) { return (1ull << 40) + (uint64_t)half * s->d.C + i; }
+// New violations since the last call end the call with REMOE_E_ORDER.
+int l_verdict(remoe_stack* s) {
+  if (!s->ledger || s->ledger->violations() == s->ledger_reported) return REMOE_OK;
+  s->ledger_reported = s->ledger->violations();
+  s->cuda_err = "schedule order: " + s->ledger->first_violation();
+  return REMOE_E_ORDER;
+}
 
 template <typename T>
 int dev_alloc(remoe_stack* s, T** p, size_t count) {
@@ -180,6 +207,7 @@ int reset_state(remoe_stack* s) {
   CK(cudaMemsetAsync(d.mass_sum, 0, L * d.B * sizeof(double), s->stream));
   CK(cudaMemsetAsync(s->dev_block, 0, s->block_ints * sizeof(int), s->stream));
   CK(cudaStreamSynchronize(s->stream));
+  l_host_sync(s, kStCompute);
   std::memset(s->host_block, 0, s->block_ints * sizeof(int));
   if (s->host_block2) std::memset(s->host_block2, 0, s->block_ints * sizeof(int));
   s->steps = 0;
@@ -271,7 +299,7 @@ cudaError_t launch_batched(remoe_stack* s, const BatchArgs& a) {
 // by layer; each (depth, layer) group computed once its copies have landed.  The resident-phase launch
 // covering these layers must already be enqueued with ev_resident recorded behind it.  Adds the
 // algorithmic bytes of that launch to *resident_bytes.
-int batched_waves(remoe_stack* s, BatchArgs& a, int l0, int l1, uint64_t* resident_bytes) {
+int batched_waves(remoe_stack* s, BatchArgs& a, int l0, int l1, uint64_t* resident_bytes, const LOp& op_res) {
   DevStack& d = s->d;
   const int BK = s->BK;
   int* tr = s->host_block + 1;
@@ -285,7 +313,11 @@ int batched_waves(remoe_stack* s, BatchArgs& a, int l0, int l1, uint64_t* reside
     if (t_nu[l] < 0 || t_nu[l] > BK) return REMOE_E_DEVICE_FLAG;
     for (int i = 0; i < t_nu[l]; ++i) {
       const int j = l * BK + i;
-      if (t_hit[j]) { *resident_bytes += d.slot_bytes; continue; }
+      if (t_hit[j]) {
+        *resident_bytes += d.slot_bytes;
+        if (t_slot[j] >= 0 && t_slot[j] < d.C) l_read(s, op_res, slot_cell(s, l, t_slot[j]), "resident-phase launch");
+        continue;
+      }
       if (t_req[j] < 0 || t_req[j] >= d.N || t_slot[j] < 0 || t_slot[j] >= d.C || t_depth[j] < 0)
         return REMOE_E_DEVICE_FLAG;
       if (t_depth[j] > max_depth) max_depth = t_depth[j];
@@ -309,12 +341,18 @@ int batched_waves(remoe_stack* s, BatchArgs& a, int l0, int l1, uint64_t* reside
   // half of the staging pool and the retile kernel, on the compute stream behind those readers, writes
   // the slot; the copy engine then only ever waits for a staging half to be free.
   const bool staged = s->use_tc;
-  if (max_depth >= 0 && !staged) CK(cudaStreamWaitEvent(s->copy_stream, s->ev_trace, 0));
+  if (max_depth >= 0 && !staged) {
+    CK(cudaStreamWaitEvent(s->copy_stream, s->ev_trace, 0));
+    l_wait(s, kStCopy, s->ev_trace);
+  }
   std::vector<size_t> src_off;
   std::vector<char*> dst_ptr;
   std::vector<const void*> src_ptr;
   for (int dep = 0; dep <= max_depth; ++dep) {
-    if (dep == 1 && !staged) CK(cudaStreamWaitEvent(s->copy_stream, s->ev_resident, 0));   // displaced hits are done
+    if (dep == 1 && !staged) {
+      CK(cudaStreamWaitEvent(s->copy_stream, s->ev_resident, 0));   // displaced hits are done
+      l_wait(s, kStCopy, s->ev_resident);
+    }
     for (int l = l0; l < l1; ++l) {
       // one (depth, layer) group: its copies, then (enqueued at once, run when they have landed) its
       // retile and compute launches.  Streams keep the order depth-major, layer-minor.
@@ -330,7 +368,10 @@ int batched_waves(remoe_stack* s, BatchArgs& a, int l0, int l1, uint64_t* reside
           if (!misses) {
             // the half's previous user is the group before last: its retile is already enqueued
             half = (int)(s->stage_group++ & 1);
-            if (s->stage_used[half]) CK(cudaStreamWaitEvent(s->copy_stream, s->ev_stage[half], 0));
+            if (s->stage_used[half]) {
+              CK(cudaStreamWaitEvent(s->copy_stream, s->ev_stage[half], 0));
+              l_wait(s, kStCopy, s->ev_stage[half]);
+            }
           }
           if (misses >= d.C) return REMOE_E_DEVICE_FLAG;         // more misses of one depth than slots: bad trace
           src_off.push_back(((size_t)half * d.C + misses) * s->fetch_bytes);
@@ -338,17 +379,21 @@ int batched_waves(remoe_stack* s, BatchArgs& a, int l0, int l1, uint64_t* reside
           land = s->stage_pool + src_off.back();
         } else if (!misses && dep >= 1 && had[(size_t)(dep - 1) * d.L + l]) {
           CK(cudaStreamWaitEvent(s->copy_stream, ev_comp(dep - 1, l), 0));        // displaced misses are done
+          l_wait(s, kStCopy, ev_comp(dep - 1, l));
         }
         CK(cudaMemcpyAsync(land, s->host_ptrs[(size_t)l * d.N + t_req[j]], s->fetch_bytes, cudaMemcpyHostToDevice,
                            s->copy_stream));
+        l_write(s, l_op(s, kStCopy), staged ? stage_cell(s, half, misses) : slot_cell(s, l, t_slot[j]), "miss fetch");
         ++misses;
       }
       if (!misses) continue;
       had[(size_t)dep * d.L + l] = 1;
       s->h2d_bytes[l] += (uint64_t)misses * s->fetch_bytes;
       CK(cudaEventRecord(ev_copy(dep, l), s->copy_stream));
+      l_record(s, ev_copy(dep, l), kStCopy);
 
       CK(cudaStreamWaitEvent(s->stream, ev_copy(dep, l), 0));
+      l_wait(s, kStCompute, ev_copy(dep, l));
       if (staged) {
         if (s->widen_fp8) {
           src_ptr.clear();
@@ -358,7 +403,18 @@ int batched_waves(remoe_stack* s, BatchArgs& a, int l0, int l1, uint64_t* reside
           CK(launch_retile_tc(d, s->tc_maps, misses, src_off.data(), dst_ptr.data(), d.I, s->stream));
         }
         s->kernel_launches += (misses + 63) / 64;
+        if (s->ledger) {
+          const LOp ot = l_op(s, kStCompute);             // reads the staging half, rewrites the slots
+          int m = 0;
+          for (int i = 0; i < t_nu[l]; ++i) {
+            const int j = l * BK + i;
+            if (t_hit[j] || t_depth[j] != dep) continue;
+            l_read(s, ot, stage_cell(s, half, m++), "retile");
+            l_write(s, ot, slot_cell(s, l, t_slot[j]), "retile");
+          }
+        }
         CK(cudaEventRecord(s->ev_stage[half], s->stream));
+        l_record(s, s->ev_stage[half], kStCompute);
         s->stage_used[half] = true;
       }
       a.phase = 1;
@@ -368,9 +424,17 @@ int batched_waves(remoe_stack* s, BatchArgs& a, int l0, int l1, uint64_t* reside
       if (rc != REMOE_OK) return rc;
       CK(launch_batched(s, a));
       s->kernel_launches += 2;
+      if (s->ledger) {
+        const LOp om = l_op(s, kStCompute);
+        for (int i = 0; i < t_nu[l]; ++i) {
+          const int j = l * BK + i;
+          if (!t_hit[j] && t_depth[j] == dep) l_read(s, om, slot_cell(s, l, t_slot[j]), "miss-phase launch");
+        }
+      }
       rc = prof_end(s, s->stream);
       if (rc != REMOE_OK) return rc;
       CK(cudaEventRecord(ev_comp(dep, l), s->stream));
+      l_record(s, ev_comp(dep, l), kStCompute);
     }
   }
   return REMOE_OK;
@@ -396,7 +460,9 @@ int decode_step_batched(remoe_stack* s, const float* hin, float* hout, int32_t* 
 
   CK(launch_route(d, hin, ids, gates, s->contrib, 0, d.L, s->stream));
   s->kernel_launches += 2;
+  l_op(s, kStCompute);
   CK(cudaEventRecord(s->ev_trace, s->stream));      // the route kernel has written the trace to the host mirror
+  l_record(s, s->ev_trace, kStCompute);
 
   BatchArgs a{};
   a.d = d;
@@ -414,12 +480,15 @@ int decode_step_batched(remoe_stack* s, const float* hin, float* hout, int32_t* 
   if (rc != REMOE_OK) return rc;
   CK(launch_batched(s, a));
   s->kernel_launches += 2;
+  const LOp op_res = l_op(s, kStCompute);
   rc = prof_end(s, s->stream);
   if (rc != REMOE_OK) return rc;
   const size_t prof_slot = s->profiling ? s->ev_used.size() - 1 : 0;
   CK(cudaEventRecord(s->ev_resident, s->stream));
+  l_record(s, s->ev_resident, kStCompute);
 
   CK(cudaEventSynchronize(s->ev_trace));
+  l_host_wait(s, s->ev_trace);
   s->steps += 1;
   s->steps_since_reset += 1;
   if (check_device_flag(s) != REMOE_OK) return REMOE_E_DEVICE_FLAG;
@@ -430,12 +499,13 @@ int decode_step_batched(remoe_stack* s, const float* hin, float* hout, int32_t* 
   s->hist_tok_hits.push_back(tk);
 
   uint64_t resident_bytes = 0;
-  rc = batched_waves(s, a, 0, d.L, &resident_bytes);
+  rc = batched_waves(s, a, 0, d.L, &resident_bytes, op_res);
   if (rc != REMOE_OK) return rc;
   if (s->profiling) s->ev_used[prof_slot].bytes = resident_bytes;
   CK(launch_combine_batched(a, hout, 0, d.L, nullptr, s->stream));
   s->kernel_launches += 1;
-  return REMOE_OK;
+  l_op(s, kStCompute);
+  return l_verdict(s);
 }
 
 // Chained step for B > 1: every layer has its own norm -> route -> trace -> waves -> combine round trip,
@@ -463,21 +533,27 @@ int decode_step_chained_batched(remoe_stack* s, const float* hin, float* hout, f
     CK(launch_rmsnorm(s->chain_in + l * rows, s->chain_x + l * rows, d.H, d.B, s->stream));
     CK(launch_route(d, s->chain_x, ids, gates, s->contrib, l, 1, s->stream));
     s->kernel_launches += 3;
+    l_op(s, kStCompute);
     CK(cudaEventRecord(s->ev_trace, s->stream));
+    l_record(s, s->ev_trace, kStCompute);
     a.phase = 0;
     a.layer = l;
     a.depth = 0;
     CK(launch_batched(s, a));
     s->kernel_launches += 2;
+    const LOp op_res = l_op(s, kStCompute);
     CK(cudaEventRecord(s->ev_resident, s->stream));
+    l_record(s, s->ev_resident, kStCompute);
     CK(cudaEventSynchronize(s->ev_trace));
+    l_host_wait(s, s->ev_trace);
     if (check_device_flag(s) != REMOE_OK) return REMOE_E_DEVICE_FLAG;
     trace_totals(s, l, l + 1, &um, &tk);
     uint64_t unused = 0;
-    int rc = batched_waves(s, a, l, l + 1, &unused);
+    int rc = batched_waves(s, a, l, l + 1, &unused, op_res);
     if (rc != REMOE_OK) return rc;
     CK(launch_combine_batched(a, s->chain_out, l, 1, s->chain_in, s->stream));
     s->kernel_launches += 1;
+    l_op(s, kStCompute);
   }
   s->steps += 1;
   s->steps_since_reset += 1;
@@ -487,7 +563,7 @@ int decode_step_chained_batched(remoe_stack* s, const float* hin, float* hout, f
   if (layer_inputs)
     CK(cudaMemcpyAsync(layer_inputs, s->chain_in, rows * d.L * sizeof(float), cudaMemcpyDeviceToDevice,
                        s->stream));
-  return REMOE_OK;
+  return l_verdict(s);
 }
 
 }  // namespace
@@ -505,6 +581,7 @@ const char* remoe_strerror(int code) {
     case REMOE_E_DEVICE_FLAG: return "device-side error flag set";
     case REMOE_E_UNSUPPORTED: return "unsupported shape";
     case REMOE_E_NOMEM: return "out of memory";
+    case REMOE_E_ORDER: return "schedule ordering check failed";
     default: return "unknown error";
   }
 }
@@ -588,6 +665,8 @@ int remoe_stack_create(const remoe_shape* sh, int32_t cache_slots, void* cuda_st
   for (auto& e : s->ev_layer)
     if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return bail(REMOE_E_CUDA);
 
+  if (const char* chk = std::getenv("REMOE_CHECK_ORDER"))
+    if (std::strcmp(chk, "1") == 0) s->ledger.reset(new (std::nothrow) OrderLedger());
   if (const char* inj = std::getenv("REMOE_FAULT_INJECT"))
     s->inject_lost_copy = std::strcmp(inj, "lost_copy") == 0 && sh->batch == 1;
   DevStack& d = s->d;
@@ -754,7 +833,9 @@ int remoe_decode_step(remoe_stack* s, const float* hin, float* hout, int32_t* id
 
   CK(launch_route(d, hin, ids, gates, s->contrib, 0, d.L, s->stream));
   s->kernel_launches += d.B > 1 ? 2 : 1;
+  l_op(s, kStCompute);
   CK(cudaEventRecord(s->ev_trace, s->stream));      // the route kernel has written the trace to the host mirror
+  l_record(s, s->ev_trace, kStCompute);
 
   FfnArgs a{};
   a.d = d;
@@ -777,11 +858,13 @@ int remoe_decode_step(remoe_stack* s, const float* hin, float* hout, int32_t* id
   a.lose_row1 = 0;
   a.spin_limit = 0;
   s->kernel_launches += 1;
+  const LOp op_res = l_op(s, kStCompute);
   rc = prof_end(s, s->stream);
   if (rc != REMOE_OK) return rc;
   const size_t prof_slot = s->profiling ? s->ev_used.size() - 1 : 0;
 
   CK(cudaEventSynchronize(s->ev_trace));
+  l_host_wait(s, s->ev_trace);
   s->steps += 1;
   s->steps_since_reset += 1;
   if (check_device_flag(s) != REMOE_OK) return REMOE_E_DEVICE_FLAG;
@@ -803,7 +886,11 @@ int remoe_decode_step(remoe_stack* s, const float* hin, float* hout, int32_t* id
     int misses = 0;
     for (int k = 0; k < d.K; ++k) {
       const int i = l * s->BK + k;
-      if (t_hit[i]) { resident_bytes += d.slot_bytes; continue; }
+      if (t_hit[i]) {
+        resident_bytes += d.slot_bytes;
+        if (t_slot[i] >= 0 && t_slot[i] < d.C) l_read(s, op_res, slot_cell(s, l, t_slot[i]), "resident-phase launch");
+        continue;
+      }
       const int e = t_req[i], slot = t_slot[i];
       if (e < 0 || e >= d.N || slot < 0 || slot >= d.C) {
         s->cuda_err = "trace holds an expert id or slot out of range (layer " + std::to_string(l) + ")";
@@ -813,23 +900,32 @@ int remoe_decode_step(remoe_stack* s, const float* hin, float* hout, int32_t* id
         // Victim slots may still be read by the previous step's kernels, all of which precede
         // this step's route kernel on the compute stream.
         CK(cudaStreamWaitEvent(s->copy_stream, s->ev_trace, 0));
+        l_wait(s, kStCopy, s->ev_trace);
         copy_ordered = true;
       }
       CK(cudaMemcpyAsync(d.slots + ((size_t)l * d.C + slot) * d.slot_bytes, s->host_ptrs[(size_t)l * d.N + e],
                          d.slot_bytes, cudaMemcpyHostToDevice, s->copy_stream));
+      l_write(s, l_op(s, kStCopy), slot_cell(s, l, slot), "miss fetch");
       ++misses;
     }
     resident_bytes += (uint64_t)d.S * d.shared_bytes;
     if (misses) {
       s->h2d_bytes[l] += (uint64_t)misses * d.slot_bytes;
       CK(cudaEventRecord(s->ev_layer[l], s->copy_stream));
+      l_record(s, s->ev_layer[l], kStCopy);
       CK(cudaStreamWaitEvent(s->stream, s->ev_layer[l], 0));
+      l_wait(s, kStCompute, s->ev_layer[l]);
       a.phase = 1;
       a.layer = l;
       rc = prof_begin(s, s->stream, (uint64_t)misses * d.slot_bytes, 1);
       if (rc != REMOE_OK) return rc;
       CK(launch_ffn_stream(a, s->grid, s->stream));
       s->kernel_launches += 1;
+      if (s->ledger) {
+        const LOp om = l_op(s, kStCompute);
+        for (int k = 0; k < d.K; ++k)
+          if (!t_hit[l * s->BK + k]) l_read(s, om, slot_cell(s, l, t_slot[l * s->BK + k]), "miss-phase launch");
+      }
       rc = prof_end(s, s->stream);
       if (rc != REMOE_OK) return rc;
     }
@@ -837,7 +933,8 @@ int remoe_decode_step(remoe_stack* s, const float* hin, float* hout, int32_t* id
   if (s->profiling) s->ev_used[prof_slot].bytes = resident_bytes;
   CK(launch_combine(a, hout, 0, d.L, nullptr, s->stream));
   s->kernel_launches += 1;
-  return REMOE_OK;
+  l_op(s, kStCompute);
+  return l_verdict(s);
 }
 
 // Second buffer set, route stream and events of remoe_decode_steps.
@@ -896,6 +993,9 @@ int remoe_decode_steps(remoe_stack* s, int32_t n_steps, const float* hin, float*
   CK(cudaEventRecord(s->ev_entry, s->stream));          // everything before the call, the inputs included
   CK(cudaStreamWaitEvent(s->route_stream, s->ev_entry, 0));
   CK(cudaStreamWaitEvent(s->copy_stream, s->ev_entry, 0));
+  l_record(s, s->ev_entry, kStCompute);
+  l_wait(s, kStRoute, s->ev_entry);
+  l_wait(s, kStCopy, s->ev_entry);
 
   auto route = [&](int t) -> int {
     const int p = t & 1;
@@ -904,11 +1004,16 @@ int remoe_decode_steps(remoe_stack* s, int32_t n_steps, const float* hin, float*
     d.trace = dev_blk[p] + 1;
     d.host_mirror = host_blk[p];
     d.shared_scale = scale[p];
-    if (t >= 2) CK(cudaStreamWaitEvent(s->route_stream, s->ev_free2[p], 0));
+    if (t >= 2) {
+      CK(cudaStreamWaitEvent(s->route_stream, s->ev_free2[p], 0));
+      l_wait(s, kStRoute, s->ev_free2[p]);
+    }
     CK(launch_route(d, hin + (size_t)t * io, ids + (size_t)t * kk, gates + (size_t)t * kk, contrib[p], 0, L,
                     s->route_stream));
     s->kernel_launches += 1;
+    l_op(s, kStRoute);
     CK(cudaEventRecord(s->ev_route2[p], s->route_stream));
+    l_record(s, s->ev_route2[p], kStRoute);
     return REMOE_OK;
   };
 
@@ -929,16 +1034,20 @@ int remoe_decode_steps(remoe_stack* s, int32_t n_steps, const float* hin, float*
     a.phase = 0;
     a.layer = -1;
     CK(cudaStreamWaitEvent(s->stream, s->ev_route2[p], 0));
+    l_wait(s, kStCompute, s->ev_route2[p]);
     rc = prof_begin(s, s->stream, 0, 0);
     if (rc != REMOE_OK) return rc;
     CK(launch_ffn_stream(a, s->grid, s->stream));
     s->kernel_launches += 1;
+    const LOp op_res = l_op(s, kStCompute);
     rc = prof_end(s, s->stream);
     if (rc != REMOE_OK) return rc;
     const size_t prof_slot = s->profiling ? s->ev_used.size() - 1 : 0;
     CK(cudaEventRecord(s->ev_res2[p], s->stream));
+    l_record(s, s->ev_res2[p], kStCompute);
 
     CK(cudaEventSynchronize(s->ev_route2[p]));
+    l_host_wait(s, s->ev_route2[p]);
     s->steps += 1;
     if (check_device_flag(s, host_blk[p]) != REMOE_OK) {
       s->steps_since_reset += (uint64_t)t + 1;
@@ -959,7 +1068,11 @@ int remoe_decode_steps(remoe_stack* s, int32_t n_steps, const float* hin, float*
       tk += (uint32_t)t_th[l];
       for (int k = 0; k < K; ++k) {
         const int i = l * K + k;
-        if (t_hit[i]) { resident_bytes += d.slot_bytes; continue; }
+        if (t_hit[i]) {
+          resident_bytes += d.slot_bytes;
+          if (t_slot[i] >= 0 && t_slot[i] < d.C) l_read(s, op_res, slot_cell(s, l, t_slot[i]), "resident-phase launch");
+          continue;
+        }
         const int e = t_req[i], slot = t_slot[i];
         if (e < 0 || e >= d.N || slot < 0 || slot >= d.C) {
           s->cuda_err = "trace holds an expert id or slot out of range (layer " + std::to_string(l) + ")";
@@ -968,10 +1081,15 @@ int remoe_decode_steps(remoe_stack* s, int32_t n_steps, const float* hin, float*
         }
         if (!misses && t > 0) {
           CK(cudaStreamWaitEvent(s->copy_stream, s->ev_res2[q], 0));
-          if (missed[q][l]) CK(cudaStreamWaitEvent(s->copy_stream, s->ev_miss2[(size_t)q * L + l], 0));
+          l_wait(s, kStCopy, s->ev_res2[q]);
+          if (missed[q][l]) {
+            CK(cudaStreamWaitEvent(s->copy_stream, s->ev_miss2[(size_t)q * L + l], 0));
+            l_wait(s, kStCopy, s->ev_miss2[(size_t)q * L + l]);
+          }
         }
         CK(cudaMemcpyAsync(d.slots + ((size_t)l * d.C + slot) * d.slot_bytes, s->host_ptrs[(size_t)l * d.N + e],
                            d.slot_bytes, cudaMemcpyHostToDevice, s->copy_stream));
+        l_write(s, l_op(s, kStCopy), slot_cell(s, l, slot), "miss fetch");
         ++misses;
       }
       resident_bytes += (uint64_t)d.S * d.shared_bytes;
@@ -980,35 +1098,46 @@ int remoe_decode_steps(remoe_stack* s, int32_t n_steps, const float* hin, float*
       if (!misses) continue;
       s->h2d_bytes[l] += (uint64_t)misses * d.slot_bytes;
       CK(cudaEventRecord(s->ev_copy2[(size_t)p * L + l], s->copy_stream));
+      l_record(s, s->ev_copy2[(size_t)p * L + l], kStCopy);
       CK(cudaStreamWaitEvent(s->stream, s->ev_copy2[(size_t)p * L + l], 0));
+      l_wait(s, kStCompute, s->ev_copy2[(size_t)p * L + l]);
       a.phase = 1;
       a.layer = l;
       rc = prof_begin(s, s->stream, (uint64_t)misses * d.slot_bytes, 1);
       if (rc != REMOE_OK) return rc;
       CK(launch_ffn_stream(a, s->grid, s->stream));
       s->kernel_launches += 1;
+      if (s->ledger) {
+        const LOp om = l_op(s, kStCompute);
+        for (int k = 0; k < K; ++k)
+          if (!t_hit[l * K + k]) l_read(s, om, slot_cell(s, l, t_slot[l * K + k]), "miss-phase launch");
+      }
       rc = prof_end(s, s->stream);
       if (rc != REMOE_OK) return rc;
       CK(cudaEventRecord(s->ev_miss2[(size_t)p * L + l], s->stream));
+      l_record(s, s->ev_miss2[(size_t)p * L + l], kStCompute);
     }
     if (s->profiling) s->ev_used[prof_slot].bytes = resident_bytes;
     s->hist_umiss.push_back(um);
     s->hist_tok_hits.push_back(tk);
     CK(launch_combine(a, hout + (size_t)t * io, 0, L, nullptr, s->stream));
     s->kernel_launches += 1;
+    l_op(s, kStCompute);
     CK(cudaEventRecord(s->ev_free2[p], s->stream));
+    l_record(s, s->ev_free2[p], kStCompute);
   }
   s->steps_since_reset += (uint64_t)n_steps;
   // Later calls use buffer set 0 and the stack's stream: leave the copy stream behind this call's last
   // readers, and the device trace of the last step where remoe_last_step_trace looks for it.
   CK(cudaStreamWaitEvent(s->copy_stream, s->ev_free2[(n_steps - 1) & 1], 0));
+  l_wait(s, kStCopy, s->ev_free2[(n_steps - 1) & 1]);
   if ((n_steps - 1) & 1) {
     CK(cudaMemcpyAsync(s->dev_block + 1, s->dev_block2 + 1, (s->block_ints - 1) * sizeof(int),
                        cudaMemcpyDeviceToDevice, s->stream));
     CK(cudaMemcpyAsync(s->d.shared_scale, s->shared_scale2, (size_t)L * base.B * sizeof(float),
                        cudaMemcpyDeviceToDevice, s->stream));
   }
-  return REMOE_OK;
+  return l_verdict(s);
 }
 
 int remoe_decode_step_chained(remoe_stack* s, const float* hin, float* hout, float* layer_inputs, int32_t* ids,
@@ -1038,12 +1167,16 @@ int remoe_decode_step_chained(remoe_stack* s, const float* hin, float* hout, flo
     CK(launch_rmsnorm(s->chain_in + (size_t)l * d.H, s->chain_x + (size_t)l * d.H, d.H, 1, s->stream));
     CK(launch_route(d, s->chain_x, ids, gates, s->contrib, l, 1, s->stream));
     s->kernel_launches += 1;
+    l_op(s, kStCompute);
     CK(cudaEventRecord(s->ev_trace, s->stream));
+    l_record(s, s->ev_trace, kStCompute);
     a.phase = 0;
     a.layer = l;
     CK(launch_ffn_stream(a, s->grid, s->stream));
     s->kernel_launches += 2;
+    const LOp op_res = l_op(s, kStCompute);
     CK(cudaEventSynchronize(s->ev_trace));
+    l_host_wait(s, s->ev_trace);
     if (check_device_flag(s) != REMOE_OK) return REMOE_E_DEVICE_FLAG;
     int* tr = s->host_block + 1;
     const int* t_req = trace_requests(tr, d.L, s->BK);
@@ -1053,28 +1186,43 @@ int remoe_decode_step_chained(remoe_stack* s, const float* hin, float* hout, flo
     int misses = 0;
     for (int k = 0; k < d.K; ++k) {
       const int i = l * s->BK + k;
-      if (t_hit[i]) continue;
+      if (t_hit[i]) {
+        if (t_slot[i] >= 0 && t_slot[i] < d.C) l_read(s, op_res, slot_cell(s, l, t_slot[i]), "resident-phase launch");
+        continue;
+      }
       const int e = t_req[i], slot = t_slot[i];
       if (e < 0 || e >= d.N || slot < 0 || slot >= d.C) {
         s->cuda_err = "trace holds an expert id or slot out of range (layer " + std::to_string(l) + ")";
         return REMOE_E_DEVICE_FLAG;
       }
-      if (!misses) CK(cudaStreamWaitEvent(s->copy_stream, s->ev_trace, 0));
+      if (!misses) {
+        CK(cudaStreamWaitEvent(s->copy_stream, s->ev_trace, 0));
+        l_wait(s, kStCopy, s->ev_trace);
+      }
       CK(cudaMemcpyAsync(d.slots + ((size_t)l * d.C + slot) * d.slot_bytes, s->host_ptrs[(size_t)l * d.N + e],
                          d.slot_bytes, cudaMemcpyHostToDevice, s->copy_stream));
+      l_write(s, l_op(s, kStCopy), slot_cell(s, l, slot), "miss fetch");
       ++misses;
     }
     um += (uint32_t)misses;
     if (misses) {
       s->h2d_bytes[l] += (uint64_t)misses * d.slot_bytes;
       CK(cudaEventRecord(s->ev_layer[l], s->copy_stream));
+      l_record(s, s->ev_layer[l], kStCopy);
       CK(cudaStreamWaitEvent(s->stream, s->ev_layer[l], 0));
+      l_wait(s, kStCompute, s->ev_layer[l]);
       a.phase = 1;
       CK(launch_ffn_stream(a, s->grid, s->stream));
       s->kernel_launches += 1;
+      if (s->ledger) {
+        const LOp om = l_op(s, kStCompute);
+        for (int k = 0; k < d.K; ++k)
+          if (!t_hit[l * s->BK + k]) l_read(s, om, slot_cell(s, l, t_slot[l * s->BK + k]), "miss-phase launch");
+      }
     }
     CK(launch_combine(a, s->chain_out, l, 1, s->chain_in, s->stream));
     s->kernel_launches += 1;
+    l_op(s, kStCompute);
   }
   s->steps += 1;
   s->steps_since_reset += 1;
@@ -1083,7 +1231,7 @@ int remoe_decode_step_chained(remoe_stack* s, const float* hin, float* hout, flo
   CK(cudaMemcpyAsync(hout, s->chain_in + (size_t)d.L * d.H, row, cudaMemcpyDeviceToDevice, s->stream));
   if (layer_inputs)
     CK(cudaMemcpyAsync(layer_inputs, s->chain_in, row * d.L, cudaMemcpyDeviceToDevice, s->stream));
-  return REMOE_OK;
+  return l_verdict(s);
 }
 
 int remoe_decode_step_host(remoe_stack* s, const float* hin, float* hout, int32_t* ids, float* gates) {
@@ -1268,6 +1416,8 @@ int remoe_cache_reset(remoe_stack* s) {
   ON_STACK_DEVICE(s);
   CK(cudaStreamSynchronize(s->stream));
   CK(cudaStreamSynchronize(s->copy_stream));
+  l_host_sync(s, kStCompute);
+  l_host_sync(s, kStCopy);
   return reset_state(s);
 }
 
@@ -1305,6 +1455,13 @@ int remoe_kernel_time(remoe_stack* s, int32_t phase, double* ms_sum, uint64_t* l
   if (ms_sum) *ms_sum = s->prof_ms[phase];
   if (launches) *launches = s->prof_launches[phase];
   if (bytes) *bytes = s->prof_bytes[phase];
+  return REMOE_OK;
+}
+
+int remoe_order_check_counts(remoe_stack* s, uint64_t* comparisons, uint64_t* violations) {
+  if (!s) return REMOE_E_ARG;
+  if (comparisons) *comparisons = s->ledger ? s->ledger->checks() : 0;
+  if (violations) *violations = s->ledger ? s->ledger->violations() : 0;
   return REMOE_OK;
 }
 

@@ -249,6 +249,60 @@ def test_wait_that_runs_out_is_reported_and_reset_restores_service(monkeypatch, 
         wl.close()
 
 
+def test_schedule_order_checker_on_every_path(monkeypatch):
+    """REMOE_CHECK_ORDER=1: the host-side ledger replays every launch, copy, event record and wait of the
+    scheduler and checks each slot write against the slot's earlier readers and each read against the
+    write that filled it.  Single steps, the multi-step call (routes ahead on a third stream), the chained
+    step and both batched schedules (copies straight into slots; copies into the staging pool) run under
+    it at cache sizes that evict all the time; a call that enqueued an unordered access would return
+    REMOE_E_ORDER (and the binding would raise)."""
+    import torch
+    from paper_2605_27081_b200.loader import LoadedWorkload
+
+    monkeypatch.setenv("REMOE_CHECK_ORDER", "1")
+
+    def drive(shape, c, steps, mode):
+        wl = LoadedWorkload(shape, c, seed=31)
+        try:
+            L, B, H, K = shape.n_layers, shape.batch, shape.hidden, shape.top_k
+            hid = torch.from_numpy(synth.HiddenStream(31, shape, 0.3).take(steps)).to("cuda")
+            out = torch.empty((steps, L, B, H), device="cuda")
+            ids = torch.empty((steps, L, B, K), dtype=torch.int32, device="cuda")
+            g = torch.empty((steps, L, B, K), device="cuda")
+            if mode == "multi":
+                wl.stack.decode_steps(steps // 2, hid, out, ids, g)
+                wl.stack.decode_step(hid[steps // 2], out[0], ids[0], g[0])       # back to the single-step path
+                wl.stack.decode_steps(steps - steps // 2 - 1, hid[steps // 2 + 1:], out, ids, g)
+            elif mode == "chained":
+                fin = torch.empty((B, H), device="cuda")
+                for t in range(steps):
+                    wl.stack.decode_step_chained(hid[t, 0], fin, None, ids[0], g[0])
+            else:
+                for t in range(steps):
+                    wl.stack.decode_step(hid[t], out[t], ids[t], g[t])
+            torch.cuda.synchronize()
+            compared, bad = wl.stack.order_check_counts()
+            assert bad == 0 and compared > 10 * steps, (mode, compared, bad)
+            assert wl.stack.cache_stats()["uniq_misses"] > steps
+        finally:
+            wl.close()
+
+    b1 = synth.Shape(4, 256, 16, 3, 24, 1, 8, 0, 0, 1, 1)
+    drive(b1, 3, 40, "single")                      # C = K: every slot may be replaced at every step
+    drive(b1, 4, 41, "multi")
+    drive(b1, 3, 20, "chained")
+    drive(synth.Shape(3, 256, 16, 2, 40, 1, 24, 0, 0, 1, 6), 5, 20, "single")     # batched, mma.sync kernel: copies into slots
+    drive(synth.Shape(3, 512, 24, 3, 64, 1, 64, 0, 0, 1, 12), 8, 20, "single")    # batched, tcgen05 kernel: staging pool
+    drive(synth.Shape(3, 512, 24, 3, 64, 1, 64, 0, 0, 2, 12), 8, 12, "single")    # the same over an FP8 store
+    drive(synth.Shape(3, 512, 24, 3, 64, 1, 64, 0, 0, 1, 12), 8, 8, "chained")
+    monkeypatch.delenv("REMOE_CHECK_ORDER")
+    wl = LoadedWorkload(b1, 3, seed=31)
+    try:
+        assert wl.stack.order_check_counts() == (0, 0)              # off unless asked for
+    finally:
+        wl.close()
+
+
 def test_policy_switch_and_second_stack_share_a_store():
     """Two stacks over the same pinned store (different capacity and policy) stay independent."""
     import torch
