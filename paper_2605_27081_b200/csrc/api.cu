@@ -51,6 +51,7 @@ struct remoe_stack {
   float* chain_in = nullptr;               // [L + 1][H] residual stream h_l of the chained mode
   float* chain_x = nullptr;                // [L][H] normalised layer inputs x_l = rmsnorm(h_l)
   float* chain_out = nullptr;              // [L][H] per-layer MoE outputs of the chained mode
+  unsigned* link_ticket = nullptr;         // ticket word of the chained step's link kernel
   cudaEvent_t ev_trace = nullptr;
   std::vector<cudaEvent_t> ev_layer;
   // second set of per-step buffers and the streams/events of the multi-step entry point, which routes
@@ -715,6 +716,8 @@ int remoe_stack_create(const remoe_shape* sh, int32_t cache_slots, void* cuda_st
   TRY(dev_alloc(s, &s->chain_in, (L + 1) * d.B * d.H));
   TRY(dev_alloc(s, &s->chain_out, L * d.B * d.H));
   TRY(dev_alloc(s, &s->chain_x, L * d.B * d.H));
+  TRY(dev_alloc(s, &s->link_ticket, 1));
+  if (cudaMemset(s->link_ticket, 0, sizeof(unsigned)) != cudaSuccess) return bail(REMOE_E_CUDA);
   if (d.B > 1) {
     if (!ffn_batched_supported(d)) return bail(REMOE_E_UNSUPPORTED);
     const size_t P = d.K + d.S;
@@ -1161,19 +1164,19 @@ int remoe_decode_step_chained(remoe_stack* s, const float* hin, float* hout, flo
   a.contrib = s->contrib;
   a.grid_cap = s->grid;
   uint32_t um = 0, tk = 0;
+  // The layer's input exists only once the previous layer is done, so every layer has its own
+  // norm -> route -> trace -> fetch -> compute round trip.  The link kernel joins two layers in one
+  // launch: sum of the upper layer's partials, residual add, pre-norm and routing of the lower layer.
+  CK(launch_chain_link(d, a, 0, s->chain_in, s->chain_out, s->chain_x, s->link_ticket, 0, 1, ids, gates, s->stream));
+  s->kernel_launches += 1;
   for (int l = 0; l < d.L; ++l) {
-    // The layer's input exists only once the previous layer is done, so every layer has its own
-    // norm -> route -> trace -> fetch -> compute round trip.
-    CK(launch_rmsnorm(s->chain_in + (size_t)l * d.H, s->chain_x + (size_t)l * d.H, d.H, 1, s->stream));
-    CK(launch_route(d, s->chain_x, ids, gates, s->contrib, l, 1, s->stream));
-    s->kernel_launches += 1;
     l_op(s, kStCompute);
     CK(cudaEventRecord(s->ev_trace, s->stream));
     l_record(s, s->ev_trace, kStCompute);
     a.phase = 0;
     a.layer = l;
     CK(launch_ffn_stream(a, s->grid, s->stream));
-    s->kernel_launches += 2;
+    s->kernel_launches += 1;
     const LOp op_res = l_op(s, kStCompute);
     CK(cudaEventSynchronize(s->ev_trace));
     l_host_wait(s, s->ev_trace);
@@ -1220,10 +1223,12 @@ int remoe_decode_step_chained(remoe_stack* s, const float* hin, float* hout, flo
           if (!t_hit[l * s->BK + k]) l_read(s, om, slot_cell(s, l, t_slot[l * s->BK + k]), "miss-phase launch");
       }
     }
-    CK(launch_combine(a, s->chain_out, l, 1, s->chain_in, s->stream));
+    // the link also reads the contributor table the miss-phase launch (if any) has just completed
+    CK(launch_chain_link(d, a, l + 1, s->chain_in, s->chain_out, s->chain_x, s->link_ticket, 1, l + 1 < d.L ? 1 : 0, ids,
+                         gates, s->stream));
     s->kernel_launches += 1;
-    l_op(s, kStCompute);
   }
+  l_op(s, kStCompute);
   s->steps += 1;
   s->steps_since_reset += 1;
   s->hist_umiss.push_back(um);

@@ -11,8 +11,8 @@
 // on the caller's stream.  The price is a fixed ceiling on the problem size and one shared
 // scratch area per device.
 //
-// It is a variant of the expert-streaming kernel of ffn_stream.cu (same channel-major expert
-// block, same bulk-copy stage ring, same warp-per-triple arithmetic), restricted to one layer
+// It runs the same per-CTA body as the stack's expert-streaming kernel (ffn_stream_body.cuh: channel-major
+// expert block, bulk-copy stage ring fed by four producer lanes, warp-per-triple arithmetic), for one layer
 // whose experts are given directly as device pointers.
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -20,13 +20,13 @@
 #include <mutex>
 
 #include "remoe.h"
-#include "tma_ring.cuh"
+#include "ffn_stream_body.cuh"
 
 namespace {
 
-constexpr int kConsumerWarps = 8;
-constexpr int kThreads = (kConsumerWarps + 1) * 32;
-constexpr int kStages = 16;                                 // multiple of kConsumerWarps
+using remoe::stream::kConsumerWarps;
+using remoe::stream::kThreads;
+constexpr int kStages = remoe::stream::kMaxStages;
 constexpr int kMaxCtas = 160;                               // scratch rows; grids are capped to this
 constexpr int kMaxDevices = 64;
 
@@ -55,25 +55,30 @@ constexpr size_t smem_bytes() {
          (size_t)kStages * 3 * H * WB;
 }
 
+// One layer, experts given as pointers; one partial row per CTA in the fixed scratch array.  There is no
+// error word to report through without allocating one, so a wait that ran out poisons the CTA's partial:
+// the caller sees NaN in the output instead of a wrong number.
+template <int H>
+struct StaticWork {
+  static constexpr bool kPoison = true;
+  const StaticArgs& a;
+  __device__ __forceinline__ const char* base(int pair, bool&) const { return a.base[pair]; }
+  __device__ __forceinline__ float scale(int pair, int) const { return a.scale[pair]; }
+  __device__ __forceinline__ const float* hidden(int) const { return a.hidden_in; }
+  __device__ __forceinline__ float* partial(int) const { return a.partial + (size_t)blockIdx.x * H; }
+  __device__ __forceinline__ void fail(int) const {}
+};
+
 template <int WB, int H>
 __global__ void __launch_bounds__(kThreads, 1) ffn_static_kernel(const __grid_constant__ StaticArgs a) {
-  using E = Elems<WB>;
-  constexpr int kVec = E::kVec;
-  constexpr int kIter = H / (32 * kVec);
-  constexpr int kCols = kIter * kVec;
-  constexpr int kPassCols = 32 * kVec;
-  constexpr uint32_t kStageBytes = 3u * H * WB;
-  constexpr uint32_t kRowBytes = (uint32_t)H * WB;
-
   extern __shared__ __align__(128) unsigned char smem[];
   uint64_t* full = reinterpret_cast<uint64_t*>(smem);
   uint64_t* empty = full + kStages;
   float* red = reinterpret_cast<float*>(smem + 2 * kStages * sizeof(uint64_t));
-  unsigned char* stages = reinterpret_cast<unsigned char*>(red + kConsumerWarps * kPassCols);
+  unsigned char* stages = reinterpret_cast<unsigned char*>(red + kConsumerWarps * 32 * Elems<WB>::kVec);
   __shared__ int s_abort;
 
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  if (tid == 0) {
+  if (threadIdx.x == 0) {
     s_abort = 0;
     for (int s = 0; s < kStages; ++s) { mbar_init(full + s, 1); mbar_init(empty + s, 1); }
     mbar_fence_init();
@@ -84,106 +89,10 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_static_kernel(const __grid_co
   const int r0 = min(M, (int)blockIdx.x * a.rows_per_cta), r1 = min(M, r0 + a.rows_per_cta);
   if (r0 >= r1) return;
 
-  if (warp == kConsumerWarps) {
-    // producer: one thread streams this CTA's channel triples into the stage ring
-    if (lane == 0) {
-      int e = 0, issued = 0;
-      bool ok = true;
-      for (int r = r0; r < r1; ++r, ++issued) {
-        while (a.prefix[e + 1] <= r) ++e;
-        const int n = r - r0, s = n % kStages;
-        if (n >= kStages &&
-            (*(volatile int*)&s_abort || !mbar_wait(empty + s, ((n / kStages) - 1) & 1))) { ok = false; break; }
-        mbar_expect_tx(full + s, kStageBytes);
-        bulk_g2s(stages + (size_t)s * kStageBytes, a.base[e] + (size_t)(r - a.prefix[e]) * kStageBytes,
-                 kStageBytes, full + s);
-      }
-      if (!ok) {
-        // let the consumers leave, then wait (bounded) for copies that are still landing
-        atomicExch(&s_abort, 1);
-        for (int n = max(0, issued - kStages); n < issued; ++n) mbar_wait(full + (n % kStages), (n / kStages) & 1);
-      }
-    }
-    return;
-  }
-
-  float hreg[kCols], acc[kCols];
-#pragma unroll
-  for (int it = 0; it < kIter; ++it)
-#pragma unroll
-    for (int v4 = 0; v4 < kVec / 4; ++v4) {
-      const float4 x = __ldg(reinterpret_cast<const float4*>(a.hidden_in + (it * 32 + lane) * kVec) + v4);
-      hreg[it * kVec + v4 * 4 + 0] = x.x; hreg[it * kVec + v4 * 4 + 1] = x.y;
-      hreg[it * kVec + v4 * 4 + 2] = x.z; hreg[it * kVec + v4 * 4 + 3] = x.w;
-    }
-#pragma unroll
-  for (int c = 0; c < kCols; ++c) acc[c] = 0.f;
-
-  int e = 0;
-  for (int r = r0 + warp; r < r1; r += kConsumerWarps) {
-    while (a.prefix[e + 1] <= r) ++e;
-    const float scale = a.scale[e];
-    const int n = r - r0, s = n % kStages;
-    // decided for the whole warp: the shuffles below need every lane
-    if (__any_sync(kFull, *(volatile int*)&s_abort || !mbar_wait(full + s, (n / kStages) & 1))) {
-      // A wait that ran out: there is no flag word to report through without allocating, so
-      // poison this CTA's partial; the caller sees NaN in the output instead of a wrong number.
-      atomicExch(&s_abort, 1);
-#pragma unroll
-      for (int c = 0; c < kCols; ++c) acc[c] = __int_as_float(0x7fc00000);
-      break;
-    }
-    const char* st = reinterpret_cast<const char*>(stages) + (size_t)s * kStageBytes;
-    float g = 0.f, u = 0.f;
-#pragma unroll
-    for (int it = 0; it < kIter; ++it) {
-      float w[kVec];
-      E::load(st + (it * 32 + lane) * 16, w);
-#pragma unroll
-      for (int j = 0; j < kVec; ++j) g = fmaf(w[j], hreg[it * kVec + j], g);
-    }
-#pragma unroll
-    for (int it = 0; it < kIter; ++it) {
-      float w[kVec];
-      E::load(st + kRowBytes + (it * 32 + lane) * 16, w);
-#pragma unroll
-      for (int j = 0; j < kVec; ++j) u = fmaf(w[j], hreg[it * kVec + j], u);
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      g += __shfl_xor_sync(kFull, g, o);
-      u += __shfl_xor_sync(kFull, u, o);
-    }
-    const float av = g / (1.f + __expf(-g)) * u * scale;
-#pragma unroll
-    for (int it = 0; it < kIter; ++it) {
-      float w[kVec];
-      E::load(st + 2 * kRowBytes + (it * 32 + lane) * 16, w);
-#pragma unroll
-      for (int j = 0; j < kVec; ++j) acc[it * kVec + j] = fmaf(av, w[j], acc[it * kVec + j]);
-    }
-    __syncwarp();
-    if (lane == 0) mbar_arrive(empty + s);
-  }
-
-  // add the eight warps' private sums in warp order and write this CTA's row of the scratch
-  float* dst = a.partial + (size_t)blockIdx.x * H;
-#pragma unroll
-  for (int it = 0; it < kIter; ++it) {
-    float* mine = red + (size_t)warp * kPassCols + lane * kVec;
-#pragma unroll
-    for (int v4 = 0; v4 < kVec / 4; ++v4)
-      *reinterpret_cast<float4*>(mine + v4 * 4) = make_float4(
-          acc[it * kVec + v4 * 4], acc[it * kVec + v4 * 4 + 1], acc[it * kVec + v4 * 4 + 2], acc[it * kVec + v4 * 4 + 3]);
-    consumer_bar();
-    if (tid < kPassCols) {
-      float t = 0.f;
-#pragma unroll
-      for (int w = 0; w < kConsumerWarps; ++w) t += red[(size_t)w * kPassCols + tid];
-      dst[it * kPassCols + tid] = t;
-    }
-    consumer_bar();
-  }
+  const remoe::stream::Ring ring{full, empty, red, stages, kStages, &s_abort};
+  const StaticWork<H> wk{a};
+  // all experts form one "layer" of n_experts pairs
+  remoe::stream::stream_rows<WB, H>(wk, a.prefix, a.n_experts, r0, r1, ring, kSpinLimit, 0);
 }
 
 __global__ void __launch_bounds__(256) combine_static_kernel(const float* __restrict__ partial, int n_active, int H,

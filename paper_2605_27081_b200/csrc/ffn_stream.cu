@@ -21,22 +21,18 @@
 // atomics are used.  HBM traffic is the weight bytes once plus O(grid * H) partials.
 #include "remoe_internal.cuh"
 #include "tma_ring.cuh"
+#include "ffn_stream_body.cuh"
 
 namespace remoe {
 
 namespace {
 
-constexpr int kConsumerWarps = 8;
-constexpr int kThreads = (kConsumerWarps + 1) * 32;
-constexpr int kMaxStages = 16;                 // multiple of kConsumerWarps
-constexpr int kProducerLanes = 4;              // divides kConsumerWarps, hence every ring depth
 using namespace ring;
+using stream::kConsumerWarps;
+using stream::kMaxStages;
+using stream::kThreads;
 
 // Shared-memory carve-up (dynamic): barriers | row prefix table | reduce buffer | stage ring.
-// The ring depth is a multiple of the consumer-warp count, so a stage is always consumed by
-// the same warp.  That warp has waited for fill k-1 of the stage before it waits for fill k,
-// hence the barrier can never be a whole phase behind the parity it is asked about (a parity
-// wait cannot tell "phase k done" from "phase k-2 done").
 struct Layout {
   size_t bars, prefix, red, stages, total;
   int n_stages;
@@ -69,30 +65,45 @@ __device__ __forceinline__ int pair_rows(const FfnArgs& a, int pair) {
   return hit ? 0 : d.I;
 }
 
+// Where a stack launch finds its rows and puts its partials: routed experts in the cache slots the step
+// trace names, shared experts in their resident blocks; one partial per (phase, layer, CTA).
+template <int H>
+struct StackWork {
+  static constexpr bool kPoison = false;
+  const FfnArgs& a;
+  const int* t_slot;
+  __device__ __forceinline__ const char* base(int pair, bool& ok) const {
+    const DevStack& d = a.d;
+    const int P = d.K + d.S, l = pair / P, p = pair % P;
+    if (p >= d.K) return d.shared_blocks + ((size_t)l * d.S + (p - d.K)) * d.shared_bytes;
+    const int slot = t_slot[l * d.K + p];
+    if (slot < 0 || slot >= d.C) { atomicCAS(d.err, kErrNone, kErrBadIndex); ok = false; return nullptr; }
+    return d.slots + ((size_t)l * d.C + slot) * d.slot_bytes;
+  }
+  __device__ __forceinline__ float scale(int pair, int l) const {
+    const int p = pair % (a.d.K + a.d.S);
+    return p < a.d.K ? a.gates[l * a.d.K + p] : a.d.shared_scale[l];
+  }
+  __device__ __forceinline__ const float* hidden(int l) const { return a.hidden_in + (size_t)l * H; }
+  __device__ __forceinline__ float* partial(int l) const {
+    return a.partial + (((size_t)a.phase * a.d.L + l) * a.grid_cap + blockIdx.x) * H;
+  }
+  __device__ __forceinline__ void fail(int code) const { atomicCAS(a.d.err, kErrNone, code); }
+};
+
 template <int WB, int H>
 __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(const __grid_constant__ FfnArgs a) {
-  using E = Elems<WB>;
-  constexpr int kVec = E::kVec;
-  constexpr int kIter = H / (32 * kVec);
-  constexpr int kCols = kIter * kVec;                  // columns of h / out owned by one lane
-  constexpr uint32_t kRowBytes = (uint32_t)weight_row_bytes(H, WB);
-  constexpr uint32_t kStageBytes = 3u * kRowBytes;
-  constexpr bool kGrouped = WB == 0;                   // per-group scales follow the codes of a row
-
   extern __shared__ __align__(128) unsigned char smem[];
   const Layout lay = make_layout(H, WB);
   uint64_t* full = reinterpret_cast<uint64_t*>(smem + lay.bars);
   uint64_t* empty = full + kMaxStages;
   int* prefix = reinterpret_cast<int*>(smem + lay.prefix);
-  float* red = reinterpret_cast<float*>(smem + lay.red);
-  unsigned char* stages = smem + lay.stages;
   const int NS = lay.n_stages;
   __shared__ int s_abort;
 
   const DevStack& d = a.d;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int P = d.K + d.S, n_pairs = d.L * P;
-  const unsigned spin = a.spin_limit ? a.spin_limit : kSpinLimit;
 
   // Work table: exclusive prefix of rows per pair.
   for (int i = tid; i < n_pairs; i += kThreads) prefix[i + 1] = pair_rows(a, i);
@@ -119,6 +130,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(const __grid_co
   }
   __syncthreads();
 
+  // The row list of the launch is cut into equal contiguous ranges, one per CTA.
   const int M = prefix[n_pairs];
   const int G = gridDim.x;
   const int q = (M + G - 1) / G;                       // rows per CTA
@@ -134,180 +146,9 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(const __grid_co
   }
   if (r0 >= r1) return;
 
-  const int* t_slot = trace_slot(d.trace, d.L, d.K);
-
-  if (warp == kConsumerWarps) {
-    // ------------------------------------------------------------------ producer
-    // Issuing one copy (free-stage wait, expect_tx, bulk copy) is a chain of a few hundred cycles for one
-    // thread; with small stages (FP8, narrow H) a single issuer cannot keep the ring full, so a few
-    // lanes issue side by side, lane j taking the rows whose local index is j modulo kProducerLanes.
-    if (lane < kProducerLanes) {
-      int pair = 0;
-      const char* base = nullptr;
-      int pair_of_base = -1;
-      int issued = lane;                             // local index after this lane's last issued row
-      bool ok = true;
-      for (int r = r0 + lane; r < r1 && ok; r += kProducerLanes, issued += kProducerLanes) {
-        while (prefix[pair + 1] <= r) ++pair;
-        if (pair != pair_of_base) {
-          const int l = pair / P, p = pair % P;
-          if (p < d.K) {
-            const int slot = t_slot[l * d.K + p];
-            if (slot < 0 || slot >= d.C) { atomicCAS(d.err, kErrNone, kErrBadIndex); ok = false; break; }
-            base = d.slots + ((size_t)l * d.C + slot) * d.slot_bytes;
-          } else {
-            base = d.shared_blocks + ((size_t)l * d.S + (p - d.K)) * d.shared_bytes;
-          }
-          pair_of_base = pair;
-        }
-        const int i = r - prefix[pair];
-        const int n = r - r0, s = n % NS;
-        if (n >= NS) {
-          if (*(volatile int*)&s_abort) { ok = false; break; }
-          if (!mbar_wait(empty + s, ((n / NS) - 1) & 1, spin)) {
-            atomicCAS(d.err, kErrNone, kErrWaitEmpty);
-            ok = false;
-            break;
-          }
-        }
-        if (r + 1 == a.lose_row1) continue;                // test aid: this stage is never filled
-        mbar_expect_tx(full + s, kStageBytes);
-        bulk_g2s(stages + (size_t)s * kStageBytes, base + (size_t)i * kStageBytes, kStageBytes, full + s);
-      }
-      if (!ok || *(volatile int*)&s_abort) {
-        // Let the consumers leave, then wait (bounded) for copies that are still landing.
-        atomicExch(&s_abort, 1);
-        for (int n = issued - kProducerLanes; n >= 0 && n >= issued - NS; n -= kProducerLanes)
-          if (!mbar_wait(full + (n % NS), (n / NS) & 1, spin)) atomicCAS(d.err, kErrNone, kErrDrain);
-      }
-    }
-  } else {
-    // ----------------------------------------------------------------- consumers
-    float hreg[kCols], acc[kCols];
-    int pair = 0;
-    while (prefix[pair + 1] <= r0) ++pair;
-    int l_first = pair / P;
-    int pair_last = pair;
-    while (prefix[pair_last + 1] < r1) ++pair_last;
-    const int l_last = pair_last / P;
-    bool aborted = false;
-
-    for (int l = l_first; l <= l_last; ++l) {
-      const int lo = max(r0, prefix[l * P]), hi = min(r1, prefix[(l + 1) * P]);
-      if (lo >= hi) continue;
-      const float* h = a.hidden_in + (size_t)l * H;
-#pragma unroll
-      for (int it = 0; it < kIter; ++it) {
-#pragma unroll
-        for (int v4 = 0; v4 < kVec / 4; ++v4) {
-          const float4 x = __ldg(reinterpret_cast<const float4*>(h + (it * 32 + lane) * kVec) + v4);
-          hreg[it * kVec + v4 * 4 + 0] = x.x;
-          hreg[it * kVec + v4 * 4 + 1] = x.y;
-          hreg[it * kVec + v4 * 4 + 2] = x.z;
-          hreg[it * kVec + v4 * 4 + 3] = x.w;
-        }
-      }
-#pragma unroll
-      for (int c = 0; c < kCols; ++c) acc[c] = 0.f;
-
-      // first row of this layer handled by this warp: local index n = r - r0 with n % 8 == warp
-      int r = lo + ((warp - (lo - r0)) % kConsumerWarps + kConsumerWarps) % kConsumerWarps;
-      float scale = 0.f;
-      int pair_of_scale = -1;
-      for (; r < hi && !aborted; r += kConsumerWarps) {
-        while (prefix[pair + 1] <= r) ++pair;
-        if (pair != pair_of_scale) {
-          const int p = pair % P;
-          scale = p < d.K ? a.gates[l * d.K + p] : d.shared_scale[l];
-          pair_of_scale = pair;
-        }
-        const int n = r - r0, s = n % NS;
-        // decided for the whole warp: the shuffles below need every lane
-        if (__any_sync(kFull, *(volatile int*)&s_abort || !mbar_wait(full + s, (n / NS) & 1, spin))) {
-          if (!*(volatile int*)&s_abort) { atomicCAS(d.err, kErrNone, kErrWaitFull); atomicExch(&s_abort, 1); }
-          aborted = true;
-          break;
-        }
-        const char* st = reinterpret_cast<const char*>(stages) + (size_t)s * kStageBytes;
-        float g = 0.f, u = 0.f;
-        float gs[kGrouped ? kIter : 1];                  // grouped format: this lane's group scales of the third row
-        if constexpr (kGrouped) {
-#pragma unroll
-          for (int it = 0; it < kIter; ++it) {
-            float w[kVec], t = 0.f;
-            E::load(st + (it * 32 + lane) * 16, w);
-#pragma unroll
-            for (int j = 0; j < kVec; ++j) t = fmaf(w[j], hreg[it * kVec + j], t);
-            g = fmaf(E::scale(st, H, it * 32 + lane), t, g);
-          }
-#pragma unroll
-          for (int it = 0; it < kIter; ++it) {
-            float w[kVec], t = 0.f;
-            E::load(st + kRowBytes + (it * 32 + lane) * 16, w);
-#pragma unroll
-            for (int j = 0; j < kVec; ++j) t = fmaf(w[j], hreg[it * kVec + j], t);
-            u = fmaf(E::scale(st + kRowBytes, H, it * 32 + lane), t, u);
-            gs[it] = E::scale(st + 2 * kRowBytes, H, it * 32 + lane);
-          }
-        } else {
-#pragma unroll
-          for (int it = 0; it < kIter; ++it) {
-            float w[kVec];
-            E::load(st + (it * 32 + lane) * 16, w);
-#pragma unroll
-            for (int j = 0; j < kVec; ++j) g = fmaf(w[j], hreg[it * kVec + j], g);
-          }
-#pragma unroll
-          for (int it = 0; it < kIter; ++it) {
-            float w[kVec];
-            E::load(st + kRowBytes + (it * 32 + lane) * 16, w);
-#pragma unroll
-            for (int j = 0; j < kVec; ++j) u = fmaf(w[j], hreg[it * kVec + j], u);
-          }
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-          g += __shfl_xor_sync(kFull, g, o);
-          u += __shfl_xor_sync(kFull, u, o);
-        }
-        g *= WScale<WB>::kDot;
-        u *= WScale<WB>::kDot;
-        const float av = g / (1.f + __expf(-g)) * u * scale * WScale<WB>::kAct;
-#pragma unroll
-        for (int it = 0; it < kIter; ++it) {
-          float w[kVec];
-          E::load(st + 2 * kRowBytes + (it * 32 + lane) * 16, w);
-          const float a_it = kGrouped ? av * gs[kGrouped ? it : 0] : av;
-#pragma unroll
-          for (int j = 0; j < kVec; ++j) acc[it * kVec + j] = fmaf(a_it, w[j], acc[it * kVec + j]);
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(empty + s);
-      }
-
-      // Layer flush: add the eight private copies in warp order, write this CTA's partial.
-      // One pass per 32*kVec columns keeps the exchange buffer at a few KB.
-      float* dst = a.partial + (((size_t)a.phase * d.L + l) * a.grid_cap + blockIdx.x) * H;
-      constexpr int kPassCols = 32 * kVec;
-#pragma unroll
-      for (int it = 0; it < kIter; ++it) {
-        float* mine = red + (size_t)warp * kPassCols + lane * kVec;
-#pragma unroll
-        for (int v4 = 0; v4 < kVec / 4; ++v4)
-          *reinterpret_cast<float4*>(mine + v4 * 4) =
-              make_float4(acc[it * kVec + v4 * 4], acc[it * kVec + v4 * 4 + 1],
-                          acc[it * kVec + v4 * 4 + 2], acc[it * kVec + v4 * 4 + 3]);
-        consumer_bar();
-        for (int c = tid; c < kPassCols; c += kConsumerWarps * 32) {
-          float t = 0.f;
-#pragma unroll
-          for (int w = 0; w < kConsumerWarps; ++w) t += red[(size_t)w * kPassCols + c];
-          dst[it * kPassCols + c] = t;
-        }
-        consumer_bar();
-      }
-    }
-  }
+  const stream::Ring ring{full, empty, reinterpret_cast<float*>(smem + lay.red), smem + lay.stages, NS, &s_abort};
+  const StackWork<H> wk{a, trace_slot(d.trace, d.L, d.K)};
+  stream::stream_rows<WB, H>(wk, prefix, P, r0, r1, ring, a.spin_limit ? a.spin_limit : kSpinLimit, a.lose_row1);
 }
 
 __global__ void __launch_bounds__(256) combine_kernel(FfnArgs a, float* __restrict__ hidden_out, int layer0,

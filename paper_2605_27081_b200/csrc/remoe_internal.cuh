@@ -148,6 +148,13 @@ cudaError_t launch_widen_retile_tc(const DevStack& d, int n, const void* const* 
 cudaError_t launch_route(const DevStack& d, const float* hidden_in, int* ids, float* gates,
                          int* contrib, int layer0, int n_layers, cudaStream_t st);
 cudaError_t launch_ffn_stream(const FfnArgs& a, int grid, cudaStream_t st);
+// Link between two layers of the chained batch-1 step, one launch: with `do_combine` the fixed-order sum of layer
+// (layer - 1)'s partials into chain_out[layer - 1] and the residual add chain_in[layer] = chain_in[layer - 1] + out;
+// with `do_route` the pre-norm chain_x[layer] = rmsnorm(chain_in[layer]) and the routing of `layer` on it.
+// `ticket` is one zero-initialised device word owned by the stack.
+cudaError_t launch_chain_link(const DevStack& d, const FfnArgs& f, int layer, float* chain_in, float* chain_out,
+                              float* chain_x, unsigned* ticket, int do_combine, int do_route, int* ids, float* gates,
+                              cudaStream_t st);
 // Adds the partials of layers [layer0, layer0 + n_layers) into hidden_out[L, 1, H]; with `chain_in`
 // ([L + 1, 1, H]) also writes chain_in[l + 1] = chain_in[l] + out[l] (residual chaining).
 cudaError_t launch_combine(const FfnArgs& a, float* hidden_out, int layer0, int n_layers, float* chain_in,

@@ -267,22 +267,27 @@ __device__ void resolve_layer(const DevStack& d, int l, const int* flat, int n_f
   }
 }
 
-__global__ void __launch_bounds__(1024) route_kernel(DevStack d, const float* __restrict__ hidden_in,
-                                                    int* __restrict__ ids, float* __restrict__ gates,
-                                                    int* contrib, int layer0) {
-  __shared__ float z[kMaxRouted];
-  __shared__ int s_ids[32];
-  __shared__ float s_g[32];
-  __shared__ __align__(16) float h[kMaxHidden];
-  __shared__ DirSmem dir;
+// Shared memory of one routing CTA.
+struct RouteSmem {
+  float z[kMaxRouted];
+  int ids[32];
+  float g[32];
+  __align__(16) float h[kMaxHidden];
+  DirSmem dir;
+};
 
-  const int lb = layer0 * d.B + blockIdx.x;
+// Routing of one (layer, sequence) by one CTA whose input vector is already in sm.h: router logits (one warp
+// per expert row), shared-expert gate, then, by warp 0, softmax, top-K, gate weights, reuse statistics and,
+// at batch 1, the cache directory update.  Every thread of the CTA must call it.
+__device__ void route_block(const DevStack& d, RouteSmem& sm, int lb, int* __restrict__ ids,
+                            float* __restrict__ gates, int* contrib) {
+  float* z = sm.z;
+  int* s_ids = sm.ids;
+  float* s_g = sm.g;
+  const float* h = sm.h;
   const int l = lb / d.B;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const size_t row_bytes = (size_t)d.H * d.rbytes;
-  for (int c = threadIdx.x; c < d.H / 4; c += blockDim.x)
-    reinterpret_cast<float4*>(h)[c] = __ldg(reinterpret_cast<const float4*>(hidden_in + (size_t)lb * d.H) + c);
-  __syncthreads();
 
   const int n_warps = blockDim.x >> 5;
   for (int e = warp; e < d.N; e += n_warps) {
@@ -299,7 +304,6 @@ __global__ void __launch_bounds__(1024) route_kernel(DevStack d, const float* __
   }
   __syncthreads();
   if (warp != 0) return;
-
   // Softmax over all N logits and top-K on the (optionally residency-biased) logits.
   float v[kMaskWords], sc[kMaskWords];
   float m = -CUDART_INF_F;
@@ -377,7 +381,120 @@ __global__ void __launch_bounds__(1024) route_kernel(DevStack d, const float* __
       atomicAdd(d.counters + (size_t)l * kCounters + 5, 1ull);
     }
   }
-  if (d.B == 1) resolve_layer(d, l, s_ids, d.K, dir, lane, contrib);
+  if (d.B == 1) resolve_layer(d, l, s_ids, d.K, sm.dir, lane, contrib);
+}
+
+
+__global__ void __launch_bounds__(1024) route_kernel(DevStack d, const float* __restrict__ hidden_in,
+                                                    int* __restrict__ ids, float* __restrict__ gates,
+                                                    int* contrib, int layer0) {
+  __shared__ RouteSmem sm;
+  const int lb = layer0 * d.B + blockIdx.x;
+  for (int c = threadIdx.x; c < d.H / 4; c += blockDim.x)
+    reinterpret_cast<float4*>(sm.h)[c] = __ldg(reinterpret_cast<const float4*>(hidden_in + (size_t)lb * d.H) + c);
+  __syncthreads();
+  route_block(d, sm, lb, ids, gates, contrib);
+}
+
+// Link between two layers of the chained batch-1 step, one launch instead of four: the fixed-order sum of
+// layer (layer - 1)'s partial rows (the work of combine_kernel), the residual add h_layer = h_{layer-1} + out,
+// the pre-norm x = h / sqrt(mean(h^2) + 1e-6) and the routing of `layer` on x.
+//   grid = kLinkCtas CTAs of 1024 threads.  CTA c sums 1/kLinkCtas of the columns: 16 row groups of 64 threads,
+//   a thread adding the float4 pieces of its group's rows in order, the groups then added in order (fixed
+//   order, no float atomics).  The CTA that finishes last (a ticket counter; nobody waits for anybody) reads the
+//   complete h back, normalises it and routes.  With do_combine == 0 (first layer) one CTA normalises and
+//   routes h as it stands; with do_route == 0 (after the last layer) the sum and the residual add are all.
+constexpr int kLinkCtas = 8;
+struct LinkArgs {
+  const float* partial;       // [2][L][grid_cap][H]
+  const int* contrib_in;      // [2][L][2]
+  int grid_cap;
+  int layer;                  // layer to route; the partials summed are those of layer - 1
+  float* chain_in;            // [L + 1][H] residual stream
+  float* chain_out;           // [L][H] per-layer MoE outputs
+  float* chain_x;             // [L][H] normalised layer inputs
+  unsigned* ticket;
+  int do_combine, do_route;
+};
+
+__global__ void __launch_bounds__(1024) chain_link_kernel(DevStack d, LinkArgs a, int* __restrict__ ids,
+                                                         float* __restrict__ gates, int* contrib) {
+  __shared__ RouteSmem sm;
+  __shared__ float4 red[16][64];
+  __shared__ int s_last;
+  __shared__ float warp_ss[32];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int H = d.H, l = a.layer;
+
+  if (a.do_combine) {
+    const int lp = l - 1;
+    const int cols = H / kLinkCtas;                       // columns of this CTA; H / 8 <= 256, a multiple of 4
+    const int c4 = tid & 63, rg = tid >> 6;
+    const int col = blockIdx.x * cols + c4 * 4;
+    const bool active = c4 * 4 < cols;
+    // rows: resident-phase partials lo0..hi0, then miss-phase partials lo1..hi1
+    const int lo0 = a.contrib_in[(0 * d.L + lp) * 2], hi0 = a.contrib_in[(0 * d.L + lp) * 2 + 1];
+    const int lo1 = a.contrib_in[(1 * d.L + lp) * 2], hi1 = a.contrib_in[(1 * d.L + lp) * 2 + 1];
+    const int n0 = hi0 >= lo0 ? hi0 - lo0 + 1 : 0, n1 = hi1 >= lo1 ? hi1 - lo1 + 1 : 0;
+    const int n = n0 + n1, per = (n + 15) / 16;
+    const int ra = min(n, rg * per), rb = min(n, ra + per);
+    float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (active) {
+      const float* p0 = a.partial + ((size_t)(0 * d.L + lp) * a.grid_cap) * H + col;
+      const float* p1 = a.partial + ((size_t)(1 * d.L + lp) * a.grid_cap) * H + col;
+#pragma unroll 8
+      for (int r = ra; r < rb; ++r) {
+        const float* src = r < n0 ? p0 + (size_t)(lo0 + r) * H : p1 + (size_t)(lo1 + r - n0) * H;
+        const float4 v = __ldcg(reinterpret_cast<const float4*>(src));
+        t.x += v.x; t.y += v.y; t.z += v.z; t.w += v.w;
+      }
+    }
+    red[rg][c4] = t;
+    __syncthreads();
+    if (rg == 0 && active) {
+      float4 o = red[0][c4];
+#pragma unroll
+      for (int g2 = 1; g2 < 16; ++g2) { o.x += red[g2][c4].x; o.y += red[g2][c4].y; o.z += red[g2][c4].z; o.w += red[g2][c4].w; }
+      *reinterpret_cast<float4*>(a.chain_out + (size_t)lp * H + col) = o;
+      const float4 hp = *reinterpret_cast<const float4*>(a.chain_in + (size_t)lp * H + col);
+      *reinterpret_cast<float4*>(a.chain_in + (size_t)l * H + col) =
+          make_float4(hp.x + o.x, hp.y + o.y, hp.z + o.z, hp.w + o.w);
+    }
+    // the CTA that takes the last ticket sees every other CTA's columns (fence, then ticket)
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+      const unsigned t0 = atomicAdd(a.ticket, 1u);
+      s_last = t0 == gridDim.x - 1 ? 1 : 0;
+      if (s_last) *a.ticket = 0u;                          // ready for the next launch
+    }
+    __syncthreads();
+    if (!s_last || !a.do_route) return;
+    __threadfence();
+  }
+
+  // pre-norm of h_l (fixed summation order), x_l to shared memory for the router and to global memory for
+  // the expert kernels
+  const float* hl = a.chain_in + (size_t)l * H;
+  float ss = 0.f;
+  for (int c = tid; c < H; c += 1024) {
+    const float v = __ldcg(hl + c);
+    sm.h[c] = v;
+    ss = fmaf(v, v, ss);
+  }
+  ss = warp_sum(ss);
+  if (lane == 0) warp_ss[warp] = ss;
+  __syncthreads();
+  float tot = 0.f;
+  for (int w = 0; w < 32; ++w) tot += warp_ss[w];
+  const float sc = rsqrtf(tot / (float)H + 1e-6f);
+  for (int c = tid; c < H; c += 1024) {
+    const float x = sm.h[c] * sc;
+    sm.h[c] = x;
+    a.chain_x[(size_t)l * H + c] = x;
+  }
+  __syncthreads();
+  route_block(d, sm, l, ids, gates, contrib);
 }
 
 __global__ void __launch_bounds__(32) resolve_kernel(DevStack d, const int* __restrict__ ids, int* contrib,
@@ -404,6 +521,26 @@ cudaError_t launch_route(const DevStack& d, const float* hidden_in, int* ids, fl
     e = cudaGetLastError();
   }
   return e;
+}
+
+// Chained batch-1 step: sum of layer (layer - 1)'s partials + residual add (do_combine), then pre-norm and
+// routing of `layer` (do_route), in one launch.  `ticket` is one zero-initialised word owned by the stack.
+cudaError_t launch_chain_link(const DevStack& d, const FfnArgs& f, int layer, float* chain_in, float* chain_out,
+                              float* chain_x, unsigned* ticket, int do_combine, int do_route, int* ids, float* gates,
+                              cudaStream_t st) {
+  LinkArgs a{};
+  a.partial = f.partial;
+  a.contrib_in = f.contrib;
+  a.grid_cap = f.grid_cap;
+  a.layer = layer;
+  a.chain_in = chain_in;
+  a.chain_out = chain_out;
+  a.chain_x = chain_x;
+  a.ticket = ticket;
+  a.do_combine = do_combine;
+  a.do_route = do_route;
+  chain_link_kernel<<<do_combine ? kLinkCtas : 1, 1024, 0, st>>>(d, a, ids, gates, f.contrib);
+  return cudaGetLastError();
 }
 
 }  // namespace remoe

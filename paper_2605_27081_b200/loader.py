@@ -50,7 +50,15 @@ class LoadedWorkload:
             synth.fill_expert_store(seed, gen_shape, self.store, threads=threads)
         self.routers = [synth.gen_router(seed, shape, l) for l in range(L)]
         self.shared_gates = [synth.gen_shared_gate(seed, shape, l) for l in range(L)] if shape.shared_gate else None
-        self.shared = [[synth.gen_shared_block(seed, shape, l, i) for i in range(shape.n_shared)] for l in range(L)]
+        jobs = [(l, i) for l in range(L) for i in range(shape.n_shared)]
+        if len(jobs) >= 4:
+            from concurrent.futures import ThreadPoolExecutor
+            import os
+            with ThreadPoolExecutor(threads or len(os.sched_getaffinity(0))) as ex:
+                blocks = list(ex.map(lambda li: synth.gen_shared_block(seed, shape, li[0], li[1]), jobs))
+        else:
+            blocks = [synth.gen_shared_block(seed, shape, l, i) for l, i in jobs]
+        self.shared = [[blocks[l * shape.n_shared + i] for i in range(shape.n_shared)] for l in range(L)]
 
         self.stack = self.new_stack(cache_slots, stream)
 

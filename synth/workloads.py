@@ -149,19 +149,23 @@ def _fp8_table() -> np.ndarray:
 
 
 _FP8 = _fp8_table()
-_FP8_POS = _FP8[:127].astype(np.float64)            # non-negative finite values, ascending (0 .. 448)
-_FP8_MID = (_FP8_POS[1:] + _FP8_POS[:-1]) / 2
 
 
 def fp8_e4m3_round_to_bits(x: np.ndarray) -> np.ndarray:
-    """float32 -> FP8 E4M3 bytes: nearest value, ties to the even code, magnitudes above 448 saturate."""
-    x = np.asarray(x, dtype=np.float32)
-    a = np.abs(x).astype(np.float64)
-    idx = np.searchsorted(_FP8_MID, a, side="left")                  # first midpoint >= |x|
-    tie = (idx < len(_FP8_MID)) & (a == _FP8_MID[np.minimum(idx, len(_FP8_MID) - 1)])
-    idx = np.where(tie & (idx % 2 == 1), idx + 1, idx)              # at a midpoint: the even neighbour
-    idx = np.minimum(idx, 126).astype(np.uint8)
-    return (idx | np.where(np.signbit(x), 0x80, 0).astype(np.uint8)).astype(np.uint8)
+    """float32 -> FP8 E4M3 bytes: nearest value, ties to the even code, magnitudes above 448 saturate.
+
+    Done on the bit patterns: in the normal range (|x| >= 2^-6) the 23-bit mantissa is rounded to 3 bits,
+    nearest even, with the carry running into the exponent, and the exponent is re-biased from 127 to 7;
+    below that the format is subnormal, multiples of 2^-9, and |x| * 2^9 is rounded to an integer."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    u = x.view(np.uint32)
+    a = u & np.uint32(0x7FFFFFFF)
+    r = (a + np.uint32(0x7FFFF) + ((a >> np.uint32(20)) & np.uint32(1))) >> np.uint32(20)
+    code = r.astype(np.int32) - ((127 - 7) << 3)
+    small = a < np.uint32(0x3C800000)                                   # |x| < 2^-6
+    sub = np.rint(np.minimum(a.view(np.float32), np.float32(1.0)) * np.float32(512.0)).astype(np.int32)
+    code = np.clip(np.where(small, sub, code), 0, 126).astype(np.uint8)
+    return code | ((u >> np.uint32(24)) & np.uint32(0x80)).astype(np.uint8)
 
 
 def fp8_e4m3_bits_to_f32(bits: np.ndarray) -> np.ndarray:

@@ -34,6 +34,17 @@ def dsv2lite_base():
     wl.torch_stream = stream
     yield wl
     wl.close()
+    del wl
+    _release_pinned()
+
+
+def _release_pinned():
+    """Give freed pinned host blocks back to the system (the host allocator would keep them cached)."""
+    import gc
+    import torch
+    gc.collect()
+    if hasattr(torch._C, "_host_emptyCache"):
+        torch._C._host_emptyCache()
 
 
 def _with_new_stack(base, cache_slots):
@@ -88,6 +99,9 @@ def _full(name, rho, steps, distinct=None, sample_layers=(0, -1), policy=None, b
         return out
     finally:
         wl.stack.close()
+        if base is None:
+            del wl
+            _release_pinned()
 
 
 def test_dsv2lite_full_store_all_rhos(dsv2lite_base):
@@ -197,5 +211,60 @@ def test_dsv2lite_b32_full_shape_mma_kernel(dsv2lite_base, monkeypatch):
     with per-slot ordering).  Routing and the cache directory are the same code under both kernels, so the
     default run covers a prefix of the 1024 steps; REMOE_LONG_TESTS=1 runs them all."""
     monkeypatch.setenv("REMOE_BATCHED_KERNEL", "mma")
-    n = 1024 if os.environ.get("REMOE_LONG_TESTS") == "1" else 160
+    n = 1024 if os.environ.get("REMOE_LONG_TESTS") == "1" else 96
     _b32(dsv2lite_base, n, {0, 1, n // 2, n - 1})
+
+
+@pytest.fixture(scope="module")
+def dsv2lite_fp8_base():
+    """The same stack over an FP8 E4M3 host store (all 26 x 64 blocks distinct, 14.4 GB)."""
+    import torch
+    from paper_2605_27081_b200.loader import LoadedWorkload
+
+    cfg = synth.config("dsv2lite_fp8")
+    stream = torch.cuda.Stream()
+    wl = LoadedWorkload(cfg["shape"], cfg["cache_slots"], cfg["seed"], stream=stream.cuda_stream)
+    wl.torch_stream = stream
+    yield wl
+    wl.close()
+    del wl
+    _release_pinned()
+
+
+def test_dsv2lite_fp8_store_full_shape(dsv2lite_fp8_base):
+    """Lower-precision host store at the benchmark's shape, batch 1: slots hold the FP8 bytes."""
+    res = _full("dsv2lite_fp8", 0.9, 192, base=dsv2lite_fp8_base)
+    print("dsv2lite_fp8:", res)
+
+
+def test_dsv2lite_b32_fp8_store_full_shape(dsv2lite_fp8_base):
+    """... and under the batched stack: FP8 fetches (half the bytes per miss), widened to bf16 operand tiles."""
+    import torch
+    from paper_2605_27081_b200.loader import LoadedWorkload
+    from parity_util import StepChecker, oracle_for
+
+    cfg = synth.config("dsv2lite_b32_fp8")
+    shape = cfg["shape"]
+    stream = dsv2lite_fp8_base.torch_stream
+    wl = LoadedWorkload(shape, cfg["cache_slots"], cfg["seed"], stream=stream.cuda_stream, store_of=dsv2lite_fp8_base)
+    try:
+        chk = StepChecker(wl, oracle_for(wl), torch)
+        hs = synth.HiddenStream(cfg["seed"], shape, None)
+        n = 64
+        with torch.cuda.stream(stream):
+            for t in range(n):
+                if t in (0, n - 1):
+                    chk.step_overlapped(hs.step(), ffn="selected", ffn_layers=[(11 * t) % shape.n_layers])
+                else:
+                    chk.step_overlapped(hs.step(), ffn=None)
+        chk.check_counters()                      # h2d_bytes = misses x FP8 block bytes, exactly
+        assert wl.stack.cache_stats()["h2d_bytes"] == sum(chk.o.uniq_misses) * 3 * 1408 * 2048
+        print("dsv2lite_b32_fp8:", chk.tie_report(), "max out err", chk.max_out_err, "uHR", chk.o.uhr())
+    finally:
+        wl.close()
+
+
+def test_dsv2lite_int4_store_full_shape():
+    """4-bit grouped host store at the benchmark's shape, batch 1 (all blocks distinct, 8.1 GB)."""
+    res = _full("dsv2lite_int4", 0.9, 160)
+    print("dsv2lite_int4:", res)

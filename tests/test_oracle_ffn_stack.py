@@ -270,6 +270,14 @@ def test_fp8_storage_matches_library_cast():
     ref_bits = torch.from_numpy(x).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
     assert np.array_equal(synth.fp8_e4m3_round_to_bits(x), ref_bits)
     assert list(synth.fp8_e4m3_round_to_bits(np.array([1000.0, -1000.0], np.float32))) == [126, 254]
+    # every midpoint between neighbouring codes goes to the even code, its float32 neighbours to either side
+    vals = synth.fp8_e4m3_bits_to_f32(np.arange(127, dtype=np.uint8)).astype(np.float64)
+    mids = ((vals[1:] + vals[:-1]) / 2).astype(np.float32)
+    lo = np.arange(126)
+    assert np.array_equal(synth.fp8_e4m3_round_to_bits(mids), np.where(lo % 2 == 0, lo, lo + 1).astype(np.uint8))
+    assert np.array_equal(synth.fp8_e4m3_round_to_bits(np.nextafter(mids, np.float32(0))), lo.astype(np.uint8))
+    assert np.array_equal(synth.fp8_e4m3_round_to_bits(np.nextafter(mids, np.float32(1e9))), (lo + 1).astype(np.uint8))
+    assert np.array_equal(synth.fp8_e4m3_round_to_bits(-mids), (np.where(lo % 2 == 0, lo, lo + 1) | 0x80).astype(np.uint8))
     shape = synth.Shape(1, 512, 4, 2, 8, 0, 0, 0, 0, 2, 1)
     blk = synth.gen_expert_block(0, shape, 0, 1)
     assert blk.dtype == np.uint8 and synth.gen_router(0, shape, 0).dtype == np.uint16
