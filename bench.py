@@ -412,9 +412,11 @@ def reduce_over_ranks(dist, maxima: dict, sums: dict, device):
 def step_roofline(shape, r, steps, peak_hbm, h2d_peak):
     """bytes one step must move: resident experts + shared + router from HBM, misses over the host link"""
     # a batched stack over an FP8 store keeps bf16 blocks on the device (widened on arrival)
-    dev_elem = 2 if (shape.weight_dtype == 2 and shape.batch > 1) else shape.elem_bytes
-    S_dev = synth.expert_block_elems(shape.hidden, shape.inter_routed) * dev_elem
-    S_sh = synth.expert_block_elems(shape.hidden, shape.inter_shared) * dev_elem
+    if shape.weight_dtype == 2 and shape.batch > 1:
+        S_dev = synth.expert_block_elems(shape.hidden, shape.inter_routed) * 2
+        S_sh = synth.expert_block_elems(shape.hidden, shape.inter_shared) * 2
+    else:
+        S_dev, S_sh = synth.expert_block_bytes(shape), synth.expert_block_bytes(shape, shared=True)
     router = shape.n_layers * shape.n_routed * shape.hidden * (4 if shape.weight_dtype == 0 else 2)
     hbm = (r["uniq_hits"] + r["uniq_misses"]) * S_dev / steps + shape.n_layers * shape.n_shared * S_sh + router
     t_hbm = hbm / (peak_hbm * 1e9)
