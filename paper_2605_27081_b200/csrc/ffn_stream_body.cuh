@@ -135,6 +135,19 @@ __device__ __forceinline__ void stream_rows(const Work& wk, const int* prefix, i
     }
 #pragma unroll
     for (int c = 0; c < kCols; ++c) acc[c] = 0.f;
+    // grouped format: the decoded codes carry an offset that is taken out once per group -- from a dot product
+    // with the sum of this lane's h over the group, from the AXPY with the sum of the row activations
+    float hsum[kGrouped ? kIter : 1], asum[kGrouped ? kIter : 1];
+    if constexpr (kGrouped) {
+#pragma unroll
+      for (int it = 0; it < kIter; ++it) {
+        float t = 0.f;
+#pragma unroll
+        for (int j = 0; j < kVec; ++j) t += hreg[it * kVec + j];
+        hsum[it] = t * E::kBias;
+        asum[it] = 0.f;
+      }
+    }
 
     // first row of this layer handled by this warp: local index n = r - r0 with n % 8 == warp
     int r = lo + ((warp - (lo - r0)) % kConsumerWarps + kConsumerWarps) % kConsumerWarps;
@@ -167,7 +180,7 @@ __device__ __forceinline__ void stream_rows(const Work& wk, const int* prefix, i
           E::load(st + (it * 32 + lane) * 16, w);
 #pragma unroll
           for (int j = 0; j < kVec; ++j) t = fmaf(w[j], hreg[it * kVec + j], t);
-          g = fmaf(E::scale(st, H, it * 32 + lane), t, g);
+          g = fmaf(E::scale(st, H, it * 32 + lane), t - hsum[it], g);
         }
 #pragma unroll
         for (int it = 0; it < kIter; ++it) {
@@ -175,7 +188,7 @@ __device__ __forceinline__ void stream_rows(const Work& wk, const int* prefix, i
           E::load(st + kRowBytes + (it * 32 + lane) * 16, w);
 #pragma unroll
           for (int j = 0; j < kVec; ++j) t = fmaf(w[j], hreg[it * kVec + j], t);
-          u = fmaf(E::scale(st + kRowBytes, H, it * 32 + lane), t, u);
+          u = fmaf(E::scale(st + kRowBytes, H, it * 32 + lane), t - hsum[it], u);
           gs[it] = E::scale(st + 2 * kRowBytes, H, it * 32 + lane);
         }
       } else {
@@ -207,6 +220,7 @@ __device__ __forceinline__ void stream_rows(const Work& wk, const int* prefix, i
         float w[kVec];
         E::load(st + 2 * kRowBytes + (it * 32 + lane) * 16, w);
         const float a_it = kGrouped ? av * gs[kGrouped ? it : 0] : av;
+        if constexpr (kGrouped) asum[it] += a_it;
 #pragma unroll
         for (int j = 0; j < kVec; ++j) acc[it * kVec + j] = fmaf(a_it, w[j], acc[it * kVec + j]);
       }
@@ -214,6 +228,12 @@ __device__ __forceinline__ void stream_rows(const Work& wk, const int* prefix, i
       if (lane == 0) mbar_arrive(empty + s);
     }
 
+    if constexpr (kGrouped) {
+#pragma unroll
+      for (int it = 0; it < kIter; ++it)
+#pragma unroll
+        for (int j = 0; j < kVec; ++j) acc[it * kVec + j] = fmaf(-E::kBias, asum[it], acc[it * kVec + j]);
+    }
     // Layer flush: add the eight private copies in warp order, write this CTA's partial.
     // One pass per 32*kVec columns keeps the exchange buffer at a few KB.
     float* dst = wk.partial(l);

@@ -118,14 +118,20 @@ struct Elems<1> {
 };
 // 4-bit grouped format (tag 0): sixteen stored bytes are one group of 32 codes, element 2i in the low and element
 // 2i+1 in the high half of byte i; a code c stands for (c - 8) * the group's scale, the scales (bfloat16) follow
-// the codes of a row.  load() yields the 32 integers c - 8 as floats (2^23 + c is the float with bit pattern
-// 0x4B000000 | c); the caller multiplies a group's finished partial sum by its scale.
+// the codes of a row.  load() yields the 32 numbers c + 128 as floats: 128 + c is the float with bit pattern
+// 0x43000000 | (c << 16), so a code costs one shift and one logic operation (the code that already sits at
+// bits 16-19 only the latter).  The caller removes the offset kBias = 136 once per group, from the finished
+// partial sum (sum_j (c_j + 128) h_j - 136 sum_j h_j), and multiplies by the group's scale.
 template <>
 struct Elems<0> {
   static constexpr int kVec = 32;
+  static constexpr float kBias = 136.f;
+  __device__ static __forceinline__ float code(uint32_t at_bit16) {
+    return __uint_as_float((at_bit16 & 0x000f0000u) | 0x43000000u);
+  }
   __device__ static __forceinline__ void word(uint32_t w, float* f) {
-#pragma unroll
-    for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(((w >> (4 * i)) & 0xfu) | 0x4b000000u) - 8388616.f;
+    f[0] = code(w << 16); f[1] = code(w << 12); f[2] = code(w << 8); f[3] = code(w << 4);
+    f[4] = code(w);       f[5] = code(w >> 4);  f[6] = code(w >> 8); f[7] = code(w >> 12);
   }
   __device__ static __forceinline__ void load(const char* p, float* f) {
     const uint4 v = *reinterpret_cast<const uint4*>(p);

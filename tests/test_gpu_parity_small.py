@@ -157,6 +157,9 @@ def test_reset_and_errors():
 @pytest.mark.parametrize("shape,c", [
     (synth.Shape(6, 512, 24, 3, 64, 1, 32, 1, 0, 1, 1), 6),
     (synth.Shape(4, 256, 16, 2, 40, 0, 0, 0, 1, 0, 1), 4),
+    (synth.Shape(5, 128, 12, 2, 24, 1, 16, 0, 0, 0, 1), 2),        # narrowest width: the link kernel's column slices are 16 wide
+    (synth.Shape(4, 2048, 32, 4, 24, 2, 16, 1, 0, 3, 1), 6),       # full width, 4-bit grouped store, sigmoid gate
+    (synth.Shape(4, 1024, 32, 4, 24, 0, 0, 0, 0, 2, 1), 4),        # FP8 store, C = K
 ])
 def test_chained_stack(shape, c):
     """Layers feeding each other through the residual: routing of layer l+1 sees layer l's output."""
@@ -336,6 +339,8 @@ def test_policy_switch_and_second_stack_share_a_store():
     (synth.Shape(6, 512, 24, 3, 64, 1, 32, 1, 0, 1, 1), 6, 0.6, 23),       # odd number of steps, sigmoid gate
     (synth.Shape(3, 1024, 40, 4, 200, 2, 100, 0, 1, 1, 1), 9, 0.3, 16),    # many misses per step, renormalised
     (synth.Shape(2, 256, 16, 2, 32, 0, 0, 0, 0, 0, 1), 2, 0.0, 9),         # float32, C = K: every slot turns over
+    (synth.Shape(3, 1024, 24, 3, 72, 1, 40, 0, 0, 2, 1), 4, 0.4, 12),      # FP8 store
+    (synth.Shape(3, 1024, 24, 3, 72, 1, 40, 0, 0, 3, 1), 4, 0.4, 12),      # 4-bit grouped store
 ])
 def test_multi_step_call_equals_single_steps(shape, c, rho, n):
     """remoe_decode_steps routes step t+1 while step t is still fetching; everything it returns must be
