@@ -92,9 +92,9 @@ struct DirSmem {
 
 // Cache resolution for one layer by one warp.  `flat` holds the step's B*K requested ids in
 // (sequence, rank) order (App. E.2.3: R); U = Unique(R) keeps first occurrences.
-__device__ void resolve_layer(const DevStack& d, int l, const int* flat, int n_flat, DirSmem& sm,
-                              int lane, int* contrib) {
-  const int C = d.C, N = d.N, BK = d.B * d.K;
+// The layer's directory as it stands before the step, into shared memory (one warp).
+__device__ __forceinline__ void load_directory(const DevStack& d, int l, DirSmem& sm, int lane) {
+  const int C = d.C, N = d.N;
   for (int s = lane; s < C; s += 32) {
     sm.sgen[s] = 0;
     sm.eos[s] = d.expert_of_slot[l * C + s];
@@ -103,6 +103,12 @@ __device__ void resolve_layer(const DevStack& d, int l, const int* flat, int n_f
   }
   for (int e = lane; e < N; e += 32) sm.soe[e] = d.slot_of_expert[l * N + e];
   if (lane < kMaskWords) sm.seen[lane] = 0u;
+}
+
+__device__ void resolve_layer(const DevStack& d, int l, const int* flat, int n_flat, DirSmem& sm,
+                              int lane, int* contrib, bool directory_loaded = false) {
+  const int C = d.C, N = d.N, BK = d.B * d.K;
+  if (!directory_loaded) load_directory(d, l, sm, lane);
   __syncwarp();
 
   const unsigned lt = (1u << lane) - 1u;
@@ -290,6 +296,10 @@ __device__ void route_block(const DevStack& d, RouteSmem& sm, int lb, int* __res
   const size_t row_bytes = (size_t)d.H * d.rbytes;
 
   const int n_warps = blockDim.x >> 5;
+  // at batch 1 the directory update follows in this CTA: one warp fetches the directory image while the
+  // others are waiting for their router rows, so that round trip is off the resolve warp's chain
+  const bool preload = d.B == 1 && n_warps >= 3;
+  if (preload && warp == n_warps - 2) load_directory(d, l, sm.dir, lane);
   for (int e = warp; e < d.N; e += n_warps) {
     const float acc = row_dot(d.router + ((size_t)l * d.N + e) * row_bytes, h, d.H, d.rbytes, lane);
     if (lane == 0) z[e] = acc;
@@ -312,7 +322,7 @@ __device__ void route_block(const DevStack& d, RouteSmem& sm, int lb, int* __res
     const int e = lane + 32 * j;
     v[j] = e < d.N ? z[e] : -CUDART_INF_F;
     sc[j] = v[j];
-    if (d.beta != 0.f && e < d.N && d.slot_of_expert[l * d.N + e] >= 0) sc[j] += d.beta;
+    if (d.beta != 0.f && e < d.N && (preload ? sm.dir.soe[e] : d.slot_of_expert[l * d.N + e]) >= 0) sc[j] += d.beta;
     m = fmaxf(m, v[j]);
   }
   m = warp_max(m);
@@ -357,20 +367,22 @@ __device__ void route_block(const DevStack& d, RouteSmem& sm, int lb, int* __res
 
   // Reuse: |E_t n E_{t-1}| from selection bit masks (Eq. 1) and the reuse mass
   // m_t = (1/K) sum_{k in E_{t-1}} P_t^(k) (Eq. 2); both counted from the second step on.
+  // The previous step's mask words are read in one round trip (lane j holds word j) and handed round by
+  // shuffle; the new words go back the same way.
   int ov = 0;
   float mass = 0.f;
+  unsigned* pm = d.prev_mask + (size_t)lb * kMaskWords;
+  const unsigned prev_mine = (d.has_prev && lane < kMaskWords) ? pm[lane] : 0u;
+  unsigned word_mine = 0u;
 #pragma unroll
   for (int j = 0; j < kMaskWords; ++j) {
     const unsigned word = __ballot_sync(kFull, (taken >> j) & 1u);
-    unsigned* pm = d.prev_mask + (size_t)lb * kMaskWords + j;
-    const unsigned prev = d.has_prev ? *pm : 0u;
-    __syncwarp();
+    const unsigned prev = __shfl_sync(kFull, prev_mine, j);
     if ((prev >> lane) & 1u) mass += expf(v[j] - m) / sum;
-    if (lane == 0) {
-      ov += __popc(word & prev);
-      *pm = word;
-    }
+    ov += __popc(word & prev);
+    if (lane == j) word_mine = word;
   }
+  if (lane < kMaskWords) pm[lane] = word_mine;
   mass = warp_sum(mass) / (float)d.K;
   if (lane == 0) {
     d.last_overlap[lb] = d.has_prev ? ov : -1;
@@ -381,7 +393,7 @@ __device__ void route_block(const DevStack& d, RouteSmem& sm, int lb, int* __res
       atomicAdd(d.counters + (size_t)l * kCounters + 5, 1ull);
     }
   }
-  if (d.B == 1) resolve_layer(d, l, s_ids, d.K, sm.dir, lane, contrib);
+  if (d.B == 1) resolve_layer(d, l, s_ids, d.K, sm.dir, lane, contrib, preload);
 }
 
 

@@ -5,11 +5,11 @@ at every step of the full number of decode steps of each configuration (512, 512
 batched stack, 1024); floating-point outputs at sampled (step, layer) pairs, which the oracle
 computes one by one.  The DeepSeek-V2-Lite-shaped stacks (batch 1, its policy variants, the multi-step
 call and the batched stack) share one full host store of 26 x 64 distinct expert blocks; the
-Qwen1.5-MoE-shaped stack also has all its blocks distinct.  The Qwen3-30B-shaped stack keeps its full
-shape (layers, experts, router, cache) but lets expert ids share distinct weight blocks per layer
-through the pointer table (both sides read the same aliased blocks): an expert fetched in place of
-another one whose id is congruent modulo that number would not show in its output comparison, only in
-its cache trace.
+Qwen1.5-MoE-shaped and Qwen3-30B-shaped stacks also have all their blocks distinct (25 and 58 GB of
+pinned host memory).  With REMOE_SMALL_HOST=1 the latter lets expert ids share 16 distinct weight blocks
+per layer through the pointer table (both sides read the same aliased blocks); an expert fetched in place
+of another one whose id is congruent modulo 16 would then not show in its output comparison, only in its
+cache trace.
 """
 import copy
 import os
@@ -104,6 +104,20 @@ def _full(name, rho, steps, distinct=None, sample_layers=(0, -1), policy=None, b
             _release_pinned()
 
 
+# The two stacks with their own full stores run first, so that their pinned memory (25 and 58 GB) is released
+# before the shared DeepSeek-V2-Lite store is built.
+def test_qwen15moe_full_shape():
+    res = _full("qwen15moe", 0.8, 512)                  # all 24 x 60 blocks distinct
+    print("qwen15moe:", res)
+
+
+def test_qwen3_30b_full_shape():
+    # all 48 x 128 blocks distinct: 58 GB of pinned host memory (REMOE_SMALL_HOST=1: 16 distinct blocks per layer)
+    distinct = 16 if os.environ.get("REMOE_SMALL_HOST") == "1" else None
+    res = _full("qwen3_30b", [0.5, 0.9], [1024, 1024], distinct=distinct)
+    print("qwen3_30b:", res, "distinct blocks per layer:", distinct or 128)
+
+
 def test_dsv2lite_full_store_all_rhos(dsv2lite_base):
     res = _full("dsv2lite", [0.9, 0.5, 0.0], [512, 512, 512], base=dsv2lite_base)
     print("dsv2lite:", res)
@@ -149,18 +163,6 @@ def test_dsv2lite_multi_step_call_full_shape(dsv2lite_base):
     finally:
         other.close()
         one.close()
-
-
-def test_qwen15moe_full_shape():
-    res = _full("qwen15moe", 0.8, 512)                  # all 24 x 60 blocks distinct
-    print("qwen15moe:", res)
-
-
-def test_qwen3_30b_full_shape():
-    # 16 distinct blocks per layer by default; REMOE_LONG_TESTS=1 generates all 48 x 128 (58 GB of pinned memory)
-    distinct = None if os.environ.get("REMOE_LONG_TESTS") == "1" else 16
-    res = _full("qwen3_30b", [0.5, 0.9], [1024, 1024], distinct=distinct)
-    print("qwen3_30b:", res, "distinct blocks per layer:", distinct or 128)
 
 
 def _b32(base, n, float_steps):
