@@ -367,28 +367,34 @@ def median_rep(reps, key="ms"):
     return reps[order[len(order) // 2]]
 
 
-def measure_h2d(torch, nbytes, reps=12):
-    """Pinned host -> device copy rate (GB/s): the better of a train of expert-sized copies and
-    one large copy, best of `reps`, CUDA events on the copying stream."""
-    n_copies = int(min(256, max(32, -(-(512 << 20) // nbytes))))        # at least 512 MB per round where that takes <= 256 copies
-    h = torch.empty(n_copies * nbytes, dtype=torch.uint8).pin_memory()
-    h.fill_(1)
+def measure_h2d(torch, nbytes, reps=12, store=None):
+    """Pinned host -> device copy rate (GB/s): the better of a train of expert-sized copies and one large
+    copy, best of `reps`, CUDA events on the copying stream.  Sources: a fresh pinned buffer and, when given,
+    the head of the expert store itself (`store`: pinned uint8 tensor) -- the memory the steps fetch from,
+    which may sit on another NUMA node than a fresh allocation."""
+    n_copies = int(min(256, max(32, -(-(512 << 20) // nbytes))))        # at least 512 MB per pass where that takes <= 256 copies
+    fresh = torch.empty(n_copies * nbytes, dtype=torch.uint8).pin_memory()
+    fresh.fill_(1)
+    sources = [fresh]
+    if store is not None and store.numel() >= n_copies * nbytes:
+        sources.append(store[:n_copies * nbytes])
     d = torch.empty(n_copies * nbytes, dtype=torch.uint8, device="cuda")
     st = torch.cuda.Stream()
     best = 0.0
     with torch.cuda.stream(st):
-        for rep in range(reps + 2):
-            for pieces in (n_copies, 1):
-                chunk = n_copies * nbytes // pieces
-                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                torch.cuda.synchronize()
-                a.record(st)
-                for i in range(pieces):
-                    d[i * chunk:(i + 1) * chunk].copy_(h[i * chunk:(i + 1) * chunk], non_blocking=True)
-                b.record(st)
-                torch.cuda.synchronize()
-                if rep >= 2:                                   # the first rounds touch the pages
-                    best = max(best, n_copies * nbytes / a.elapsed_time(b) / 1e6)
+        for h in sources:
+            for rep in range(reps + 2):
+                for pieces in (n_copies, 1):
+                    chunk = n_copies * nbytes // pieces
+                    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    torch.cuda.synchronize()
+                    a.record(st)
+                    for i in range(pieces):
+                        d[i * chunk:(i + 1) * chunk].copy_(h[i * chunk:(i + 1) * chunk], non_blocking=True)
+                    b.record(st)
+                    torch.cuda.synchronize()
+                    if rep >= 2:                                   # the first passes touch the pages
+                        best = max(best, n_copies * nbytes / a.elapsed_time(b) / 1e6)
     return best
 
 
@@ -412,8 +418,8 @@ def reduce_over_ranks(dist, maxima: dict, sums: dict, device):
 
 def step_roofline(shape, r, steps, peak_hbm, h2d_peak):
     """bytes one step must move: resident experts + shared + router from HBM, misses over the host link"""
-    # a batched stack over an FP8 store keeps bf16 blocks on the device (widened on arrival)
-    if shape.weight_dtype == 2 and shape.batch > 1:
+    # a batched stack over an FP8 or 4-bit store keeps bf16 blocks on the device (widened on arrival)
+    if shape.weight_dtype in (2, 3) and shape.batch > 1:
         S_dev = synth.expert_block_elems(shape.hidden, shape.inter_routed) * 2
         S_sh = synth.expert_block_elems(shape.hidden, shape.inter_shared) * 2
     else:
@@ -472,7 +478,7 @@ def short_run(torch, name, steps, warmup, peak_hbm, h2d_peak_of, store_of=None, 
            "cache_slots": C, "steps": steps, "warmup": warmup,
            "distinct_experts_per_layer": wl.n_distinct, "blocks_aliased": wl.n_distinct < shape.n_routed}
     try:
-        h2d_peak = h2d_peak_of(S_e)
+        h2d_peak = h2d_peak_of(S_e, wl._store_t)
         out["h2d_peak_gbs"] = h2d_peak
         runs = {}
         for rho in cfg["rhos"]:
@@ -521,12 +527,12 @@ def run_ours(args, rank, world, local_rank):
     note(f"{args.workload}: store of {wl.n_distinct} distinct blocks per layer loaded")
     h2d_cache = {}
 
-    def h2d_peak_of(nbytes):
+    def h2d_peak_of(nbytes, store=None):
         if nbytes not in h2d_cache:
-            h2d_cache[nbytes] = measure_h2d(torch, nbytes)
+            h2d_cache[nbytes] = measure_h2d(torch, nbytes, store=store)
         return h2d_cache[nbytes]
 
-    h2d_peak = h2d_peak_of(S_e)
+    h2d_peak = h2d_peak_of(S_e, wl._store_t)
 
     def barrier():
         torch.cuda.synchronize()
@@ -691,7 +697,7 @@ def run_ours(args, rank, world, local_rank):
         others, kept = {}, {}
         n_o, w_o = min(args.steps, 24), min(max(args.warmup, 8), 16)
         for name in ("tiny_fp32", "qwen15moe", "qwen3_30b", "dsv2lite_b32", "dsv2lite_fp8", "dsv2lite_b32_fp8",
-                     "dsv2lite_int4"):
+                     "dsv2lite_int4", "dsv2lite_b32_int4"):
             if name not in synth.CONFIGS:
                 continue
             borrow = None
@@ -699,6 +705,8 @@ def run_ours(args, rank, world, local_rank):
                 borrow = wl_keep
             if name == "dsv2lite_b32_fp8":
                 borrow = kept.get("dsv2lite_fp8")
+            if name == "dsv2lite_b32_int4":
+                borrow = kept.get("dsv2lite_int4")
             try:
                 others[name] = short_run(torch, name, n_o, w_o, peak_hbm, h2d_peak_of, store_of=borrow, keep=kept)
             except Exception as ex:              # a workload that cannot run here must not lose the line

@@ -79,13 +79,14 @@ typedef struct {
                          /* the slots hold the FP8 bytes; at batch > 1 (I, I_shared        */
                          /* multiples of 64) a fetched block is widened, exactly, to bf16  */
                          /* operand tiles on arrival and the grouped GEMM is the bf16 one. */
-                         /* REMOE_INT4_G32 (batch 1; H 1024 or 2048): 4-bit codes in groups*/
+                         /* REMOE_INT4_G32 (H 1024 or 2048): 4-bit codes in groups         */
                          /* of 32 consecutive elements of a row, value = (code - 8) * the  */
                          /* group's bf16 scale; a stored row is H/2 bytes of codes (element*/
                          /* 2i in the low half of byte i) then H/32 scales, so a row takes */
                          /* 0.5625 H bytes: 3.6x fewer bytes per miss than bf16.  Router   */
-                         /* and shared gate bf16.                                          */
-  int32_t batch;         /* B sequences per step; B > 1 needs bf16 or FP8 weights and I, I_shared */
+                         /* and shared gate bf16.  At batch > 1 as for FP8: widened to     */
+                         /* bf16 operand tiles on arrival (one rounding to bf16 per weight)*/
+  int32_t batch;         /* B sequences per step; B > 1 needs bf16, FP8 or 4-bit weights and I, I_shared */
                          /* multiples of 8, B * K <= 1024                                   */
 } remoe_shape;
 

@@ -73,7 +73,8 @@ struct remoe_stack {
   int step_serial = 0;                    // never reset: stamps partial rows
   cudaEvent_t ev_resident = nullptr;
   bool use_tc = false;                     // batched experts on tcgen05 / TMEM, slots in operand-tile order
-  bool widen_fp8 = false;                  // batched stack over an FP8 host store: blocks are widened to bf16 on arrival
+  bool widen_fp8 = false;                  // batched stack over an FP8 / 4-bit host store: blocks are widened to bf16 on arrival
+  int host_wbytes = 0;                     // element tag of the host store (see weight_row_bytes)
   size_t fetch_bytes = 0, fetch_shared_bytes = 0;   // bytes of one routed / shared expert block in HOST memory
   char* stage_pool = nullptr;              // [2][C] channel-major landing area of fetched blocks (use_tc)
   size_t stage_bytes = 0;
@@ -399,7 +400,7 @@ int batched_waves(remoe_stack* s, BatchArgs& a, int l0, int l1, uint64_t* reside
         if (s->widen_fp8) {
           src_ptr.clear();
           for (size_t off : src_off) src_ptr.push_back(s->stage_pool + off);
-          CK(launch_widen_retile_tc(d, misses, src_ptr.data(), dst_ptr.data(), d.I, s->stream));
+          CK(launch_widen_retile_tc(d, s->host_wbytes, misses, src_ptr.data(), dst_ptr.data(), d.I, s->stream));
         } else {
           CK(launch_retile_tc(d, s->tc_maps, misses, src_off.data(), dst_ptr.data(), d.I, s->stream));
         }
@@ -633,10 +634,10 @@ int remoe_stack_create(const remoe_shape* sh, int32_t cache_slots, void* cuda_st
   // host store: bytes per element, 0 tagging the 4-bit grouped format
   const int wbytes = sh->weight_dtype == REMOE_BF16 ? 2
                      : sh->weight_dtype == REMOE_FP8_E4M3 ? 1 : sh->weight_dtype == REMOE_INT4_G32 ? 0 : 4;
-  if (sh->weight_dtype == REMOE_INT4_G32 && sh->batch > 1) return REMOE_E_UNSUPPORTED;
+
   const int rbytes = sh->weight_dtype == REMOE_F32 ? 4 : 2;
   // A batched stack over an FP8 store keeps its slots as bf16 operand tiles: fetched bytes are widened on arrival.
-  const bool widen = sh->weight_dtype == REMOE_FP8_E4M3 && sh->batch > 1;
+  const bool widen = (sh->weight_dtype == REMOE_FP8_E4M3 || sh->weight_dtype == REMOE_INT4_G32) && sh->batch > 1;
   const int dev_wbytes = widen ? 2 : wbytes;
   const long pairs = (long)sh->n_layers * (sh->top_k + sh->n_shared);
   if (sh->hidden > kMaxHidden || sh->n_routed > kMaxRouted || sh->top_k > 32 || cache_slots > kMaxSlots || cache_slots > sh->n_routed ||
@@ -680,6 +681,7 @@ int remoe_stack_create(const remoe_shape* sh, int32_t cache_slots, void* cuda_st
   s->fetch_bytes = (size_t)3 * d.I * weight_row_bytes(d.H, wbytes);
   s->fetch_shared_bytes = (size_t)3 * d.Is * weight_row_bytes(d.H, wbytes);
   s->widen_fp8 = widen;
+  s->host_wbytes = wbytes;
   const size_t L = d.L;
   char *router = nullptr, *sgw = nullptr, *shared = nullptr, *slots = nullptr;
 #define TRY(x) do { rc = (x); if (rc != REMOE_OK) return bail(rc); } while (0)
@@ -791,7 +793,7 @@ int remoe_load_shared(remoe_stack* s, int32_t layer, int32_t idx, const void* bl
     const size_t off = 0;
     if (s->widen_fp8) {
       const void* src = s->stage_pool;
-      CK(launch_widen_retile_tc(s->d, 1, &src, &dst, s->d.Is, s->stream));
+      CK(launch_widen_retile_tc(s->d, s->host_wbytes, 1, &src, &dst, s->d.Is, s->stream));
     } else {
       CK(launch_retile_tc(s->d, s->tc_maps, 1, &off, &dst, s->d.Is, s->stream));
     }

@@ -524,24 +524,27 @@ __global__ void __launch_bounds__(32) retile_kernel(const __grid_constant__ TcMa
   }
 }
 
-// ------------------------------------------------------------------------- FP8 widen + retile
-// A stack with an FP8 E4M3 host store (value = byte * 2^-8) at batch > 1 fetches FP8 bytes -- half of what
-// a bf16 block moves over the host link -- and keeps its slots as bf16 operand tiles, so the MMA kernel
-// above is the same.  This kernel does both steps at once for freshly fetched channel-major FP8 blocks:
-// every 16-byte piece of an operand tile is eight consecutive stored bytes of one row, widened exactly
-// (an E4M3 value times 2^-8 has at most 4 significant bits and fits bf16), written at the swizzled place
-// the tensor-map path would have put it.  One CTA per (64-channel group, block); plain loads and stores.
+// ------------------------------------------------------------------- low-precision widen + retile
+// A batched stack over an FP8 E4M3 (value = byte * 2^-8) or a 4-bit grouped host store fetches the stored bytes
+// -- a half or 0.28 of what a bf16 block moves over the host link -- and keeps its slots as bf16 operand tiles,
+// so the MMA kernel above is the same.  This kernel does both steps at once for freshly fetched channel-major
+// blocks: every 16-byte piece of an operand tile is eight consecutive stored elements of one row, widened to
+// bf16 and written at the swizzled place the tensor-map path would have put it.  FP8 widens exactly (an E4M3
+// value times 2^-8 has at most 4 significant bits); a 4-bit value (code - 8) * bf16 scale has up to 11 and is
+// rounded to nearest even once.  One CTA per (64-channel group, block); plain loads and stores.
 struct WidenArgs {
   int n, inter;
-  const unsigned char* src[kRetileJobs];   // channel-major FP8 block in the staging pool
+  const unsigned char* src[kRetileJobs];   // channel-major stored block in the staging pool
   char* dst[kRetileJobs];                  // destination block (slot or shared block), bf16 tile order
 };
 
-template <int H>
+// WB: 1 = FP8 E4M3 bytes, 0 = 4-bit grouped format
+template <int H, int WB>
 __global__ void __launch_bounds__(256) widen_retile_kernel(const __grid_constant__ WidenArgs r) {
   using G = TcGeo<H>;
   constexpr int T = G::kChunks + G::kTiles;
-  const unsigned char* src = r.src[blockIdx.y] + (size_t)blockIdx.x * kTcBlockCh * 3 * H;
+  constexpr size_t kRow = weight_row_bytes(H, WB);
+  const unsigned char* src = r.src[blockIdx.y] + (size_t)blockIdx.x * kTcBlockCh * 3 * kRow;
   char* dst = r.dst[blockIdx.y] + (size_t)blockIdx.x * T * kTileBytes;
   for (int q = threadIdx.x; q < T * 1024; q += 256) {
     const int t = q >> 10, line = (q >> 3) & 127, pos = q & 7;
@@ -552,14 +555,24 @@ __global__ void __launch_bounds__(256) widen_retile_kernel(const __grid_constant
     } else {                                             // A2 tile: two halves of 64 channel lines
       ch = line & 63; kind = 2; col = (t - G::kChunks) * 128 + (line >> 6) * 64 + c * 8;
     }
-    const uint2 b = __ldg(reinterpret_cast<const uint2*>(src + ((size_t)ch * 3 + kind) * H + col));
+    const unsigned char* row = src + ((size_t)ch * 3 + kind) * kRow;
     float f[8];
-    Elems<1>::pair(b.x & 0xffffu, f[0], f[1]); Elems<1>::pair(b.x >> 16, f[2], f[3]);
-    Elems<1>::pair(b.y & 0xffffu, f[4], f[5]); Elems<1>::pair(b.y >> 16, f[6], f[7]);
-    constexpr float k = WScale<1>::kDot;                 // the store's power-of-two scale
+    if constexpr (WB == 1) {
+      const uint2 b = __ldg(reinterpret_cast<const uint2*>(row + col));
+      Elems<1>::pair(b.x & 0xffffu, f[0], f[1]); Elems<1>::pair(b.x >> 16, f[2], f[3]);
+      Elems<1>::pair(b.y & 0xffffu, f[4], f[5]); Elems<1>::pair(b.y >> 16, f[6], f[7]);
+      constexpr float k = WScale<1>::kDot;               // the store's power-of-two scale
+#pragma unroll
+      for (int i = 0; i < 8; ++i) f[i] *= k;
+    } else {
+      const uint32_t w = __ldg(reinterpret_cast<const uint32_t*>(row + col / 2));        // eight codes
+      const float sc = __uint_as_float(
+          (uint32_t)__ldg(reinterpret_cast<const unsigned short*>(row + H / 2 + 2 * (col / 32))) << 16);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) f[i] = (float)((int)((w >> (4 * i)) & 0xfu) - 8) * sc;
+    }
     *reinterpret_cast<uint4*>(dst + (size_t)t * kTileBytes + line * 128 + pos * 16) =
-        make_uint4(pack_bf16(f[0] * k, f[1] * k), pack_bf16(f[2] * k, f[3] * k), pack_bf16(f[4] * k, f[5] * k),
-                   pack_bf16(f[6] * k, f[7] * k));
+        make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
   }
 }
 
@@ -641,8 +654,21 @@ cudaError_t launch_ffn_batched_tc(const BatchArgs& a, int grid, cudaStream_t st)
   return cudaErrorInvalidValue;
 }
 
-cudaError_t launch_widen_retile_tc(const DevStack& d, int n, const void* const* src, char* const* dst, int inter,
-                                   cudaStream_t st) {
+template <int WB>
+cudaError_t launch_widen(const DevStack& d, const WidenArgs& r, dim3 grid, cudaStream_t st) {
+  switch (d.H) {
+    case 256: widen_retile_kernel<256, WB><<<grid, 256, 0, st>>>(r); break;
+    case 512: widen_retile_kernel<512, WB><<<grid, 256, 0, st>>>(r); break;
+    case 1024: widen_retile_kernel<1024, WB><<<grid, 256, 0, st>>>(r); break;
+    case 2048: widen_retile_kernel<2048, WB><<<grid, 256, 0, st>>>(r); break;
+    default: return cudaErrorInvalidValue;
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_widen_retile_tc(const DevStack& d, int src_wbytes, int n, const void* const* src, char* const* dst,
+                                   int inter, cudaStream_t st) {
+  if (src_wbytes != 0 && src_wbytes != 1) return cudaErrorInvalidValue;
   for (int i0 = 0; i0 < n; i0 += kRetileJobs) {
     WidenArgs r{};
     r.n = n - i0 < kRetileJobs ? n - i0 : kRetileJobs;
@@ -653,14 +679,7 @@ cudaError_t launch_widen_retile_tc(const DevStack& d, int n, const void* const* 
       r.dst[i] = dst[i0 + i];
     }
     const dim3 grid(inter / kTcBlockCh, r.n);
-    switch (d.H) {
-      case 256: widen_retile_kernel<256><<<grid, 256, 0, st>>>(r); break;
-      case 512: widen_retile_kernel<512><<<grid, 256, 0, st>>>(r); break;
-      case 1024: widen_retile_kernel<1024><<<grid, 256, 0, st>>>(r); break;
-      case 2048: widen_retile_kernel<2048><<<grid, 256, 0, st>>>(r); break;
-      default: return cudaErrorInvalidValue;
-    }
-    const cudaError_t e = cudaGetLastError();
+    const cudaError_t e = src_wbytes == 1 ? launch_widen<1>(d, r, grid, st) : launch_widen<0>(d, r, grid, st);
     if (e != cudaSuccess) return e;
   }
   return cudaSuccess;

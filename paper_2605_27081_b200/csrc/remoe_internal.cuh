@@ -139,10 +139,11 @@ cudaError_t launch_ffn_batched_tc(const BatchArgs& a, int grid, cudaStream_t st)
 cudaError_t launch_retile_tc(const DevStack& d, const void* maps, int n, const size_t* src_offsets,
                              char* const* dst, int inter, cudaStream_t st);
 
-// FP8 host store at batch > 1: n channel-major FP8 E4M3 blocks (value = byte * 2^-8) at src[i] (device,
-// 8-byte aligned) are widened to bf16 and written to dst[i] in operand-tile order.  Host arrays.
-cudaError_t launch_widen_retile_tc(const DevStack& d, int n, const void* const* src, char* const* dst, int inter,
-                                   cudaStream_t st);
+// Low-precision host store at batch > 1: n channel-major stored blocks at src[i] (device, 8-byte aligned) --
+// src_wbytes 1: FP8 E4M3 bytes, value = byte * 2^-8; 0: the 4-bit grouped format -- are widened to bf16 and
+// written to dst[i] in operand-tile order.  Host arrays.
+cudaError_t launch_widen_retile_tc(const DevStack& d, int src_wbytes, int n, const void* const* src, char* const* dst,
+                                   int inter, cudaStream_t st);
 
 // Routes layers [layer0, layer0 + n_layers); `hidden_in`, `ids`, `gates` are the full [L, B, .] arrays.
 cudaError_t launch_route(const DevStack& d, const float* hidden_in, int* ids, float* gates,

@@ -101,6 +101,9 @@ CONFIGS = {
     "dsv2lite_b32": dict(
         shape=Shape(26, 2048, 64, 6, 1408, 2, 1408, 0, 0, 1, 32),
         cache_slots=32, steps=1024, rhos=(None,), seed=0),
+    "dsv2lite_b32_int4": dict(
+        shape=Shape(26, 2048, 64, 6, 1408, 2, 1408, 0, 0, 3, 32),
+        cache_slots=32, steps=1024, rhos=(None,), seed=0),
     "dsv2lite_b32_fp8": dict(
         shape=Shape(26, 2048, 64, 6, 1408, 2, 1408, 0, 0, 2, 32),
         cache_slots=32, steps=1024, rhos=(None,), seed=0),

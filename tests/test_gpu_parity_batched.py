@@ -65,13 +65,24 @@ def test_batched_fp8_store(shape, c, rho):
     """FP8 E4M3 host store under a batched stack: a miss moves half the bytes; the fetched block is widened
     (exactly) to bf16 operand tiles on arrival, so outputs match the oracle on the FP8-denoted values."""
     from paper_2605_27081_b200 import binding as B
-    chk, deepest = _run(shape, c, rho, steps=10, seed=6)
+    chk, deepest = _run(shape, c, rho, steps=8 if shape.hidden == 2048 else 10, seed=6)
     assert chk.max_out_err <= 2e-2
     if shape.batch * shape.top_k > 2 * c:
         assert deepest > c
     # intermediate sizes the tensor-core path is not built for have no FP8 batched variant
     rc, _ = B.remoe_stack_create(synth.Shape(2, 512, 16, 2, 40, 0, 0, 0, 0, 2, 4), 6)
     assert rc == B.REMOE_E_UNSUPPORTED
+
+
+@pytest.mark.parametrize("shape,c,rho", [
+    (synth.Shape(3, 1024, 24, 3, 128, 2, 64, 1, 0, 3, 12), 8, None),     # union far above capacity, sigmoid gate
+    (synth.Shape(2, 2048, 64, 6, 192, 2, 192, 0, 0, 3, 32), 32, None),   # the serving configuration's layer shape
+])
+def test_batched_int4_store(shape, c, rho):
+    """4-bit grouped host store under a batched stack: a miss moves 0.28 of the bf16 bytes; the fetched block is
+    widened to bf16 operand tiles on arrival (one rounding to bf16 per weight, inside the bf16 tolerance)."""
+    chk, deepest = _run(shape, c, rho, steps=8, seed=7)
+    assert chk.max_out_err <= 2e-2 and deepest > c
 
 
 def test_batched_other_policy():

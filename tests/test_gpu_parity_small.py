@@ -86,7 +86,7 @@ def test_int4_store_limits():
     from paper_2605_27081_b200 import binding as B
     rc, _ = B.remoe_stack_create(synth.Shape(2, 512, 16, 2, 32, 0, 0, 0, 0, 3, 1), 4)      # H not 1024 / 2048
     assert rc == B.REMOE_E_UNSUPPORTED
-    rc, _ = B.remoe_stack_create(synth.Shape(2, 1024, 16, 2, 64, 0, 0, 0, 0, 3, 4), 4)     # batched
+    rc, _ = B.remoe_stack_create(synth.Shape(2, 1024, 16, 2, 40, 0, 0, 0, 0, 3, 4), 4)     # batched needs I % 64 == 0
     assert rc == B.REMOE_E_UNSUPPORTED
 
 
