@@ -85,6 +85,19 @@ def test_batched_int4_store(shape, c, rho):
     assert chk.max_out_err <= 2e-2 and deepest > c
 
 
+@pytest.mark.parametrize("seed", range(10))
+def test_random_batched_shapes(seed):
+    """Valid batched stacks drawn at random (both expert kernels, all three host formats, any capacity from
+    one slot to all experts, batch sizes that are no multiple of a token tile)."""
+    import numpy as np
+    from test_gpu_parity_small import _random_shape
+    rng = np.random.default_rng(2000 + seed)
+    shape, c = _random_shape(rng, batched=True)
+    chk, _ = _run(shape, c, None if rng.random() < 0.5 else 0.6, steps=6, seed=seed, dense_steps=1,
+                  policy=int(rng.integers(0, 3)))
+    assert chk.max_out_err <= 2e-2
+
+
 def test_batched_other_policy():
     _run(synth.Shape(2, 256, 16, 2, 64, 0, 0, 0, 0, 1, 6), 5, 0.4, steps=30, seed=4, dense_steps=0, policy=2)
 

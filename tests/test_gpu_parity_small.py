@@ -90,6 +90,35 @@ def test_int4_store_limits():
     assert rc == B.REMOE_E_UNSUPPORTED
 
 
+def _random_shape(rng, batched):
+    """A valid stack shape drawn at random: element type, width, expert count, top-K, capacity, intermediate
+    sizes, shared experts, gate, renormalisation."""
+    dt = int(rng.choice([1, 2, 3] if batched else [0, 1, 2, 3]))
+    widths = {0: [128, 256, 512, 1024], 1: [256, 512, 1024, 2048], 2: [512, 1024, 2048], 3: [1024, 2048]}[dt]
+    H = int(rng.choice(widths))
+    N = int(rng.integers(2, 41))
+    K = int(rng.integers(1, min(N, 8) + 1))
+    B = int(rng.integers(2, 25)) if batched else 1
+    C = int(rng.integers(K if not batched else 1, N + 1))
+    tc_only = batched and dt != 1                        # low-precision batched stacks run on the tensor-core path only
+    step = 64 if tc_only or (batched and rng.random() < 0.5) else (8 if batched else 1)
+    inter = step * int(rng.integers(1, 3 if step == 64 else (12 if step == 8 else 90)))
+    S = int(rng.integers(0, 3))
+    Is = step * int(rng.integers(1, 3 if step == 64 else (8 if step == 8 else 60))) if S else 0
+    return synth.Shape(int(rng.integers(1, 5)), H, N, K, inter, S, Is, int(rng.integers(0, 2)) if S else 0,
+                       int(rng.integers(0, 2)), dt, B), C
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_random_batch1_shapes(seed):
+    rng = np.random.default_rng(1000 + seed)
+    shape, c = _random_shape(rng, batched=False)
+    policy = int(rng.integers(0, 3))
+    beta = float(rng.choice([0.0, 0.0, 0.4]))
+    _run(shape, c, float(rng.choice([0.0, 0.5, 0.9])), steps=10, seed=seed, dense_steps=1, host_api_every=4,
+         policy=policy, beta=beta)
+
+
 def test_many_layers_span_ctas():
     """Enough rows that CTAs cross expert and layer boundaries in the streaming kernel."""
     shape = synth.Shape(12, 512, 16, 4, 300, 1, 300, 0, 0, 1, 1)
