@@ -398,6 +398,28 @@ def measure_h2d(torch, nbytes, reps=12, store=None):
     return best
 
 
+def measure_copy_peak(torch):
+    """This box's device-to-device copy rate (read + write bytes, GB/s), the way the stored peak was taken:
+    b.copy_(a) over 1 Gi bf16 elements, best of 10, CUDA events.  Boxes of the pool differ by a few per cent."""
+    n = 1 << 30
+    a = torch.empty(n, dtype=torch.bfloat16, device="cuda")
+    b = torch.empty_like(a)
+    a.zero_()
+    best = 0.0
+    for rep in range(12):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        b.copy_(a)
+        e1.record()
+        torch.cuda.synchronize()
+        if rep >= 2:
+            best = max(best, 2 * n * 2 / e0.elapsed_time(e1) / 1e6)
+    del a, b
+    torch.cuda.empty_cache()
+    return best
+
+
 def reduce_over_ranks(dist, maxima: dict, sums: dict, device):
     """Whole-job figures of N independent replicas: times are the maximum over ranks, counts the
     sum.  `dist` is torch.distributed (initialised) or None for a single process."""
@@ -533,6 +555,7 @@ def run_ours(args, rank, world, local_rank):
         return h2d_cache[nbytes]
 
     h2d_peak = h2d_peak_of(S_e, wl._store_t)
+    copy_here = measure_copy_peak(torch) if rank == 0 else None
 
     def barrier():
         torch.cuda.synchronize()
@@ -638,7 +661,8 @@ def run_ours(args, rank, world, local_rank):
                 "peak_kind": f"of {peak_kind}", "kernel": kname + " resident phase",
                 "note": "the measured peak is a copy (reads and writes); a read-only stream can run a few per cent above it",
                 "launches": kr_n, "avg_launch_ms": kr_ms / max(1, kr_n), "bytes_per_launch": kr_b / max(1, kr_n),
-                "frac_of_nominal_8TBs": ach / NOMINAL_HBM_GBS}
+                "frac_of_nominal_8TBs": ach / NOMINAL_HBM_GBS,
+                "copy_peak_this_box": copy_here, "frac_of_this_box_copy": ach / copy_here if copy_here else None}
     miss_phase = {"launches": km_n, "avg_launch_us": km_ms * 1e3 / max(1, km_n),
                   "achieved_gbs": km_b / (km_ms / 1e3) / 1e9 if km_ms > 0 else 0.0}
 

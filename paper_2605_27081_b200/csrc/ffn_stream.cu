@@ -151,21 +151,49 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(const __grid_co
   stream::stream_rows<WB, H>(wk, prefix, P, r0, r1, ring, a.spin_limit ? a.spin_limit : kSpinLimit, a.lose_row1);
 }
 
-__global__ void __launch_bounds__(256) combine_kernel(FfnArgs a, float* __restrict__ hidden_out, int layer0,
-                                                      float* __restrict__ chain_in) {
+// Fixed-order sum of a layer's per-CTA partial rows (resident phase by ascending CTA, then miss phase by ascending
+// CTA).  One CTA per (256-column slice, layer): 64 threads across the slice's float4 pieces times 16 row groups; a
+// thread adds the pieces of its group's rows in order, the groups are then added in order.  Splitting the rows
+// over groups keeps the chain of dependent additions (and of memory round trips) 16 times shorter than one
+// thread per column walking all rows.
+constexpr int kCombineGroups = 16;
+__global__ void __launch_bounds__(1024) combine_kernel(FfnArgs a, float* __restrict__ hidden_out, int layer0,
+                                                       float* __restrict__ chain_in) {
+  __shared__ float4 red[kCombineGroups][64];
   const DevStack& d = a.d;
   const int l = layer0 + blockIdx.y;
-  const int c = blockIdx.x * 256 + threadIdx.x;
-  if (c >= d.H) return;
-  float t = 0.f;
-  for (int phase = 0; phase < 2; ++phase) {
-    const int* cb = a.contrib + ((size_t)phase * d.L + l) * 2;
-    const int lo = cb[0], hi = cb[1];
-    const float* p = a.partial + (((size_t)phase * d.L + l) * a.grid_cap) * d.H + c;
-    for (int b = lo; b <= hi; ++b) t += p[(size_t)b * d.H];
+  const int c4 = threadIdx.x & 63, rg = threadIdx.x >> 6;
+  const int col = blockIdx.x * 256 + c4 * 4;
+  const bool active = col < d.H;
+  const int* cb0 = a.contrib + ((size_t)0 * d.L + l) * 2;
+  const int* cb1 = a.contrib + ((size_t)1 * d.L + l) * 2;
+  const int lo0 = cb0[0], hi0 = cb0[1], lo1 = cb1[0], hi1 = cb1[1];
+  const int n0 = hi0 >= lo0 ? hi0 - lo0 + 1 : 0, n1 = hi1 >= lo1 ? hi1 - lo1 + 1 : 0;
+  const int n = n0 + n1, per = (n + kCombineGroups - 1) / kCombineGroups;
+  const int ra = min(n, rg * per), rb = min(n, ra + per);
+  float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (active) {
+    const float* p0 = a.partial + ((size_t)(0 * d.L + l) * a.grid_cap) * d.H + col;
+    const float* p1 = a.partial + ((size_t)(1 * d.L + l) * a.grid_cap) * d.H + col;
+#pragma unroll 8
+    for (int r = ra; r < rb; ++r) {
+      const float* src = r < n0 ? p0 + (size_t)(lo0 + r) * d.H : p1 + (size_t)(lo1 + r - n0) * d.H;
+      const float4 v = __ldg(reinterpret_cast<const float4*>(src));
+      t.x += v.x; t.y += v.y; t.z += v.z; t.w += v.w;
+    }
   }
-  hidden_out[(size_t)l * d.H + c] = t;
-  if (chain_in) chain_in[(size_t)(l + 1) * d.H + c] = chain_in[(size_t)l * d.H + c] + t;
+  red[rg][c4] = t;
+  __syncthreads();
+  if (rg != 0 || !active) return;
+  float4 o = red[0][c4];
+#pragma unroll
+  for (int g = 1; g < kCombineGroups; ++g) { o.x += red[g][c4].x; o.y += red[g][c4].y; o.z += red[g][c4].z; o.w += red[g][c4].w; }
+  *reinterpret_cast<float4*>(hidden_out + (size_t)l * d.H + col) = o;
+  if (chain_in) {
+    const float4 hp = *reinterpret_cast<const float4*>(chain_in + (size_t)l * d.H + col);
+    *reinterpret_cast<float4*>(chain_in + (size_t)(l + 1) * d.H + col) =
+        make_float4(hp.x + o.x, hp.y + o.y, hp.z + o.z, hp.w + o.w);
+  }
 }
 
 __global__ void __launch_bounds__(256) rmsnorm_kernel(const float* __restrict__ h_all, float* __restrict__ x_all,
@@ -255,7 +283,7 @@ cudaError_t launch_rmsnorm(const float* h, float* x, int H, int rows, cudaStream
 cudaError_t launch_combine(const FfnArgs& a, float* hidden_out, int layer0, int n_layers, float* chain_in,
                            cudaStream_t st) {
   dim3 grid((a.d.H + 255) / 256, n_layers);
-  combine_kernel<<<grid, 256, 0, st>>>(a, hidden_out, layer0, chain_in);
+  combine_kernel<<<grid, 1024, 0, st>>>(a, hidden_out, layer0, chain_in);
   return cudaGetLastError();
 }
 
