@@ -208,6 +208,12 @@ int remoe_decode_step_host(remoe_stack*, const float* hidden_in_host, float* hid
 int remoe_last_step_trace(remoe_stack*, int32_t* requests, int32_t* hit, int32_t* slot,
                           int32_t* evicted, int32_t* n_unique);
 
+/* The directory of one layer as it stands after the most recent step (a debugging aid; App. A.1: the cache
+ * state C_{t+1}).  Host arrays, any may be NULL: expert_of_slot [C] (-1 = empty slot), stamp [C] (the slot's
+ * place in the layer's touch order: last touch under LRU and LFU, insertion under FIFO; 0 = never used),
+ * use_count [C] (selections since insertion; decides under LFU).  Waits for the stack's stream. */
+int remoe_cache_snapshot(remoe_stack*, int32_t layer, int32_t* expert_of_slot, uint64_t* stamp, uint32_t* use_count);
+
 /* Counters for one layer, or summed over layers with layer = -1 (App. E.2.4: #uMiss, uHR =
  * uniq_hits / (uniq_hits + uniq_misses), tHR likewise).  Waits for the stack's stream; like the
  * other statistics calls it fills its outputs and returns DEVICE_FLAG if a kernel has set the error word. */

@@ -26,7 +26,7 @@ EXPORTS = [
     "remoe_reuse_stats", "remoe_cache_reset", "remoe_set_policy", "remoe_set_reroute_beta",
     "remoe_set_profiling", "remoe_kernel_time", "remoe_launch_count", "remoe_last_cuda_error", "remoe_stack_destroy",
     "remoe_strerror", "remoe_expert_ffn_static", "remoe_reuse_mass", "remoe_step_history", "remoe_tpot_proxy", "remoe_decode_step_chained",
-    "remoe_expert_load", "remoe_decode_steps", "remoe_order_check_counts",
+    "remoe_expert_load", "remoe_decode_steps", "remoe_order_check_counts", "remoe_cache_snapshot",
 ]
 
 
@@ -77,6 +77,7 @@ def lib():
         L.remoe_set_profiling.argtypes = [vp, i32]
         L.remoe_kernel_time.argtypes = [vp, i32, C.POINTER(C.c_double), C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
         L.remoe_launch_count.argtypes = [vp, C.POINTER(C.c_uint64)]
+        L.remoe_cache_snapshot.argtypes = [vp, i32, vp, vp, vp]
         L.remoe_order_check_counts.argtypes = [vp, C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
         L.remoe_expert_ffn_static.argtypes = [i32, i32, i32, C.POINTER(vp), C.POINTER(i32), C.POINTER(C.c_float),
                                               vp, vp, vp]
@@ -205,6 +206,10 @@ def remoe_launch_count(h):
     n = C.c_uint64()
     rc = lib().remoe_launch_count(h, C.byref(n))
     return rc, int(n.value)
+
+
+def remoe_cache_snapshot(h, layer, expert_of_slot, stamp, use_count):
+    return lib().remoe_cache_snapshot(h, int(layer), _ptr(expert_of_slot), _ptr(stamp), _ptr(use_count))
 
 
 def remoe_order_check_counts(h):
@@ -364,6 +369,14 @@ class Stack:
         rc, n = remoe_launch_count(self.h)
         self._ck(rc, "remoe_launch_count")
         return n
+
+    def cache_snapshot(self, layer):
+        """(expert_of_slot [C] int32, stamp [C] uint64, use_count [C] uint32) of one layer."""
+        eos = np.empty(self.cache_slots, np.int32)
+        stamp = np.empty(self.cache_slots, np.uint64)
+        freq = np.empty(self.cache_slots, np.uint32)
+        self._ck(remoe_cache_snapshot(self.h, layer, eos, stamp, freq), "remoe_cache_snapshot")
+        return eos, stamp, freq
 
     def order_check_counts(self):
         rc, c, v = remoe_order_check_counts(self.h)

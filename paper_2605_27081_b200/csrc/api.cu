@@ -1277,6 +1277,17 @@ int remoe_last_step_trace(remoe_stack* s, int32_t* req, int32_t* hit, int32_t* s
   return check_device_flag(s);
 }
 
+int remoe_cache_snapshot(remoe_stack* s, int32_t layer, int32_t* eos, uint64_t* stamp, uint32_t* use_count) {
+  if (!s || layer < 0 || layer >= s->d.L) return REMOE_E_ARG;
+  ON_STACK_DEVICE(s);
+  CK(cudaStreamSynchronize(s->stream));
+  const size_t C = s->d.C, off = (size_t)layer * C;
+  if (eos) CK(cudaMemcpy(eos, s->d.expert_of_slot + off, C * sizeof(int), cudaMemcpyDeviceToHost));
+  if (stamp) CK(cudaMemcpy(stamp, s->d.stamp + off, C * sizeof(unsigned long long), cudaMemcpyDeviceToHost));
+  if (use_count) CK(cudaMemcpy(use_count, s->d.freq + off, C * sizeof(unsigned), cudaMemcpyDeviceToHost));
+  return fetch_device_flag(s);
+}
+
 int remoe_cache_stats(remoe_stack* s, int32_t layer, remoe_cache_counters* out) {
   if (!s || !out || layer < -1 || layer >= s->d.L) return REMOE_E_ARG;
   ON_STACK_DEVICE(s);

@@ -240,7 +240,20 @@ class StepChecker:
         assert list(tr["requests"][l][:K]) == r["requests"][l] and list(tr["slot"][l][:K]) == r["slot"][l]
         return r
 
+    def check_directory(self):
+        """The library's directory of every layer against the oracle's cache object: which expert sits in
+        which slot, the slots' places in the touch order and their use counts (the state C_{t+1} itself, not
+        only the trace that led to it)."""
+        for l in range(self.L):
+            eos, stamp, freq = self.wl.stack.cache_snapshot(l)
+            c = self.o.caches[l]
+            assert list(eos) == c.expert_of_slot, f"layer {l}: slot contents differ"
+            assert [int(x) for x in stamp] == c.stamp, f"layer {l}: touch order differs"
+            occupied = [s for s, e in enumerate(c.expert_of_slot) if e >= 0]
+            assert [int(freq[s]) for s in occupied] == [c.freq[s] for s in occupied], f"layer {l}: use counts differ"
+
     def check_counters(self):
+        self.check_directory()
         st = self.wl.stack
         o = self.o
         tot = st.cache_stats(-1)

@@ -24,6 +24,8 @@ def _run(shape, cache_slots, rho, steps, seed=0, dense_steps=1, policy=None):
         for t in range(steps):
             r, _ = chk.step(hs.step(), ffn="dense" if t < dense_steps else "selected", host_api=(t % 5 == 4))
             deepest = max(deepest, max(len(q) for q in r["requests"]))
+            if t % 3 == 2:
+                chk.check_directory()
         chk.check_counters()
         return chk, deepest
     finally:

@@ -27,6 +27,8 @@ def _run(shape, cache_slots, rho, steps, seed=0, dense_steps=2, host_api_every=0
             h = hs.step()
             host = bool(host_api_every) and t % host_api_every == host_api_every - 1
             last, _ = chk.step(h, ffn="dense" if t < dense_steps else "selected", host_api=host)
+            if t % 4 == 3:
+                chk.check_directory()
         chk.check_counters()
         o, p, ir = wl.stack.reuse_stats(-1, want_last_ir=True)
         exp = last["overlap"].reshape(-1)
