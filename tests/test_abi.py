@@ -32,3 +32,18 @@ def test_struct_layouts_match_header():
     body = re.search(r"typedef struct \{(.*?)\} remoe_shape;", text, flags=re.S).group(1)
     fields = re.findall(r"int32_t\s+([a-z_]+);", body)
     assert fields == [n for n, _ in binding.remoe_shape._fields_]
+
+
+def test_header_is_plain_c(tmp_path):
+    """The boundary is a C ABI: the header must compile as C99 on its own, without warnings."""
+    import shutil
+    import subprocess
+    cc = shutil.which("gcc") or shutil.which("cc")
+    if cc is None:
+        import pytest
+        pytest.skip("no C compiler")
+    src = tmp_path / "use_header.c"
+    src.write_text('#include "remoe.h"\nint main(void) { remoe_shape s; remoe_cache_counters c; (void)s; (void)c; return REMOE_OK; }\n')
+    res = subprocess.run([cc, "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-fsyntax-only",
+                          "-I", os.path.join(ROOT, "include"), str(src)], capture_output=True, text=True)
+    assert res.returncode == 0, res.stderr
