@@ -403,8 +403,7 @@ def measure_copy_peak(torch):
     b.copy_(a) over 1 Gi bf16 elements, best of 10, CUDA events.  Boxes of the pool differ by a few per cent."""
     n = 1 << 30
     a = torch.empty(n, dtype=torch.bfloat16, device="cuda")
-    b = torch.empty_like(a)
-    a.zero_()
+    b = torch.empty_like(a)                      # contents do not matter for a copy
     best = 0.0
     for rep in range(12):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
