@@ -350,6 +350,12 @@ int batched_waves(remoe_stack* s, BatchArgs& a, int l0, int l1, uint64_t* reside
   std::vector<size_t> src_off;
   std::vector<char*> dst_ptr;
   std::vector<const void*> src_ptr;
+  struct Fetch {
+    const char* src;       // the expert's block in host memory
+    char* slot;            // its cache slot
+    int j;                 // its place in the trace
+  };
+  std::vector<Fetch> group;
   for (int dep = 0; dep <= max_depth; ++dep) {
     if (dep == 1 && !staged) {
       CK(cudaStreamWaitEvent(s->copy_stream, s->ev_resident, 0));   // displaced hits are done
@@ -361,32 +367,50 @@ int batched_waves(remoe_stack* s, BatchArgs& a, int l0, int l1, uint64_t* reside
       int misses = 0, half = 0;
       src_off.clear();
       dst_ptr.clear();
+      group.clear();
       for (int i = 0; i < t_nu[l]; ++i) {
         const int j = l * BK + i;
         if (t_hit[j] || t_depth[j] != dep) continue;
-        char* slot = d.slots + ((size_t)l * d.C + t_slot[j]) * d.slot_bytes;
-        char* land = slot;
-        if (staged) {
-          if (!misses) {
-            // the half's previous user is the group before last: its retile is already enqueued
-            half = (int)(s->stage_group++ & 1);
-            if (s->stage_used[half]) {
-              CK(cudaStreamWaitEvent(s->copy_stream, s->ev_stage[half], 0));
-              l_wait(s, kStCopy, s->ev_stage[half]);
-            }
-          }
-          if (misses >= d.C) return REMOE_E_DEVICE_FLAG;         // more misses of one depth than slots: bad trace
-          src_off.push_back(((size_t)half * d.C + misses) * s->fetch_bytes);
-          dst_ptr.push_back(slot);
-          land = s->stage_pool + src_off.back();
-        } else if (!misses && dep >= 1 && had[(size_t)(dep - 1) * d.L + l]) {
-          CK(cudaStreamWaitEvent(s->copy_stream, ev_comp(dep - 1, l), 0));        // displaced misses are done
-          l_wait(s, kStCopy, ev_comp(dep - 1, l));
+        group.push_back({static_cast<const char*>(s->host_ptrs[(size_t)l * d.N + t_req[j]]),
+                         d.slots + ((size_t)l * d.C + t_slot[j]) * d.slot_bytes, j});
+      }
+      if (staged && !group.empty()) {
+        if ((int)group.size() > d.C) return REMOE_E_DEVICE_FLAG;   // more misses of one depth than slots: bad trace
+        // the half's previous user is the group before last: its retile is already enqueued
+        half = (int)(s->stage_group++ & 1);
+        if (s->stage_used[half]) {
+          CK(cudaStreamWaitEvent(s->copy_stream, s->ev_stage[half], 0));
+          l_wait(s, kStCopy, s->ev_stage[half]);
         }
-        CK(cudaMemcpyAsync(land, s->host_ptrs[(size_t)l * d.N + t_req[j]], s->fetch_bytes, cudaMemcpyHostToDevice,
-                           s->copy_stream));
-        l_write(s, l_op(s, kStCopy), staged ? stage_cell(s, half, misses) : slot_cell(s, l, t_slot[j]), "miss fetch");
-        ++misses;
+        // The landing places in the staging pool are ours to choose: the group's blocks are laid down in the
+        // order of their host addresses, so blocks that are neighbours in host memory are neighbours in the pool
+        // and go over the link as one copy (the copy engine loses a few microseconds per copy command).
+        std::sort(group.begin(), group.end(), [](const Fetch& x, const Fetch& y) { return x.src < y.src; });
+        for (size_t k = 0; k < group.size();) {
+          size_t run = 1;
+          while (k + run < group.size() && group[k + run].src == group[k].src + run * s->fetch_bytes) ++run;
+          const size_t off = ((size_t)half * d.C + k) * s->fetch_bytes;
+          CK(cudaMemcpyAsync(s->stage_pool + off, group[k].src, run * s->fetch_bytes, cudaMemcpyHostToDevice,
+                             s->copy_stream));
+          const LOp oc = l_op(s, kStCopy);
+          for (size_t r = 0; r < run; ++r) {
+            src_off.push_back(off + r * s->fetch_bytes);
+            dst_ptr.push_back(group[k + r].slot);
+            l_write(s, oc, stage_cell(s, half, (int)(k + r)), "miss fetch");
+          }
+          k += run;
+        }
+        misses = (int)group.size();
+      } else {
+        for (const Fetch& f : group) {
+          if (!misses && dep >= 1 && had[(size_t)(dep - 1) * d.L + l]) {
+            CK(cudaStreamWaitEvent(s->copy_stream, ev_comp(dep - 1, l), 0));        // displaced misses are done
+            l_wait(s, kStCopy, ev_comp(dep - 1, l));
+          }
+          CK(cudaMemcpyAsync(f.slot, f.src, s->fetch_bytes, cudaMemcpyHostToDevice, s->copy_stream));
+          l_write(s, l_op(s, kStCopy), slot_cell(s, l, t_slot[f.j]), "miss fetch");
+          ++misses;
+        }
       }
       if (!misses) continue;
       had[(size_t)dep * d.L + l] = 1;
@@ -407,12 +431,9 @@ int batched_waves(remoe_stack* s, BatchArgs& a, int l0, int l1, uint64_t* reside
         s->kernel_launches += (misses + 63) / 64;
         if (s->ledger) {
           const LOp ot = l_op(s, kStCompute);             // reads the staging half, rewrites the slots
-          int m = 0;
-          for (int i = 0; i < t_nu[l]; ++i) {
-            const int j = l * BK + i;
-            if (t_hit[j] || t_depth[j] != dep) continue;
-            l_read(s, ot, stage_cell(s, half, m++), "retile");
-            l_write(s, ot, slot_cell(s, l, t_slot[j]), "retile");
+          for (size_t k = 0; k < group.size(); ++k) {
+            l_read(s, ot, stage_cell(s, half, (int)k), "retile");
+            l_write(s, ot, slot_cell(s, l, t_slot[group[k].j]), "retile");
           }
         }
         CK(cudaEventRecord(s->ev_stage[half], s->stream));
